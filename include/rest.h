@@ -1,0 +1,192 @@
+/*
+ * rest.h - C ABI of the GPU hot path of one REST decoding step
+ * (Retrieval-Based Speculative Decoding, arXiv 2311.08252).
+ *
+ * Draft side:   rest_datastore_create, rest_draft          (Sec. 3.2, Algorithms 1 and 2)
+ * Verify side:  rest_tree_attention, rest_accept           (Sec. 3.2, draft verification / acceptance)
+ *
+ * Conventions
+ *   - Every pointer named d_* is a DEVICE pointer owned by the caller.  The library borrows
+ *     it for the duration of the call (the datastore handle: for its lifetime), never frees
+ *     it and never allocates device memory.  Scratch space is passed in by the caller; its
+ *     size comes from the matching *_workspace_bytes query.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and return
+ *     without synchronising (rest_datastore_create with REST_DS_VALIDATE is the exception).
+ *   - Host-checkable problems return a non-zero rest_status before anything is launched.
+ *     Data-dependent problems are reported per context in d_status and give an empty tree.
+ *     Nothing aborts, traps or throws.
+ *   - All integer outputs are fully determined by the inputs (no dependence on scheduling).
+ */
+#ifndef REST_H_
+#define REST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t rest_status;
+enum {
+  REST_OK = 0,
+  REST_INVALID_ARG = 1,         /* null pointer, negative size, inconsistent shapes          */
+  REST_UNSUPPORTED = 2,         /* outside the limits listed at rest_draft / rest_tree_attention */
+  REST_WORKSPACE_TOO_SMALL = 3,
+  REST_CUDA_ERROR = 4,          /* a CUDA runtime call failed; see rest_last_cuda_error()    */
+  REST_BAD_DATASTORE = 5        /* validation found an unsorted / non-permutation suffix array
+                                   or a token outside [0, vocab)                              */
+};
+
+/* Per-context codes written to d_status by rest_draft. */
+enum {
+  REST_CTX_OK = 0,
+  REST_CTX_BAD_TOKEN = 1,       /* one of the last n_max context tokens is outside [0, vocab) */
+  REST_CTX_BAD_DATASTORE = 2,   /* suffix-array entry out of range, or gathered continuations
+                                   not in lexicographic order                                 */
+  REST_CTX_INTERNAL = 3
+};
+
+enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1 };
+enum { REST_DS_VALIDATE = 1u };
+
+/* Limits of this implementation. */
+enum {
+  REST_MAX_SUFFIX = 16,   /* n_max */
+  REST_MAX_M = 16,        /* continuation length */
+  REST_MAX_N = 128,       /* draft tokens per tree */
+  REST_MAX_K = 32768,     /* candidates per context */
+  REST_HEAD_DIM = 128
+};
+
+typedef struct rest_datastore rest_datastore;   /* opaque host object holding device pointers */
+
+/* Draft hyper-parameters (Sec. 4.1 "Hyperparameters": n_max = 16, m = 10, c = 64).
+ *   n_max, n_min  longest / shortest context suffix tried by Algorithm 1 (1 <= n_min <= n_max <= 16)
+ *   K             cap on the number of continuation candidates used per context (1..32768)
+ *   m             continuation length (1..16)
+ *   N             maximum number of draft tokens, the paper's c (1..128)
+ *   sample_mode   which K of cnt > K matches are used: REST_SAMPLE_STRIDED takes suffix-array
+ *                 slot lo + floor(j*cnt/K), REST_SAMPLE_FIRST_K takes lo + j, j = 0..K-1      */
+typedef struct {
+  int32_t n_max, n_min, K, m, N, sample_mode;
+} rest_draft_params;
+
+/*
+ * Datastore (Sec. 3.2 "Datastore construction" and "Retrieving from the datastore": a token
+ * stream whose every position is a (context, continuation) pair, indexed by a suffix array).
+ *
+ *   d_tokens   int32[n_tokens], values in [0, vocab), vocab < 2^31
+ *   d_sa       int32[n_tokens] (sa_bytes = 4, n_tokens < 2^31) or int64[n_tokens] (sa_bytes = 8):
+ *              start positions of all suffixes in lexicographic order of their tokens (compared
+ *              as unsigned integers, a suffix that is a proper prefix of another sorts first).
+ *              Only the order on the first n_max + m tokens matters to rest_draft.
+ *   flags      REST_DS_VALIDATE: check on the device that d_sa is a permutation ordered on the
+ *              first 32 tokens and that tokens are in range; needs d_aux of
+ *              rest_datastore_aux_bytes() bytes; synchronises `stream`; returns
+ *              REST_BAD_DATASTORE on failure.  Without the flag d_aux may be NULL.
+ *   out        receives a host handle; free it with rest_datastore_destroy (device arrays stay
+ *              the caller's).
+ */
+size_t rest_datastore_aux_bytes(uint64_t n_tokens, int32_t sa_bytes, uint32_t vocab);
+rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n_tokens, const void* d_sa,
+                                  int32_t sa_bytes, uint32_t vocab, uint32_t flags, void* d_aux,
+                                  size_t aux_bytes, void* stream, rest_datastore** out);
+void rest_datastore_destroy(rest_datastore* ds);
+
+/*
+ * rest_draft - Algorithm 1 (longest-suffix exact-match retrieval), Algorithm 2 (Trie weights,
+ * the c heaviest nodes) and the breadth-first pseudo sequence with its tree-attention mask
+ * (Sec. 3.2 "Draft verification"), for B independent contexts.
+ *
+ * Per context b:
+ *   1. n runs from min(n_max, ctx_len[b]) down to n_min; q = last n context tokens; [lo, hi) is
+ *      the suffix-array range of suffixes starting with q; the first non-empty range wins.
+ *      No match (or ctx_len < n_min): empty tree, match_n = 0.  That is not an error.
+ *   2. Candidates: the min(hi-lo, K) sampled slots (see sample_mode); candidate j is the up to m
+ *      tokens that follow the match, cut at the end of the token stream.
+ *   3. Trie node = distinct non-empty prefix of a candidate; weight = number of candidates
+ *      having that prefix.  Kept: the N largest by (weight desc, depth asc, token path asc).
+ *   4. Output order: by depth, then token path (breadth first, siblings ascending by token).
+ *
+ *   d_ctx        int32, context b starts at d_ctx + b*ctx_stride and holds ctx_len[b] tokens
+ *   d_tokens     int32[B,N]  draft tokens;           unused slots -1
+ *   d_parents    int32[B,N]  index of the parent node, -1 for children of the root; unused -1
+ *   d_depth      int32[B,N]  1-based depth;          unused 0
+ *   d_pos_ids    int32[B,N]  ctx_len + depth - 1;    unused ctx_len
+ *   d_mask       uint32[B,N,ceil(N/32)]  bit (j & 31) of word (j >> 5) of row i is set iff node
+ *                j is node i or an ancestor of i; unused rows hold their own bit only
+ *   d_n_nodes    int32[B]
+ *   d_match_n    int32[B]    matched suffix length (0 = none)
+ *   d_match_range int64[B,2] lo, hi of the matched suffix-array range
+ *   d_node_count int32[B,N]  weight of each kept node (may be NULL)
+ *   d_status     int32[B]    REST_CTX_* code
+ *   d_ws         scratch of rest_draft_workspace_bytes() bytes (may be NULL when that is 0)
+ */
+size_t rest_draft_workspace_bytes(const rest_draft_params* params, int32_t B);
+rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params,
+                       const int32_t* d_ctx, int64_t ctx_stride, const int32_t* d_ctx_len,
+                       int32_t B, int32_t* d_tokens, int32_t* d_parents, int32_t* d_depth,
+                       int32_t* d_pos_ids, uint32_t* d_mask, int32_t* d_n_nodes,
+                       int32_t* d_match_n, int64_t* d_match_range, int32_t* d_node_count,
+                       int32_t* d_status, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * rest_tree_attention - attention of the N draft positions of each context over the prefix
+ * KV cache and over their own ancestors (Sec. 3.2 "Draft verification": the pseudo sequence
+ * is run with an attention mask under which every token sees exactly its dependencies).
+ *
+ *   For context b, head h, node i:  keys = {0..L-1} U {L+j : bit j of mask row i}, L = kv_len[b];
+ *   out = softmax(scale * q.k) v  with natural exponent, fp32 accumulation, bf16 output.
+ *
+ *   d_q       bf16, element (b,i,h,d) at b*strides[0] + i*strides[1] + h*strides[2] + d
+ *   d_k, d_v  bf16, element (b,hk,l,d) at b*strides[3] + hk*strides[4] + l*strides[5] + d;
+ *             rows L..L+N-1 hold the K/V of the draft nodes; hk = h / (H / H_kv)
+ *   d_out     bf16, element (b,i,h,d) at b*strides[6] + i*strides[7] + h*strides[8] + d
+ *   strides   host array of 9 element strides; rows of D elements are contiguous and every
+ *             stride is a multiple of 8 elements (16-byte rows); base pointers 16-byte aligned
+ *   d_kv_len  int32[B], 0 <= L and L + N <= rows available
+ *   max_kv    upper bound on L + N over the batch (sizes the split of the key range)
+ *   d_mask    uint32[B,N,ceil(N/32)] as written by rest_draft
+ *   d_lse     optional float[B,H,N]: log of the softmax denominator (natural log, of scaled scores)
+ *   d_ws      scratch of rest_tree_attention_workspace_bytes() bytes
+ *   Limits: D = 128; N in {16, 32, 48, ..., 128}; H % H_kv == 0.
+ */
+size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
+                                           int32_t max_kv);
+rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_v,
+                                const int64_t* strides, const int32_t* d_kv_len,
+                                const uint32_t* d_mask, int32_t B, int32_t H, int32_t H_kv,
+                                int32_t N, int32_t D, int32_t max_kv, float scale, void* d_out,
+                                float* d_lse, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * rest_accept - draft acceptance (Sec. 3.2 "Draft acceptance": draft tokens are accepted from
+ * the start while they coincide with the tokens sampled from the verifier; everything after
+ * the first mismatch is rejected).
+ *
+ *   d_verifier_tokens int32[B,N+1]: slot 0 = verifier's token after the prefix, slot i+1 = its
+ *                     token after draft node i (greedy argmax or a sampled token).
+ *   Walk from the root: if the current node has a child whose token equals the verifier's token
+ *   at the current node, accept it and continue from that child; stop otherwise or after
+ *   max_depth accepted nodes.
+ *   d_accept_len   int32[B]
+ *   d_accept_nodes int32[B,max_depth]    accepted node indices, unused -1
+ *   d_out_tokens   int32[B,max_depth+1]  accepted tokens followed by the verifier's token at the
+ *                  stopping node (what plain decoding would emit next); unused -1
+ */
+rest_status rest_accept(const int32_t* d_tokens, const int32_t* d_parents,
+                        const int32_t* d_n_nodes, const int32_t* d_verifier_tokens, int32_t B,
+                        int32_t N, int32_t max_depth, int32_t* d_accept_len,
+                        int32_t* d_accept_nodes, int32_t* d_out_tokens, void* stream);
+
+const char* rest_status_string(rest_status s);
+/* Text of the last CUDA runtime error seen by this library on the calling thread. */
+const char* rest_last_cuda_error(void);
+/* Number of kernels the library has launched in this process (for launch accounting). */
+uint64_t rest_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REST_H_ */
