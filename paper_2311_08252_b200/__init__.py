@@ -1,0 +1,264 @@
+"""Python binding of librest.so, the CUDA (sm_100a) hot path of one REST decoding step.
+
+Argument marshalling only: every step runs in the library's kernels.  torch is used to own
+device memory and to supply the current CUDA stream.  There is no CPU fallback: importing
+works without the library, but every call raises if librest.so is missing or cannot load.
+
+The four entry points mirror include/rest.h:
+    rest_datastore_create / Datastore   Sec. 3.2, datastore = token stream + suffix array
+    rest_draft                          Algorithms 1 and 2, breadth-first tree + mask
+    rest_tree_attention                 Sec. 3.2, draft verification (tree attention)
+    rest_accept                         Sec. 3.2, draft acceptance
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "librest.so")
+
+REST_OK = 0
+REST_SAMPLE_STRIDED = 0
+REST_SAMPLE_FIRST_K = 1
+REST_DS_VALIDATE = 1
+
+EXPORTS = (
+    "rest_datastore_aux_bytes", "rest_datastore_create", "rest_datastore_destroy",
+    "rest_draft_workspace_bytes", "rest_draft",
+    "rest_tree_attention_workspace_bytes", "rest_tree_attention",
+    "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
+)
+
+
+class RestError(RuntimeError):
+    pass
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("n_max", "n_min", "K", "m", "N", "sample_mode")]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _SO
+
+
+def lib():
+    """Loads librest.so; raises RestError when it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_SO):
+        raise RestError(f"{_SO} is missing: build it with `python -m paper_2311_08252_b200.build` "
+                        "(there is no CPU fallback)")
+    L = ctypes.CDLL(_SO)
+    vp, i32, i64, u32, u64, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64,
+                                  ctypes.c_uint32, ctypes.c_uint64, ctypes.c_size_t)
+    L.rest_datastore_aux_bytes.restype = sz
+    L.rest_datastore_aux_bytes.argtypes = [u64, i32, u32]
+    L.rest_datastore_create.restype = i32
+    L.rest_datastore_create.argtypes = [vp, u64, vp, i32, u32, u32, vp, sz, vp,
+                                        ctypes.POINTER(vp)]
+    L.rest_datastore_destroy.restype = None
+    L.rest_datastore_destroy.argtypes = [vp]
+    L.rest_draft_workspace_bytes.restype = sz
+    L.rest_draft_workspace_bytes.argtypes = [ctypes.POINTER(_Params), i32]
+    L.rest_draft.restype = i32
+    L.rest_draft.argtypes = [vp, ctypes.POINTER(_Params), vp, i64, vp, i32] + [vp] * 10 + [vp, sz, vp]
+    L.rest_tree_attention_workspace_bytes.restype = sz
+    L.rest_tree_attention_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    L.rest_tree_attention.restype = i32
+    L.rest_tree_attention.argtypes = [vp, vp, vp, ctypes.POINTER(i64), vp, vp, i32, i32, i32, i32,
+                                      i32, i32, ctypes.c_float, vp, vp, vp, sz, vp]
+    L.rest_accept.restype = i32
+    L.rest_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    L.rest_status_string.restype = ctypes.c_char_p
+    L.rest_status_string.argtypes = [i32]
+    L.rest_last_cuda_error.restype = ctypes.c_char_p
+    L.rest_launch_count.restype = u64
+    _lib = L
+    return L
+
+
+def _check(rc: int, what: str):
+    if rc != REST_OK:
+        L = lib()
+        msg = L.rest_status_string(rc).decode()
+        if rc == 4:
+            msg += ": " + L.rest_last_cuda_error().decode()
+        raise RestError(f"{what} failed: {msg} (status {rc})")
+
+
+def _stream(stream=None) -> int:
+    import torch
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _dev_i32(t, name):
+    import torch
+    if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+        raise RestError(f"{name} must be a contiguous int32 CUDA tensor")
+    return t
+
+
+def launch_count() -> int:
+    return int(lib().rest_launch_count())
+
+
+class Datastore:
+    """Handle over device-resident tokens int32[n] and suffix array int32[n] / int64[n].
+    The tensors are borrowed: this object keeps references so they outlive the handle."""
+
+    def __init__(self, tokens, sa, vocab: int, validate: bool = False, stream=None):
+        import torch
+        if not (tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()):
+            raise RestError("tokens must be a contiguous int32 CUDA tensor")
+        if not (sa.is_cuda and sa.dtype in (torch.int32, torch.int64) and sa.is_contiguous()
+                and sa.numel() == tokens.numel()):
+            raise RestError("sa must be a contiguous int32/int64 CUDA tensor as long as tokens")
+        self.tokens, self.sa, self.vocab = tokens, sa, int(vocab)
+        self.n_tokens = tokens.numel()
+        self.sa_bytes = sa.element_size()
+        L = lib()
+        aux, aux_bytes = None, 0
+        if validate:
+            aux_bytes = L.rest_datastore_aux_bytes(self.n_tokens, self.sa_bytes, self.vocab)
+            aux = torch.empty(aux_bytes, dtype=torch.uint8, device=tokens.device)
+        h = ctypes.c_void_p()
+        rc = L.rest_datastore_create(tokens.data_ptr(), self.n_tokens, sa.data_ptr(), self.sa_bytes,
+                                     self.vocab, REST_DS_VALIDATE if validate else 0, _ptr(aux),
+                                     aux_bytes, _stream(stream), ctypes.byref(h))
+        _check(rc, "rest_datastore_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().rest_datastore_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def rest_datastore_create(tokens, sa, vocab, validate=False, stream=None) -> Datastore:
+    return Datastore(tokens, sa, vocab, validate, stream)
+
+
+@dataclass
+class DraftOutput:
+    tokens: "object"
+    parents: "object"
+    depth: "object"
+    pos_ids: "object"
+    mask: "object"
+    n_nodes: "object"
+    match_n: "object"
+    match_range: "object"
+    node_count: "object"
+    status: "object"
+
+
+def alloc_draft_output(B: int, N: int, device) -> DraftOutput:
+    import torch
+    i32 = dict(dtype=torch.int32, device=device)
+    Wm = (N + 31) // 32
+    return DraftOutput(
+        torch.empty((B, N), **i32), torch.empty((B, N), **i32), torch.empty((B, N), **i32),
+        torch.empty((B, N), **i32), torch.empty((B, N, Wm), **i32), torch.empty(B, **i32),
+        torch.empty(B, **i32), torch.empty((B, 2), dtype=torch.int64, device=device),
+        torch.empty((B, N), **i32), torch.empty(B, **i32))
+
+
+def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=64,
+               sample_mode=REST_SAMPLE_STRIDED, out: DraftOutput | None = None, stream=None
+               ) -> DraftOutput:
+    """Draft trees for contexts ctx int32[B, Lc] (row b holds ctx_len[b] tokens).  The mask
+    tensor is int32 storage of the uint32 words."""
+    L = lib()
+    _dev_i32(ctx_len, "ctx_len")
+    import torch
+    if not (ctx.is_cuda and ctx.dtype == torch.int32 and ctx.dim() == 2 and ctx.stride(1) == 1):
+        raise RestError("ctx must be an int32 CUDA tensor [B, Lc] with contiguous rows")
+    B = ctx.shape[0]
+    if out is None:
+        out = alloc_draft_output(B, N, ctx.device)
+    prm = _Params(n_max, n_min, K, m, N, sample_mode)
+    rc = L.rest_draft(ds._h, ctypes.byref(prm), ctx.data_ptr(), ctx.stride(0), ctx_len.data_ptr(), B,
+                      out.tokens.data_ptr(), out.parents.data_ptr(), out.depth.data_ptr(),
+                      out.pos_ids.data_ptr(), out.mask.data_ptr(), out.n_nodes.data_ptr(),
+                      out.match_n.data_ptr(), out.match_range.data_ptr(), _ptr(out.node_count),
+                      out.status.data_ptr(), 0, 0, _stream(stream))
+    _check(rc, "rest_draft")
+    return out
+
+
+def tree_attention_workspace_bytes(B, H, N, D, max_kv) -> int:
+    return int(lib().rest_tree_attention_workspace_bytes(B, H, N, D, max_kv))
+
+
+def rest_tree_attention(q, k, v, kv_len, mask, scale, max_kv=None, out=None, lse=None,
+                        workspace=None, stream=None):
+    """q bf16 [B,N,H,D]; k, v bf16 [B,H_kv,Lcap,D] (tree rows at kv_len[b]..kv_len[b]+N-1);
+    kv_len int32[B]; mask int32/uint32 words [B,N,ceil(N/32)].  Returns out bf16 [B,N,H,D]."""
+    import torch
+    L = lib()
+    B, N, H, D = q.shape
+    H_kv, Lcap = k.shape[1], k.shape[2]
+    for t, nm in ((q, "q"), (k, "k"), (v, "v")):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.stride(-1) == 1):
+            raise RestError(f"{nm} must be a bf16 CUDA tensor with a contiguous last dimension")
+    if k.stride() != v.stride() or k.shape != v.shape:
+        raise RestError("k and v must have the same shape and strides")
+    _dev_i32(kv_len, "kv_len")
+    if not (mask.is_cuda and mask.is_contiguous() and mask.element_size() == 4):
+        raise RestError("mask must be a contiguous 32-bit CUDA tensor")
+    if out is None:
+        out = torch.empty((B, N, H, D), dtype=torch.bfloat16, device=q.device)
+    max_kv = Lcap if max_kv is None else int(max_kv)
+    need = L.rest_tree_attention_workspace_bytes(B, H, N, D, max_kv)
+    if need and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    strides = (ctypes.c_int64 * 9)(q.stride(0), q.stride(1), q.stride(2),
+                                   k.stride(0), k.stride(1), k.stride(2),
+                                   out.stride(0), out.stride(1), out.stride(2))
+    rc = L.rest_tree_attention(q.data_ptr(), k.data_ptr(), v.data_ptr(), strides, kv_len.data_ptr(),
+                               mask.data_ptr(), B, H, H_kv, N, D, max_kv, float(scale),
+                               out.data_ptr(), _ptr(lse), _ptr(workspace),
+                               0 if workspace is None else workspace.numel() * workspace.element_size(),
+                               _stream(stream))
+    _check(rc, "rest_tree_attention")
+    return out
+
+
+def rest_accept(tokens, parents, n_nodes, verifier_tokens, max_depth, out=None, stream=None):
+    """Returns (accept_len int32[B], accept_nodes int32[B,max_depth], out_tokens int32[B,max_depth+1])."""
+    import torch
+    L = lib()
+    for t, nm in ((tokens, "tokens"), (parents, "parents"), (n_nodes, "n_nodes"),
+                  (verifier_tokens, "verifier_tokens")):
+        _dev_i32(t, nm)
+    B, N = tokens.shape
+    if verifier_tokens.shape != (B, N + 1):
+        raise RestError("verifier_tokens must be [B, N+1]")
+    if out is None:
+        i32 = dict(dtype=torch.int32, device=tokens.device)
+        out = (torch.empty(B, **i32), torch.empty((B, max_depth), **i32),
+               torch.empty((B, max_depth + 1), **i32))
+    rc = L.rest_accept(tokens.data_ptr(), parents.data_ptr(), n_nodes.data_ptr(),
+                       verifier_tokens.data_ptr(), B, N, max_depth, out[0].data_ptr(),
+                       out[1].data_ptr(), out[2].data_ptr(), _stream(stream))
+    _check(rc, "rest_accept")
+    return out

@@ -1,0 +1,32 @@
+// Shared host-side helpers of the REST CUDA library (error bookkeeping, launch counter).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rest.h"
+
+namespace rest {
+
+// Records the text of a failed CUDA call for rest_last_cuda_error(); returns REST_CUDA_ERROR.
+rest_status note_cuda_error(cudaError_t e, const char* where);
+void count_launch(int n = 1);
+
+#define REST_CUDA_TRY(expr)                                              \
+  do {                                                                   \
+    cudaError_t e_ = (expr);                                             \
+    if (e_ != cudaSuccess) return ::rest::note_cuda_error(e_, #expr);    \
+  } while (0)
+
+struct DatastoreView {
+  const int32_t* tokens;
+  const void* sa;
+  int64_t n_tokens;
+  int32_t sa_bytes;
+  uint32_t vocab;
+};
+
+}  // namespace rest
+
+struct rest_datastore {
+  rest::DatastoreView v;
+};

@@ -1,0 +1,578 @@
+// rest_draft: Algorithm 1 (longest-suffix retrieval over a suffix array), Algorithm 2
+// (Trie weights and the c heaviest nodes) and the breadth-first pseudo sequence with its
+// ancestor mask (Sec. 3.2), one thread block per context, everything in one launch.
+//
+// Phases inside the block (16 warps):
+//   1 search   warp w looks for suffix length n_min + w: a 32-ary lower bound (every lane
+//              probes one suffix-array slot per round, a ballot narrows the interval), then,
+//              if the slot matches, a galloping + 32-ary upper bound.  The longest length
+//              with a non-empty range wins.
+//   2 gather   one candidate row per thread, in suffix-array order, which is also the
+//              lexicographic order of the continuations.  Only the common-prefix length with
+//              the previous row (by warp shuffle) and the row length are kept: for every
+//              depth d the bitmap "row j starts a new Trie node at depth d" (lcp_j < d).
+//   3 select   weight of node (d, j) = distance to the next set bit of bitmap d.  The N
+//              largest by (weight desc, depth asc, row asc) are found with a two-level radix
+//              histogram over (weight, depth) and an ordered scan over rows for the ties.
+//   4 emit     rank the kept nodes by (depth, row), look up parents through the bitmap of the
+//              depth above, build ancestor masks, fetch the node tokens.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+#include "rest.h"
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxM = REST_MAX_M;
+constexpr int kMaxN = REST_MAX_N;
+constexpr int kHistHi = 1056;   // bins of key >> 10, key < 2^20 + 32
+constexpr int kHistLo = 1024;
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+struct DraftArgs {
+  const int32_t* T;
+  const void* sa;
+  int64_t n_tokens;
+  uint32_t vocab;
+  int n_max, n_min, K, m, N, sample_mode;
+  const int32_t* ctx;
+  int64_t ctx_stride;
+  const int32_t* ctx_len;
+  int32_t *tokens, *parents, *depth, *pos_ids;
+  uint32_t* mask;
+  int32_t *n_nodes, *match_n;
+  int64_t* match_range;
+  int32_t *node_count, *status;
+  int nwords;   // bitmap words per depth
+  int kcap;     // K rounded up to a multiple of 32
+};
+
+// Three-way comparison of the first n tokens of the suffix stored in slot `slot` with q.
+// -1 / 0 / +1; a suffix that ends early is smaller.  An out-of-range suffix-array entry
+// compares as smaller and raises `bad`.
+template <typename SaT>
+__device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
+                                     int64_t n_tokens, int64_t slot, const int (&q)[16], int n,
+                                     bool& bad) {
+  int64_t p = (int64_t)__ldg(sa + slot);
+  if (p < 0 || p >= n_tokens) { bad = true; return -1; }
+  int tk[16];
+#pragma unroll
+  for (int k = 0; k < 16; ++k) tk[k] = (k < n && p + k < n_tokens) ? __ldg(T + p + k) : 0;
+  int r = 0;
+#pragma unroll
+  for (int k = 15; k >= 0; --k) {
+    if (k < n) {
+      if (p + k >= n_tokens) {
+        r = -1;
+      } else {
+        uint32_t a = (uint32_t)tk[k], b = (uint32_t)q[k];
+        if (a != b) r = a < b ? -1 : 1;
+      }
+    }
+  }
+  return r;
+}
+
+// First slot in [lo, hi) whose comparison is >= 0 (STRICT = false) or > 0 (STRICT = true);
+// hi when there is none.  Warp-cooperative; all lanes return the same value.  `eq` reports
+// whether the returned slot compared equal (in: whether slot `hi` is known to compare equal).
+template <typename SaT, bool STRICT>
+__device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
+                                   int64_t n_tokens, int64_t lo, int64_t hi, const int (&q)[16],
+                                   int n, int lane, bool& eq, bool& bad) {
+  while (hi - lo > 32) {
+    int64_t size = hi - lo;
+    int64_t pos = lo + ((int64_t)(lane + 1) * size) / 33;
+    int c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
+    bool t = STRICT ? (c > 0) : (c >= 0);
+    unsigned b = __ballot_sync(kFull, t);
+    if (b == 0) {
+      lo = __shfl_sync(kFull, pos, 31) + 1;
+    } else {
+      int f = __ffs(b) - 1;
+      int64_t pf = __shfl_sync(kFull, pos, f);
+      int cf = __shfl_sync(kFull, c, f);
+      int64_t pprev = __shfl_sync(kFull, pos, f > 0 ? f - 1 : 0);
+      hi = pf;
+      eq = (cf == 0);
+      if (f > 0) lo = pprev + 1;
+    }
+  }
+  int64_t pos = lo + lane;
+  int c = -1;
+  if (pos < hi) c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
+  bool t = (pos < hi) && (STRICT ? (c > 0) : (c >= 0));
+  unsigned b = __ballot_sync(kFull, t);
+  if (b != 0) {
+    int f = __ffs(b) - 1;
+    int cf = __shfl_sync(kFull, c, f);
+    eq = (cf == 0);
+    return lo + f;
+  }
+  return hi;
+}
+
+// Suffix-array slot of candidate j.
+__device__ __forceinline__ int64_t sample_slot(int64_t lo, int64_t cnt, int K, int mode, int j) {
+  if (cnt <= (int64_t)K || mode == REST_SAMPLE_FIRST_K) return lo + j;
+  return lo + (int64_t)(((unsigned long long)j * (unsigned long long)cnt) / (unsigned long long)K);
+}
+
+// Smallest set bit strictly after position j (the bitmap carries a sentinel past the rows).
+__device__ __forceinline__ int next_set(const uint32_t* __restrict__ row, int j) {
+  int w = j >> 5;
+  uint32_t bits = row[w] & ~((2u << (j & 31)) - 1u);
+  while (bits == 0) bits = row[++w];
+  return (w << 5) + __ffs(bits) - 1;
+}
+
+// Largest set bit at or before position j (bit 0 is always set).
+__device__ __forceinline__ int prev_set(const uint32_t* __restrict__ row, int j) {
+  int w = j >> 5;
+  uint32_t bits = row[w] & ((2u << (j & 31)) - 1u);
+  while (bits == 0 && w > 0) bits = row[--w];
+  return (w << 5) + 31 - __clz(bits | 1u);
+}
+
+// Executed by one warp.  hist[0..nbins) holds counts; total >= need >= 1.  Finds the largest
+// bin b with sum(hist[k], k > b) < need; returns b and that sum.
+__device__ void warp_threshold_desc(const uint32_t* hist, int nbins, uint32_t need, int lane,
+                                    int* out_bin, uint32_t* out_above) {
+  int per = (nbins + 31) / 32;
+  int top = nbins - 1 - lane * per;
+  int bot = max(0, top - per + 1);
+  uint32_t s = 0;
+  for (int b = top; b >= bot && b >= 0; --b) s += hist[b];
+  uint32_t incl = s;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t v = __shfl_up_sync(kFull, incl, o);
+    if (lane >= o) incl += v;
+  }
+  uint32_t excl = incl - s;
+  if (excl < need && need <= incl) {
+    uint32_t acc = excl;
+    for (int b = top; b >= bot; --b) {
+      uint32_t h = hist[b];
+      if (acc + h >= need) { *out_bin = b; *out_above = acc; break; }
+      acc += h;
+    }
+  }
+}
+
+struct Smem {
+  int q[16];
+  long long lb[17], ub[17];
+  uint32_t e1[kMaxM + 1];      // nodes of weight 1 per depth
+  uint32_t heavy_total;        // nodes of weight >= 2
+  int err;
+  int bin_hi;
+  uint32_t above_hi;
+  int bin_lo;
+  uint32_t above_lo;
+  uint32_t nsel;
+  uint32_t warp_cnt[kWarps];
+  uint32_t sel[kMaxN];         // depth << 16 | row
+  uint32_t selcnt[kMaxN];
+  uint32_t sorted[kMaxN];
+  uint32_t sortedcnt[kMaxN];
+  int par[kMaxN];
+  uint32_t hist_hi[kHistHi];
+  uint32_t hist_lo[kHistLo];
+};
+
+template <typename SaT>
+__global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Smem& s = *reinterpret_cast<Smem*>(smem_raw);
+  uint16_t* lenlcp = reinterpret_cast<uint16_t*>(smem_raw + sizeof(Smem));          // [kcap]
+  uint32_t* bm = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Smem) + 2 * a.kcap); // [m][nwords]
+
+  const int b = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int N = a.N, m = a.m, Wm = (N + 31) >> 5;
+  const int32_t* __restrict__ T = a.T;
+  const SaT* __restrict__ sa = static_cast<const SaT*>(a.sa);
+  const int64_t n_tokens = a.n_tokens;
+  const int clen = a.ctx_len[b];
+  const int32_t* ctx = a.ctx + (int64_t)b * a.ctx_stride;
+
+  // Unused-slot defaults; thread i owns slot i for the whole kernel.
+  if (tid < N) {
+    int64_t o = (int64_t)b * N + tid;
+    a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
+    for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (tid >> 5)) ? (1u << (tid & 31)) : 0u;
+    if (a.node_count) a.node_count[o] = 0;
+  }
+  const int nq = min(a.n_max, max(clen, 0));   // context tokens that can take part
+  if (tid == 0) { s.err = 0; s.heavy_total = 0; s.nsel = 0; }
+  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; }
+  if (tid <= kMaxM) s.e1[tid] = 0;
+  for (int i = tid; i < kHistHi; i += kThreads) s.hist_hi[i] = 0;
+  for (int i = tid; i < kHistLo; i += kThreads) s.hist_lo[i] = 0;
+  __syncthreads();
+  if (tid < nq) {
+    int t = ctx[clen - nq + tid];
+    s.q[tid] = t;
+    if (t < 0 || (uint32_t)t >= a.vocab) atomicOr(&s.err, REST_CTX_BAD_TOKEN);
+  }
+  __syncthreads();
+  if (s.err != 0 || nq < a.n_min) {
+    if (tid == 0) {
+      a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
+      a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
+    }
+    return;
+  }
+
+  // ---- phase 1: search --------------------------------------------------------------
+  {
+    const int n = a.n_min + warp;
+    if (n <= nq) {
+      int q[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
+      bool bad = false, eq = false;
+      int64_t lb = warp_first_true<SaT, false>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad);
+      int64_t ub = lb;
+      if (eq && lb < n_tokens) {
+        // gallop: lane l probes lb + 2^l
+        int64_t pos = lb + ((int64_t)1 << lane);
+        bool t = true;
+        if (pos < n_tokens) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
+        unsigned bal = __ballot_sync(kFull, t);
+        int64_t lo2, hi2 = n_tokens;
+        bool eq2 = false;
+        if (bal == 0) {
+          lo2 = lb + ((int64_t)1 << 31) + 1;
+        } else {
+          int f = __ffs(bal) - 1;
+          int64_t pf = lb + ((int64_t)1 << f);
+          hi2 = pf < n_tokens ? pf : n_tokens;
+          lo2 = f > 0 ? lb + ((int64_t)1 << (f - 1)) + 1 : lb + 1;
+        }
+        if (lo2 > hi2) lo2 = hi2;
+        ub = warp_first_true<SaT, true>(T, sa, n_tokens, lo2, hi2, q, n, lane, eq2, bad);
+      }
+      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+      if (lane == 0) { s.lb[n] = lb; s.ub[n] = ub; }
+    }
+  }
+  __syncthreads();
+  int n_win = 0;
+  for (int n = nq; n >= a.n_min; --n)
+    if (s.ub[n] > s.lb[n]) { n_win = n; break; }
+  if (s.err != 0 || n_win == 0) {
+    if (tid == 0) {
+      a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
+      a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
+    }
+    return;
+  }
+  const int64_t lo = s.lb[n_win], hi = s.ub[n_win];
+  const int64_t cnt = hi - lo;
+  const int Kp = (int)(cnt < (int64_t)a.K ? cnt : (int64_t)a.K);
+  const int nwords = a.nwords;
+  const int niter = (Kp + kThreads - 1) / kThreads;
+
+  // ---- phase 2: gather rows, common-prefix lengths, node-start bitmaps --------------------
+  for (int it = 0; it < niter; ++it) {
+    const int jbase = it * kThreads + warp * 32;
+    if (jbase >= Kp) continue;   // warp-uniform
+    const int j = jbase + lane;
+    const bool valid = j < Kp;
+    int row[kMaxM], prev[kMaxM];
+    int len = 0, plen = 0;
+    bool bad = false;
+    if (valid) {
+      int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
+      if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
+      int64_t base = p + n_win;
+      int64_t rem = n_tokens - base;
+      len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+#pragma unroll
+      for (int d = 0; d < kMaxM; ++d) row[d] = (d < len) ? __ldg(T + base + d) : 0;
+    } else {
+#pragma unroll
+      for (int d = 0; d < kMaxM; ++d) row[d] = 0;
+    }
+#pragma unroll
+    for (int d = 0; d < kMaxM; ++d) prev[d] = __shfl_up_sync(kFull, row[d], 1);
+    plen = __shfl_up_sync(kFull, len, 1);
+    if (lane == 0 && j > 0) {   // previous row belongs to another warp: fetch it again
+      int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j - 1));
+      if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
+      int64_t base = p + n_win;
+      int64_t rem = n_tokens - base;
+      plen = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+#pragma unroll
+      for (int d = 0; d < kMaxM; ++d) prev[d] = (d < plen) ? __ldg(T + base + d) : 0;
+    }
+    int lcp = 0;
+    if (valid && j > 0) {
+      const int lim = min(len, plen);
+      bool run = true;
+      bool ordered = plen <= len;   // decides when one row is a prefix of the other
+#pragma unroll
+      for (int d = 0; d < kMaxM; ++d) {
+        if (run && d < lim) {
+          if (row[d] == prev[d]) {
+            lcp = d + 1;
+          } else {
+            run = false;
+            ordered = (uint32_t)prev[d] < (uint32_t)row[d];
+          }
+        }
+      }
+      if (!ordered) bad = true;
+    }
+    if (valid) lenlcp[j] = (uint16_t)(lcp | (len << 8));
+    uint32_t myword = 0;
+#pragma unroll
+    for (int d = 1; d <= kMaxM; ++d) {
+      if (d <= m) {
+        uint32_t w = __ballot_sync(kFull, !valid || lcp < d);
+        if (lane == d - 1) myword = w;
+      }
+    }
+    if (lane < m) bm[lane * nwords + (jbase >> 5)] = myword;
+    if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+  }
+  if (tid < m) bm[tid * nwords + ((Kp + 31) >> 5)] = kFull;   // sentinel past the last row
+  __syncthreads();
+  if (s.err != 0) {
+    if (tid == 0) {
+      a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
+      a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
+    }
+    return;
+  }
+
+  // ---- phase 3a: histogram of (weight, depth) over all Trie nodes --------------------------
+  // key = weight << 5 | (16 - depth): larger key = better node.
+  for (int it = 0; it < niter; ++it) {
+    const int jbase = it * kThreads + warp * 32;
+    if (jbase >= Kp) continue;
+    const int j = jbase + lane;
+    const bool valid = j < Kp;
+    const int ll = valid ? lenlcp[j] : 0;
+    const int lcp = ll & 0xFF, len = ll >> 8;
+    uint32_t nheavy = 0;
+    for (int d = 1; d <= m; ++d) {
+      const bool act = valid && d > lcp && d <= len;
+      int c = 0;
+      if (act) c = next_set(bm + (d - 1) * nwords, j) - j;
+      uint32_t ones = __ballot_sync(kFull, act && c == 1);
+      if (lane == 0 && ones) atomicAdd(&s.e1[d], __popc(ones));
+      if (act && c >= 2) {
+        atomicAdd(&s.hist_hi[((c << 5) | (16 - d)) >> 10], 1u);
+        ++nheavy;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) nheavy += __shfl_xor_sync(kFull, nheavy, o);
+    if (lane == 0 && nheavy) atomicAdd(&s.heavy_total, nheavy);
+  }
+  __syncthreads();
+
+  // ---- phase 3b: threshold key t*, number of ties wanted ------------------------------------
+  uint32_t tstar;      // nodes with key > tstar are kept
+  uint32_t r_tie;      // plus the first r_tie nodes (by row) with key == tstar
+  const uint32_t heavy_total = s.heavy_total;
+  if (heavy_total >= (uint32_t)N) {
+    if (warp == 0) warp_threshold_desc(s.hist_hi, kHistHi, (uint32_t)N, lane, &s.bin_hi, &s.above_hi);
+    __syncthreads();
+    const int bin_hi = s.bin_hi;
+    for (int it = 0; it < niter; ++it) {
+      const int jbase = it * kThreads + warp * 32;
+      if (jbase >= Kp) continue;
+      const int j = jbase + lane;
+      if (j >= Kp) continue;
+      const int ll = lenlcp[j];
+      const int lcp = ll & 0xFF, len = ll >> 8;
+      for (int d = lcp + 1; d <= len; ++d) {
+        int c = next_set(bm + (d - 1) * nwords, j) - j;
+        if (c < 2) break;   // weights do not grow with depth
+        uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
+        if ((int)(key >> 10) == bin_hi) atomicAdd(&s.hist_lo[key & 1023u], 1u);
+      }
+    }
+    __syncthreads();
+    if (warp == 0)
+      warp_threshold_desc(s.hist_lo, kHistLo, (uint32_t)N - s.above_hi, lane, &s.bin_lo, &s.above_lo);
+    __syncthreads();
+    tstar = ((uint32_t)bin_hi << 10) | (uint32_t)s.bin_lo;
+    r_tie = (uint32_t)N - s.above_hi - s.above_lo;
+  } else {
+    // every node of weight >= 2 is kept; weight-1 nodes fill up by depth, then by row
+    uint32_t need = (uint32_t)N - heavy_total, cum = 0;
+    tstar = 0; r_tie = 0;
+    for (int d = 1; d <= m; ++d) {
+      uint32_t e = s.e1[d];
+      if (cum + e >= need) { tstar = (1u << 5) | (uint32_t)(16 - d); r_tie = need - cum; break; }
+      cum += e;
+    }
+  }
+  const int d_tie = 16 - (int)(tstar & 31u);
+  const int c_tie = (int)(tstar >> 5);
+
+  // ---- phase 3c: collect the kept nodes -----------------------------------------------------
+  uint32_t tie_base = 0;
+  for (int it = 0; it < niter; ++it) {
+    const int j = it * kThreads + tid;
+    const bool valid = j < Kp;
+    bool tie = false;
+    if (valid) {
+      const int ll = lenlcp[j];
+      const int lcp = ll & 0xFF, len = ll >> 8;
+      for (int d = lcp + 1; d <= len; ++d) {
+        int c = next_set(bm + (d - 1) * nwords, j) - j;
+        uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
+        if (key > tstar) {
+          uint32_t slot = atomicAdd(&s.nsel, 1u);
+          if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)j; s.selcnt[slot] = c; }
+        } else if (key == tstar) {
+          tie = true;
+        }
+      }
+    }
+    if (r_tie > 0) {   // block-uniform
+      uint32_t bal = __ballot_sync(kFull, tie);
+      if (lane == 0) s.warp_cnt[warp] = __popc(bal);
+      __syncthreads();
+      uint32_t before = tie_base, total = 0;
+      for (int w = 0; w < kWarps; ++w) {
+        uint32_t c = s.warp_cnt[w];
+        if (w < warp) before += c;
+        total += c;
+      }
+      uint32_t rank = before + __popc(bal & ((1u << lane) - 1u));
+      if (tie && rank < r_tie) {
+        uint32_t slot = atomicAdd(&s.nsel, 1u);
+        if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d_tie << 16) | (uint32_t)j; s.selcnt[slot] = c_tie; }
+      }
+      tie_base += total;
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+  const int nn = (int)min(s.nsel, (uint32_t)N);
+  if (s.nsel > (uint32_t)N && tid == 0) atomicOr(&s.err, REST_CTX_INTERNAL);
+
+  // ---- phase 4: breadth-first order, parents, masks, tokens ---------------------------------
+  if (tid < nn) {
+    const uint32_t me = s.sel[tid];
+    int rank = 0;
+    for (int k = 0; k < nn; ++k) rank += (s.sel[k] < me);
+    s.sorted[rank] = me;
+    s.sortedcnt[rank] = s.selcnt[tid];
+  }
+  __syncthreads();
+  if (tid < nn) {
+    const uint32_t me = s.sorted[tid];
+    const int d = (int)(me >> 16), j = (int)(me & 0xFFFFu);
+    int par = -1;
+    if (d > 1) {
+      const int jp = prev_set(bm + (d - 2) * nwords, j);
+      const uint32_t pkey = ((uint32_t)(d - 1) << 16) | (uint32_t)jp;
+      int l = 0, r = nn - 1;
+      par = -2;
+      while (l <= r) {
+        int mid = (l + r) >> 1;
+        uint32_t v = s.sorted[mid];
+        if (v == pkey) { par = mid; break; }
+        if (v < pkey) l = mid + 1; else r = mid - 1;
+      }
+      if (par < 0) { atomicOr(&s.err, REST_CTX_INTERNAL); par = -1; }
+    }
+    s.par[tid] = par;
+    int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
+    int64_t o = (int64_t)b * N + tid;
+    a.tokens[o] = __ldg(T + p + n_win + d - 1);
+    a.parents[o] = par;
+    a.depth[o] = d;
+    a.pos_ids[o] = clen + d - 1;
+    if (a.node_count) a.node_count[o] = (int32_t)s.sortedcnt[tid];
+  }
+  __syncthreads();
+  if (tid < nn) {
+    uint32_t bits[(kMaxN + 31) / 32];
+#pragma unroll
+    for (int w = 0; w < (kMaxN + 31) / 32; ++w) bits[w] = 0;
+    int k = tid;
+    for (int step = 0; step <= kMaxM && k >= 0; ++step) {
+#pragma unroll
+      for (int w = 0; w < (kMaxN + 31) / 32; ++w)
+        if (w == (k >> 5)) bits[w] |= 1u << (k & 31);
+      k = s.par[k];
+    }
+    int64_t o = ((int64_t)b * N + tid) * Wm;
+#pragma unroll
+    for (int w = 0; w < (kMaxN + 31) / 32; ++w)
+      if (w < Wm) a.mask[o + w] = bits[w];
+  }
+  __syncthreads();
+  if (tid == 0) {
+    a.status[b] = s.err;
+    a.n_nodes[b] = nn;
+    a.match_n[b] = n_win;
+    a.match_range[2 * b] = lo;
+    a.match_range[2 * b + 1] = hi;
+  }
+}
+
+size_t draft_smem_bytes(int K, int m, int* kcap_out, int* nwords_out) {
+  int kcap = (K + 31) / 32 * 32;
+  int nwords = kcap / 32 + 1;
+  if (kcap_out) *kcap_out = kcap;
+  if (nwords_out) *nwords_out = nwords;
+  size_t bytes = sizeof(Smem) + 2 * (size_t)kcap + 4 * (size_t)m * nwords;
+  return (bytes + 15) / 16 * 16;
+}
+
+}  // namespace
+
+extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params*, int32_t) { return 0; }
+
+extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* prm,
+                                  const int32_t* d_ctx, int64_t ctx_stride,
+                                  const int32_t* d_ctx_len, int32_t B, int32_t* d_tokens,
+                                  int32_t* d_parents, int32_t* d_depth, int32_t* d_pos_ids,
+                                  uint32_t* d_mask, int32_t* d_n_nodes, int32_t* d_match_n,
+                                  int64_t* d_match_range, int32_t* d_node_count,
+                                  int32_t* d_status, void* /*d_ws*/, size_t /*ws_bytes*/,
+                                  void* stream) {
+  if (!ds || !prm || B < 0) return REST_INVALID_ARG;
+  if (B == 0) return REST_OK;
+  if (!d_ctx || !d_ctx_len || !d_tokens || !d_parents || !d_depth || !d_pos_ids || !d_mask ||
+      !d_n_nodes || !d_match_n || !d_match_range || !d_status || ctx_stride < 0)
+    return REST_INVALID_ARG;
+  if (prm->n_min < 1 || prm->n_max < prm->n_min || prm->K < 1 || prm->m < 1 || prm->N < 1)
+    return REST_INVALID_ARG;
+  if (prm->sample_mode != REST_SAMPLE_STRIDED && prm->sample_mode != REST_SAMPLE_FIRST_K)
+    return REST_INVALID_ARG;
+  if (prm->n_max > REST_MAX_SUFFIX || prm->m > REST_MAX_M || prm->N > REST_MAX_N ||
+      prm->K > REST_MAX_K || prm->n_max - prm->n_min + 1 > kWarps)
+    return REST_UNSUPPORTED;
+
+  DraftArgs a;
+  a.T = ds->v.tokens; a.sa = ds->v.sa; a.n_tokens = ds->v.n_tokens; a.vocab = ds->v.vocab;
+  a.n_max = prm->n_max; a.n_min = prm->n_min; a.K = prm->K; a.m = prm->m; a.N = prm->N;
+  a.sample_mode = prm->sample_mode;
+  a.ctx = d_ctx; a.ctx_stride = ctx_stride; a.ctx_len = d_ctx_len;
+  a.tokens = d_tokens; a.parents = d_parents; a.depth = d_depth; a.pos_ids = d_pos_ids;
+  a.mask = d_mask; a.n_nodes = d_n_nodes; a.match_n = d_match_n; a.match_range = d_match_range;
+  a.node_count = d_node_count; a.status = d_status;
+  size_t smem = draft_smem_bytes(prm->K, prm->m, &a.kcap, &a.nwords);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  auto kern = ds->v.sa_bytes == 4 ? rest_draft_kernel<int32_t> : rest_draft_kernel<int64_t>;
+  REST_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<B, kThreads, smem, st>>>(a);
+  rest::count_launch();
+  REST_CUDA_TRY(cudaGetLastError());
+  return REST_OK;
+}

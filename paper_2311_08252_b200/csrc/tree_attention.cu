@@ -1,0 +1,399 @@
+// rest_tree_attention: masked attention of the N draft positions over the prefix KV cache
+// and over their own ancestors (Sec. 3.2 "Draft verification").
+//
+// Split-KV flash-decode layout: one thread block per (context, head, key split).  A block
+// holds the N x 128 query tile as tensor-core A fragments in registers (16 rows per warp)
+// and streams 64-key K/V tiles through a double-buffered, XOR-swizzled shared-memory ring
+// filled with 16-byte asynchronous copies.  Per tile: S = Q K^T (bf16 tensor-core MMA, fp32
+// accumulate), tree mask on the tiles that reach past the prefix, online softmax in base 2,
+// O += P V.  With one split the block normalises and writes bf16 output directly; otherwise
+// it writes un-normalised fp32 partials (plus running max and sum) and a second kernel merges
+// the splits.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "common.cuh"
+#include "rest.h"
+
+namespace {
+
+constexpr int kD = REST_HEAD_DIM;     // 128
+constexpr int kBN = 64;               // keys per tile
+constexpr int kStages = 2;
+constexpr int kRowBytes = kD * 2;     // 256
+constexpr int kTileBytes = kBN * kRowBytes;   // 16 KB
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kNumSMs = 148;
+
+struct AttnArgs {
+  const __nv_bfloat16 *q, *k, *v;
+  __nv_bfloat16* out;
+  float* lse;
+  const int32_t* kv_len;
+  const uint32_t* mask;
+  float* ws_o;      // [B,H,S,N,128] fp32 partial numerators
+  float* ws_ml;     // [B,H,S,N,2]   running max (base-2 units) and sum
+  int64_t q_b, q_n, q_h, kv_b, kv_h, kv_l, o_b, o_n, o_h;
+  int B, H, group, N, Wm, S;
+  float scale_log2;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool pred) {
+  int sz = pred ? 16 : 0;   // size 0: nothing is read, destination is zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                        uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                          uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+      "{%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+// byte offset of 16-byte chunk `chunk` of row `row` in a swizzled [rows][256 B] tile
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+  return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+}
+
+// Shared memory: Q tile [N][256 B] | K ring [stages][16 KB] | V ring [stages][16 KB] | mask [N][4]
+__global__ void __launch_bounds__(256)
+tree_attention_kernel(AttnArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int N = a.N;
+  unsigned char* sQ = smem;
+  unsigned char* sK = sQ + N * kRowBytes;
+  unsigned char* sV = sK + kStages * kTileBytes;
+  uint32_t* sMask = reinterpret_cast<uint32_t*>(sV + kStages * kTileBytes);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x;
+  const int g = lane >> 2, t4 = lane & 3;
+  int bid = blockIdx.x;
+  const int split = bid % a.S; bid /= a.S;
+  const int h = bid % a.H;
+  const int b = bid / a.H;
+  const int hk = h / a.group;
+  const int L = a.kv_len[b];
+  const int total = L + N;
+  const int ntiles = (total + kBN - 1) / kBN;
+  const int tps = (ntiles + a.S - 1) / a.S;
+  const int t0 = split * tps;
+  const int t1 = min(ntiles, t0 + tps);
+
+  const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h;
+  const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
+  const __nv_bfloat16* vb = a.v + b * a.kv_b + hk * a.kv_h;
+
+  // Q tile and mask rows
+  for (int c = tid; c < N * 16; c += nthreads) {
+    int row = c >> 4, chunk = c & 15;
+    cp_async16(smem_u32(sQ) + swz(row, chunk), qb + row * a.q_n + chunk * 8, true);
+  }
+  for (int c = tid; c < N * 4; c += nthreads) {
+    int row = c >> 2, w = c & 3;
+    sMask[c] = (w < a.Wm) ? a.mask[((int64_t)b * N + row) * a.Wm + w] : 0u;
+  }
+  auto load_tile = [&](int tile, int stage) {
+    const int key0 = tile * kBN;
+    const uint32_t dK = smem_u32(sK) + stage * kTileBytes;
+    const uint32_t dV = smem_u32(sV) + stage * kTileBytes;
+    for (int c = tid; c < kBN * 16; c += nthreads) {
+      int row = c >> 4, chunk = c & 15;
+      int key = key0 + row;
+      bool ok = key < total;
+      int64_t off = (int64_t)(ok ? key : 0) * a.kv_l + chunk * 8;
+      cp_async16(dK + swz(row, chunk), kb + off, ok);
+      cp_async16(dV + swz(row, chunk), vb + off, ok);
+    }
+  };
+  if (t0 < t1) load_tile(t0, 0);
+  cp_async_commit();
+
+  float o[16][4];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g+8 of this warp
+  uint32_t qf[8][4];
+  const int r0 = warp * 16 + g, r1 = r0 + 8;
+
+  for (int t = t0; t < t1; ++t) {
+    const int stage = (t - t0) & 1;
+    if (t + 1 < t1) {
+      load_tile(t + 1, stage ^ 1);
+      cp_async_commit();
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
+    __syncthreads();
+    if (t == t0) {
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        int chunk = ks * 2 + (lane >> 4);
+        ldsm_x4(smem_u32(sQ) + swz(row, chunk), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+      }
+    }
+    const uint32_t bK = smem_u32(sK) + stage * kTileBytes;
+    const uint32_t bV = smem_u32(sV) + stage * kTileBytes;
+
+    // S = Q K^T : 16 rows x 64 keys per warp
+    float s[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {   // pairs of 8-key tiles
+        uint32_t b0, b1, b2, b3;
+        int key = np * 16 + (lane & 7) + (lane >> 4) * 8;
+        int chunk = ks * 2 + ((lane >> 3) & 1);
+        ldsm_x4(bK + swz(key, chunk), b0, b1, b2, b3);
+        mma_bf16(s[np * 2], qf[ks], b0, b1);
+        mma_bf16(s[np * 2 + 1], qf[ks], b2, b3);
+      }
+    }
+
+    // scale, mask, online softmax (base 2)
+    const int key0 = t * kBN;
+    const bool need_mask = key0 + kBN > L;
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float v = s[nt][e] * a.scale_log2;
+        if (need_mask) {
+          int key = key0 + nt * 8 + t4 * 2 + (e & 1);
+          int row = (e < 2) ? r0 : r1;
+          bool ok = key < L;
+          if (!ok && key < total) {
+            int j = key - L;
+            ok = (sMask[row * 4 + (j >> 5)] >> (j & 31)) & 1u;
+          }
+          if (!ok) v = -INFINITY;
+        }
+        s[nt][e] = v;
+      }
+      mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
+      mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+    const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+    const float al0 = exp2f(m0 - ms0), al1 = exp2f(m1 - ms1);   // m = -inf gives 0
+    m0 = mn0; m1 = mn1;
+    float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      s[nt][0] = exp2f(s[nt][0] - ms0); s[nt][1] = exp2f(s[nt][1] - ms0);
+      s[nt][2] = exp2f(s[nt][2] - ms1); s[nt][3] = exp2f(s[nt][3] - ms1);
+      ps0 += s[nt][0] + s[nt][1];
+      ps1 += s[nt][2] + s[nt][3];
+    }
+    l0 = l0 * al0 + ps0;
+    l1 = l1 * al1 + ps1;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[i][0] *= al0; o[i][1] *= al0; o[i][2] *= al1; o[i][3] *= al1; }
+
+    // O += P V
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {   // 16 keys per step
+      uint32_t pa[4];
+      pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+      pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+      pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+      pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+#pragma unroll
+      for (int dp = 0; dp < 8; ++dp) {   // pairs of 8-wide output tiles
+        uint32_t b0, b1, b2, b3;
+        int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        int chunk = dp * 2 + (lane >> 4);
+        ldsm_x4_t(bV + swz(key, chunk), b0, b1, b2, b3);
+        mma_bf16(o[dp * 2], pa, b0, b1);
+        mma_bf16(o[dp * 2 + 1], pa, b2, b3);
+      }
+    }
+    __syncthreads();
+  }
+  if (t0 >= t1) { cp_async_wait<0>(); }
+
+  l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1);
+  l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
+  l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 1);
+  l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 2);
+
+  if (a.S == 1) {
+    const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
+    __nv_bfloat16* ob = a.out + b * a.o_b + h * a.o_h;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      int col = i * 8 + t4 * 2;
+      *reinterpret_cast<uint32_t*>(ob + r0 * a.o_n + col) = pack_bf16(o[i][0] * inv0, o[i][1] * inv0);
+      *reinterpret_cast<uint32_t*>(ob + r1 * a.o_n + col) = pack_bf16(o[i][2] * inv1, o[i][3] * inv1);
+    }
+    if (a.lse && t4 == 0) {
+      float* lp = a.lse + ((int64_t)b * a.H + h) * N;
+      lp[r0] = (m0 + log2f(l0)) * kLn2;
+      lp[r1] = (m1 + log2f(l1)) * kLn2;
+    }
+  } else {
+    const int64_t base = (((int64_t)b * a.H + h) * a.S + split) * N;
+    float* po = a.ws_o + base * kD;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      int col = i * 8 + t4 * 2;
+      *reinterpret_cast<float2*>(po + (int64_t)r0 * kD + col) = make_float2(o[i][0], o[i][1]);
+      *reinterpret_cast<float2*>(po + (int64_t)r1 * kD + col) = make_float2(o[i][2], o[i][3]);
+    }
+    if (t4 == 0) {
+      float* pm = a.ws_ml + base * 2;
+      pm[r0 * 2] = m0; pm[r0 * 2 + 1] = l0;
+      pm[r1 * 2] = m1; pm[r1 * 2 + 1] = l1;
+    }
+  }
+}
+
+// Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
+__global__ void __launch_bounds__(128)
+tree_attention_combine_kernel(AttnArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int64_t unit = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t nunits = (int64_t)a.B * a.H * a.N;
+  if (unit >= nunits) return;
+  const int row = (int)(unit % a.N);
+  const int64_t bh = unit / a.N;
+  const int h = (int)(bh % a.H);
+  const int64_t b = bh / a.H;
+  const float* pm = a.ws_ml + (bh * a.S * a.N + row) * 2;
+  float M = -INFINITY;
+  for (int s = 0; s < a.S; ++s) M = fmaxf(M, pm[(int64_t)s * a.N * 2]);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float lsum = 0.f;
+  for (int s = 0; s < a.S; ++s) {
+    float ms = pm[(int64_t)s * a.N * 2], ls = pm[(int64_t)s * a.N * 2 + 1];
+    float w = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
+    lsum += ls * w;
+    if (w != 0.f) {
+      const float4 v = *reinterpret_cast<const float4*>(
+          a.ws_o + ((bh * a.S + s) * a.N + row) * kD + lane * 4);
+      acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+    }
+  }
+  const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+  __nv_bfloat16* op = a.out + b * a.o_b + row * a.o_n + h * a.o_h + lane * 4;
+  uint2 pk;
+  pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+  pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(op) = pk;
+  if (a.lse && lane == 0) a.lse[bh * a.N + row] = (M + log2f(lsum)) * kLn2;
+}
+
+int choose_splits(int B, int H, int max_kv) {
+  const int ntiles = (max_kv + kBN - 1) / kBN;
+  const int64_t units = (int64_t)B * H;
+  int S = (int)((2 * kNumSMs + units - 1) / units);
+  const int cap = (ntiles + 1) / 2;   // at least two tiles per split
+  if (S > cap) S = cap;
+  if (S > 64) S = 64;
+  if (units >= 2 * kNumSMs) S = 1;
+  if (S < 1) S = 1;
+  return S;
+}
+
+size_t attn_smem_bytes(int N) {
+  return (size_t)N * kRowBytes + 2 * (size_t)kStages * kTileBytes + (size_t)N * 16;
+}
+
+}  // namespace
+
+extern "C" size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
+                                                      int32_t max_kv) {
+  if (B <= 0 || H <= 0 || N <= 0 || D != kD || max_kv <= 0) return 0;
+  const int S = choose_splits(B, H, max_kv);
+  if (S == 1) return 0;
+  return (size_t)B * H * S * N * (kD + 2) * sizeof(float);
+}
+
+extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_v,
+                                           const int64_t* strides, const int32_t* d_kv_len,
+                                           const uint32_t* d_mask, int32_t B, int32_t H,
+                                           int32_t H_kv, int32_t N, int32_t D, int32_t max_kv,
+                                           float scale, void* d_out, float* d_lse, void* d_ws,
+                                           size_t ws_bytes, void* stream) {
+  if (B < 0 || H < 1 || H_kv < 1 || N < 1 || max_kv < 1 || !strides) return REST_INVALID_ARG;
+  if (B == 0) return REST_OK;
+  if (!d_q || !d_k || !d_v || !d_kv_len || !d_mask || !d_out) return REST_INVALID_ARG;
+  if (D != kD || N > REST_MAX_N || (N % 16) != 0 || (H % H_kv) != 0) return REST_UNSUPPORTED;
+  for (int i = 0; i < 9; ++i)
+    if (strides[i] < 0 || (strides[i] % 8) != 0) return REST_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) |
+       reinterpret_cast<uintptr_t>(d_v) | reinterpret_cast<uintptr_t>(d_out)) & 15)
+    return REST_INVALID_ARG;
+  if ((int64_t)B * H * 64 > 0x7FFFFFFFll) return REST_UNSUPPORTED;
+
+  AttnArgs a;
+  a.q = static_cast<const __nv_bfloat16*>(d_q);
+  a.k = static_cast<const __nv_bfloat16*>(d_k);
+  a.v = static_cast<const __nv_bfloat16*>(d_v);
+  a.out = static_cast<__nv_bfloat16*>(d_out);
+  a.lse = d_lse; a.kv_len = d_kv_len; a.mask = d_mask;
+  a.q_b = strides[0]; a.q_n = strides[1]; a.q_h = strides[2];
+  a.kv_b = strides[3]; a.kv_h = strides[4]; a.kv_l = strides[5];
+  a.o_b = strides[6]; a.o_n = strides[7]; a.o_h = strides[8];
+  a.B = B; a.H = H; a.group = H / H_kv; a.N = N; a.Wm = (N + 31) / 32;
+  a.S = choose_splits(B, H, max_kv);
+  a.scale_log2 = scale * kLog2e;
+  a.ws_o = nullptr; a.ws_ml = nullptr;
+  if (a.S > 1) {
+    size_t need = rest_tree_attention_workspace_bytes(B, H, N, D, max_kv);
+    if (!d_ws) return REST_INVALID_ARG;
+    if (ws_bytes < need) return REST_WORKSPACE_TOO_SMALL;
+    a.ws_o = static_cast<float*>(d_ws);
+    a.ws_ml = a.ws_o + (size_t)B * H * a.S * N * kD;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t smem = attn_smem_bytes(N);
+  REST_CUDA_TRY(cudaFuncSetAttribute(tree_attention_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  tree_attention_kernel<<<B * H * a.S, (N / 16) * 32, smem, st>>>(a);
+  rest::count_launch();
+  REST_CUDA_TRY(cudaGetLastError());
+  if (a.S > 1) {
+    const int64_t units = (int64_t)B * H * N;
+    tree_attention_combine_kernel<<<(unsigned)((units + 3) / 4), 128, 0, st>>>(a);
+    rest::count_launch();
+    REST_CUDA_TRY(cudaGetLastError());
+  }
+  return REST_OK;
+}
