@@ -57,7 +57,7 @@ extern "C" rest_status rest_accept(const int32_t* d_tokens, const int32_t* d_par
   if (B < 0 || N < 1 || max_depth < 0) return REST_INVALID_ARG;
   if (B == 0) return REST_OK;
   if (!d_tokens || !d_parents || !d_n_nodes || !d_verifier_tokens || !d_accept_len ||
-      !d_accept_nodes || !d_out_tokens)
+      (!d_accept_nodes && max_depth > 0) || !d_out_tokens)
     return REST_INVALID_ARG;
   int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
   rest_accept_kernel<<<blocks, kWarpsPerBlock * 32, 0, static_cast<cudaStream_t>(stream)>>>(

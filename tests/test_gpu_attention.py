@@ -1,0 +1,118 @@
+"""Parity of rest_tree_attention with the fp64 oracle.
+
+Tolerance (from the arithmetic: bf16 inputs, bf16-rounded probabilities, fp32 accumulation,
+bf16 output, values ~N(0,1)): every element within 1e-2 absolute of the fp64 result, and every
+(context, node, head) output row within 2e-2 relative L2 error."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import datagen
+import oracle
+import paper_2311_08252_b200 as rest
+from gpu_util import attention_errors, bits, to_dev
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 1e-2
+MAX_REL = 2e-2
+
+
+def run_case(seed, B, H, N, L, Lcap=None, H_kv=None, kv_len=None, n_nodes=None, max_depth=8,
+             want_lse=True, scale=None):
+    D = 128
+    Lcap = (L + N) if Lcap is None else Lcap
+    q, k, v = datagen.make_qkv(seed, B, H, N, D, Lcap, H_kv=H_kv)
+    masks = []
+    for b in range(B):
+        _, _, mk = datagen.make_random_tree(seed * 100 + b, N, max_depth, n_nodes)
+        masks.append(mk)
+    mask = np.stack(masks)
+    kv_len = np.full(B, L, np.int32) if kv_len is None else np.asarray(kv_len, np.int32)
+    scale = 1.0 / math.sqrt(D) if scale is None else scale
+    ref, ref_lse = oracle.tree_attention(bits(q), bits(k), bits(v), kv_len, mask, scale,
+                                         H_kv=H_kv, want_lse=True)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device="cuda:0") if want_lse else None
+    out = rest.rest_tree_attention(q.cuda(), k.cuda(), v.cuda(), to_dev(kv_len), to_dev(mask),
+                                   scale, lse=lse)
+    torch.cuda.synchronize()
+    max_abs, max_rel = attention_errors(out, ref)
+    assert max_abs <= MAX_ABS and max_rel <= MAX_REL, (max_abs, max_rel)
+    if want_lse:
+        assert np.abs(lse.cpu().numpy().astype(np.float64) - ref_lse).max() <= 2e-3
+    return out, ref
+
+
+@pytest.mark.parametrize("B,H,N,L", [
+    (1, 32, 64, 256),        # tiny workload shape: split keys
+    (2, 4, 64, 37),          # prefix shorter than one tile, tree keys straddle tiles
+    (1, 2, 16, 0),           # no prefix at all
+    (3, 5, 128, 1000),       # N = 128, ragged tail
+    (2, 3, 48, 200),         # N not a multiple of 32
+    (1, 1, 64, 4096 + 17),   # many splits for one head
+    (20, 16, 64, 513),       # enough units for a single split: direct output path
+])
+def test_matches_fp64_oracle(B, H, N, L):
+    run_case(7, B, H, N, L)
+
+
+def test_ragged_batch_grouped_heads_padding_nodes_and_strides():
+    # different prefix lengths per context (some splits end up empty), grouped KV heads,
+    # trees with unused slots, KV buffer longer than needed
+    run_case(11, 4, 8, 64, 700, Lcap=900, H_kv=2, kv_len=[700, 1, 333, 64], n_nodes=41)
+    run_case(12, 2, 6, 32, 90, H_kv=3, kv_len=[90, 31], n_nodes=1, scale=0.2)
+
+
+def test_invariants_on_the_gpu_output():
+    B, H, N, L, D = 1, 2, 64, 130, 128
+    q, k, v = datagen.make_qkv(3, B, H, N, D, L + N)
+    par, dep, mask = datagen.make_random_tree(5, N, 8)
+    mask = mask[None].copy()
+    kv_len = to_dev(np.array([L], np.int32))
+    # constant V -> exactly that constant
+    vc = torch.full_like(v, 1.5)
+    out = rest.rest_tree_attention(q.cuda(), k.cuda(), vc.cuda(), kv_len, to_dev(mask), 0.1)
+    assert torch.allclose(out.float().cpu(), torch.full((B, N, H, D), 1.5), atol=8e-3)
+    # zero K -> mean of the allowed V rows
+    out = rest.rest_tree_attention(q.cuda(), torch.zeros_like(k).cuda(), v.cuda(), kv_len,
+                                   to_dev(mask), 0.1).float().cpu()
+    for i in (0, 17, 63):
+        rows, j = list(range(L)), i
+        while j >= 0:
+            rows.append(L + j)
+            j = int(par[j])
+        want = v[0][:, rows].float().mean(1)
+        assert torch.allclose(out[0, i], want, atol=1e-2)
+    # permuting the prefix rows of K and V together changes (almost) nothing
+    base = rest.rest_tree_attention(q.cuda(), k.cuda(), v.cuda(), kv_len, to_dev(mask), 0.1).float().cpu()
+    perm = torch.cat([torch.randperm(L, generator=torch.Generator().manual_seed(1)),
+                      torch.arange(L, L + N)])
+    out = rest.rest_tree_attention(q.cuda(), k[:, :, perm].contiguous().cuda(),
+                                   v[:, :, perm].contiguous().cuda(), kv_len, to_dev(mask), 0.1).float().cpu()
+    assert (out - base).abs().max() <= 1e-2
+
+
+def test_attention_on_drafted_masks_full_head_count():
+    # masks produced by rest_draft, 32 heads x 128, KV prefix 2048: the single-stream shape
+    from gpu_util import gpu_draft
+    w = datagen.WORKLOADS["single_stream"].scaled(n_tokens=1_000_000)
+    T = datagen.make_tokens(w)
+    sa = datagen.build_suffix_array(T, w.vocab)
+    ctx = datagen.make_contexts(w, T, B=2, Lc=256)
+    ref_d = oracle.draft(T, sa, w.vocab, ctx, [256, 256], K=w.K, m=w.m, N=w.N)
+    got_d, out_d = gpu_draft(T, sa, w.vocab, ctx, [256, 256], K=w.K, m=w.m, N=w.N)
+    assert np.array_equal(got_d["mask"], ref_d["mask"])
+    L = 2048
+    q, k, v = datagen.make_qkv(21, 2, 32, w.N, 128, L + w.N)
+    scale = 1.0 / math.sqrt(128)
+    out = rest.rest_tree_attention(q.cuda(), k.cuda(), v.cuda(), to_dev(np.array([L, L], np.int32)),
+                                   out_d.mask, scale)
+    torch.cuda.synchronize()
+    # the oracle on a sample of heads (all nodes): fp64 over 2 x 4 heads
+    hs = [0, 13, 31, 7]
+    ref = oracle.tree_attention(bits(q[:, :, hs]), bits(k[:, hs]), bits(v[:, hs]), [L, L],
+                                ref_d["mask"], scale)
+    max_abs, max_rel = attention_errors(out[:, :, hs], ref)
+    assert max_abs <= MAX_ABS and max_rel <= MAX_REL, (max_abs, max_rel)

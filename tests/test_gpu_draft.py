@@ -1,0 +1,117 @@
+"""Parity of rest_draft (CUDA, through the C ABI) with the CPU oracle: bit-exact match
+lengths, ranges, tokens, parents, depths, position ids, masks, weights and status."""
+import numpy as np
+import pytest
+
+import datagen
+import oracle
+from gpu_util import assert_draft_equal, gpu_draft
+
+pytestmark = pytest.mark.gpu
+
+
+def test_worked_example():
+    T = np.array([1, 2, 3, 1, 2, 4, 1, 2, 3, 5], np.int32)
+    sa = oracle.suffix_array(T).astype(np.int32)
+    ctx = np.array([[9, 7, 1, 2]], np.int32)
+    got, _ = gpu_draft(T, sa, 10, ctx, [4], validate=True, m=3, N=4)
+    assert got["tokens"][0].tolist() == [3, 4, 1, 5]
+    assert got["parents"][0].tolist() == [-1, -1, 0, 0]
+    assert got["mask"][0, :, 0].tolist() == [1, 2, 5, 9]
+    assert got["node_count"][0].tolist() == [2, 1, 1, 1]
+    assert got["match_n"][0] == 2 and got["match_range"][0].tolist() == [0, 3]
+
+
+@pytest.mark.parametrize("seed,vocab,n_tok,K,m,N,sa_bytes", [
+    (1, 3, 400, 5000, 4, 16, 4),
+    (2, 4, 1500, 5000, 6, 40, 8),
+    (3, 2, 3000, 5000, 10, 64, 4),      # binary alphabet: thousands of matches, deep shared prefixes
+    (4, 5, 2500, 7, 5, 24, 4),          # K binds
+    (5, 3, 9000, 600, 16, 128, 8),      # K binds, rows span two gather iterations, N = 128, m = 16
+    (6, 8, 4096, 5000, 10, 64, 4),
+    (7, 2, 40000, 20000, 16, 128, 4),   # stress shape: K = 20000, m = 16
+    (8, 3, 70000, 32768, 1, 1, 4),      # extremes: K max, m = 1, N = 1
+])
+def test_small_alphabets_match_oracle(seed, vocab, n_tok, K, m, N, sa_bytes):
+    rng = np.random.default_rng(seed)
+    T = rng.integers(0, vocab, n_tok).astype(np.int32)
+    sa = datagen.build_suffix_array(T, vocab, W=32, sa_bytes=sa_bytes)
+    B, Lc = 40, 24
+    ctx = rng.integers(0, vocab, (B, Lc)).astype(np.int32)
+    for b in range(0, B, 3):
+        p = int(rng.integers(0, n_tok - Lc))
+        ctx[b] = T[p:p + Lc]
+    ctx[1] = T[n_tok - Lc - 2:n_tok - 2]          # continuations cut by the end of the stream
+    ctx[4] = T[n_tok - Lc:]                        # match ends exactly at the end
+    ctx_len = rng.integers(0, Lc + 1, B).astype(np.int32)
+    ctx_len[:8] = Lc
+    for mode in (0, 1):
+        kw = dict(K=K, m=m, N=N, sample_mode=mode)
+        ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
+        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, **kw)
+        assert_draft_equal(got, ref, f"mode {mode}")
+
+
+@pytest.mark.parametrize("name,n_tok,B", [
+    ("tiny", 1_000_000, 256), ("single_stream", 3_000_000, 128), ("batched", 2_000_000, 256),
+    ("large", 2_000_000, 64), ("stress", 2_000_000, 128)])
+def test_workload_recipes_match_oracle(name, n_tok, B):
+    w = datagen.WORKLOADS[name].scaled(n_tokens=n_tok)
+    T = datagen.make_tokens(w)
+    sa = datagen.build_suffix_array(T, w.vocab, W=32, sa_bytes=w.sa_bytes)
+    ctx = datagen.make_contexts(w, T, B=B, Lc=min(w.Lc, 512))
+    ctx_len = np.full(B, ctx.shape[1], np.int32)
+    kw = dict(K=w.K, m=w.m, N=w.N, n_max=w.n_max, n_min=w.n_min)
+    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, **kw)
+    assert_draft_equal(got, ref, name)
+    assert (ref["n_nodes"] > 0).sum() > B // 2
+
+
+def test_other_suffix_limits_and_repeatability():
+    w = datagen.WORKLOADS["tiny"].scaled(n_tokens=300_000)
+    T = datagen.make_tokens(w)
+    sa = datagen.build_suffix_array(T, w.vocab)
+    ctx = datagen.make_contexts(w, T, B=96, Lc=40)
+    ctx_len = np.full(96, 40, np.int32)
+    for n_max, n_min in ((16, 1), (8, 3), (4, 4), (1, 1)):
+        kw = dict(K=300, m=7, N=48, n_max=n_max, n_min=n_min)
+        ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+        assert_draft_equal(got, ref, f"n_max={n_max} n_min={n_min}")
+        again, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+        assert_draft_equal(again, got, "second run")
+
+
+def test_bad_context_tokens_and_corrupt_datastore():
+    import paper_2311_08252_b200 as rest
+    import torch
+    T = np.array([1, 2, 3, 1, 2, 4, 1, 2, 3, 5], np.int32)
+    sa = oracle.suffix_array(T).astype(np.int32)
+    ctx = np.array([[9, 7, 1, 2], [9, 7, 1, 99], [9, 7, -1, 2]], np.int32)
+    ref = oracle.draft(T, sa, 10, ctx, [4, 4, 4], m=3, N=4)
+    got, _ = gpu_draft(T, sa, 10, ctx, [4, 4, 4], m=3, N=4)
+    assert_draft_equal(got, ref)
+    assert got["status"].tolist() == [0, 1, 1]
+    # validation refuses a non-permutation, an unsorted array and an out-of-range token
+    dev = torch.device("cuda:0")
+    for mutate in ("dup", "swap", "range", "token"):
+        s2, t2 = sa.copy(), T.copy()
+        if mutate == "dup":
+            s2[3] = s2[4]
+        elif mutate == "swap":
+            s2[[0, 5]] = s2[[5, 0]]
+        elif mutate == "range":
+            s2[2] = 1000
+        else:
+            t2[3] = 10
+        with pytest.raises(rest.RestError, match="validation"):
+            rest.Datastore(torch.from_numpy(t2).to(dev), torch.from_numpy(s2).to(dev), 10, validate=True)
+    # without validation an out-of-range entry met while gathering is reported, never dereferenced
+    Z = np.zeros(64, np.int32)
+    saz = oracle.suffix_array(Z).astype(np.int32)
+    bad = saz.copy()
+    bad[40] = 1000
+    got, _ = gpu_draft(Z, bad, 1, np.zeros((1, 20), np.int32), [20], m=3, N=4)
+    assert got["status"].tolist() == [2] and got["n_nodes"].tolist() == [0]
+    assert (got["tokens"] == -1).all()
