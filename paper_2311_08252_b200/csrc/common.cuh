@@ -10,6 +10,9 @@ namespace rest {
 // Records the text of a failed CUDA call for rest_last_cuda_error(); returns REST_CUDA_ERROR.
 rest_status note_cuda_error(cudaError_t e, const char* where);
 void count_launch(int n = 1);
+// Raises a kernel's dynamic shared-memory limit on the current device when `bytes` exceeds
+// what was set before (kernel_slot: small per-kernel index used for the per-device cache).
+cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t bytes);
 
 #define REST_CUDA_TRY(expr)                                              \
   do {                                                                   \

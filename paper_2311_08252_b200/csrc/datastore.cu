@@ -22,6 +22,20 @@ rest_status note_cuda_error(cudaError_t e, const char* where) {
 }
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t bytes) {
+  constexpr int kMaxDev = 64, kSlots = 8;
+  static std::atomic<size_t> set_bytes[kMaxDev][kSlots];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < kMaxDev && kernel_slot >= 0 && kernel_slot < kSlots;
+  if (cached && set_bytes[dev][kernel_slot].load(std::memory_order_relaxed) >= bytes)
+    return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && cached) set_bytes[dev][kernel_slot].store(bytes, std::memory_order_relaxed);
+  return e;
+}
+
 }  // namespace rest
 
 namespace {

@@ -570,7 +570,8 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   size_t smem = draft_smem_bytes(prm->K, prm->m, &a.kcap, &a.nwords);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto kern = ds->v.sa_bytes == 4 ? rest_draft_kernel<int32_t> : rest_draft_kernel<int64_t>;
-  REST_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
+                                          ds->v.sa_bytes == 4 ? 0 : 1, smem));
   kern<<<B, kThreads, smem, st>>>(a);
   rest::count_launch();
   REST_CUDA_TRY(cudaGetLastError());

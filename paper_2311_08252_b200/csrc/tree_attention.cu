@@ -384,8 +384,8 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t smem = attn_smem_bytes(N);
-  REST_CUDA_TRY(cudaFuncSetAttribute(tree_attention_kernel,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_kernel),
+                                          2, smem));
   tree_attention_kernel<<<B * H * a.S, (N / 16) * 32, smem, st>>>(a);
   rest::count_launch();
   REST_CUDA_TRY(cudaGetLastError());
