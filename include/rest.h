@@ -161,6 +161,37 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
                                 float* d_lse, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
+ * rest_tree_attention_static_scratch - rest_tree_attention for callers that cannot allocate.
+ *
+ * (The paper has no counterpart; this is a packaging variant of the call above.)
+ *
+ * Some users of this library cannot obtain the workspace that rest_tree_attention asks for:
+ * a serving process that handed every free byte of device memory to its own KV-cache pool at
+ * start-up, or a decode loop whose rules forbid allocation calls because cudaMalloc/cudaFree
+ * may stall the whole device.  For them the split-KV partials live in a fixed array of
+ * REST_STATIC_SCRATCH_BYTES (16 MiB) inside the library image.  Every GPU that loads the
+ * library holds that array until the process exits, whether or not this call is used.
+ *
+ *   - Arguments, layouts, results and limits are those of rest_tree_attention, without
+ *     d_ws / ws_bytes.  The call itself performs no device or host allocation.
+ *   - Returns REST_WORKSPACE_TOO_SMALL, launching nothing, when
+ *     rest_tree_attention_workspace_bytes(B, H, N, D, max_kv) exceeds REST_STATIC_SCRATCH_BYTES
+ *     (e.g. B = 1, H = 32, N = 64, max_kv = 2112 needs 10.2 MiB and fits; shapes with enough
+ *     (context, head) pairs to fill the GPU need no scratch at all and always fit).
+ *   - The first call on each device looks up the array's device address (one runtime query,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     That is harmless here: each call writes every partial it later reads, so nothing has to
+ *     start at zero.  But two calls whose kernels may overlap on the GPU (different streams)
+ *     race on the array: serialise them.
+ */
+enum { REST_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 };
+rest_status rest_tree_attention_static_scratch(
+    const void* d_q, const void* d_k, const void* d_v, const int64_t* strides,
+    const int32_t* d_kv_len, const uint32_t* d_mask, int32_t B, int32_t H, int32_t H_kv, int32_t N,
+    int32_t D, int32_t max_kv, float scale, void* d_out, float* d_lse, void* stream);
+
+/*
  * rest_accept - draft acceptance (Sec. 3.2 "Draft acceptance": draft tokens are accepted from
  * the start while they coincide with the tokens sampled from the verifier; everything after
  * the first mismatch is rejected).

@@ -28,6 +28,7 @@ EXPORTS = (
     "rest_datastore_aux_bytes", "rest_datastore_create", "rest_datastore_destroy",
     "rest_draft_workspace_bytes", "rest_draft",
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
+    "rest_tree_attention_static_scratch",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -74,6 +75,10 @@ def lib():
     L.rest_tree_attention.restype = i32
     L.rest_tree_attention.argtypes = [vp, vp, vp, ctypes.POINTER(i64), vp, vp, i32, i32, i32, i32,
                                       i32, i32, ctypes.c_float, vp, vp, vp, sz, vp]
+    L.rest_tree_attention_static_scratch.restype = i32
+    L.rest_tree_attention_static_scratch.argtypes = [vp, vp, vp, ctypes.POINTER(i64), vp, vp, i32,
+                                                     i32, i32, i32, i32, i32, ctypes.c_float, vp,
+                                                     vp, vp]
     L.rest_accept.restype = i32
     L.rest_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     L.rest_status_string.restype = ctypes.c_char_p
@@ -240,6 +245,27 @@ def rest_tree_attention(q, k, v, kv_len, mask, scale, max_kv=None, out=None, lse
                                0 if workspace is None else workspace.numel() * workspace.element_size(),
                                _stream(stream))
     _check(rc, "rest_tree_attention")
+    return out
+
+
+def rest_tree_attention_static_scratch(q, k, v, kv_len, mask, scale, out, max_kv=None, lse=None,
+                                       stream=None):
+    """rest_tree_attention without a workspace argument, for callers that must not allocate:
+    the split partials go to a fixed 16 MiB array inside the library.  `out` (bf16 [B,N,H,D])
+    is supplied by the caller, so this wrapper allocates nothing on the device either.
+    Raises RestError (workspace too small) when the shape needs more than the fixed array.
+    Calls share that array: do not let two of them overlap on the GPU."""
+    L = lib()
+    B, N, H, D = q.shape
+    H_kv, Lcap = k.shape[1], k.shape[2]
+    max_kv = Lcap if max_kv is None else int(max_kv)
+    strides = (ctypes.c_int64 * 9)(q.stride(0), q.stride(1), q.stride(2),
+                                   k.stride(0), k.stride(1), k.stride(2),
+                                   out.stride(0), out.stride(1), out.stride(2))
+    rc = L.rest_tree_attention_static_scratch(
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), strides, kv_len.data_ptr(), mask.data_ptr(),
+        B, H, H_kv, N, D, max_kv, float(scale), out.data_ptr(), _ptr(lse), _stream(stream))
+    _check(rc, "rest_tree_attention_static_scratch")
     return out
 
 

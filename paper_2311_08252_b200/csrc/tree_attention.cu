@@ -397,3 +397,47 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   }
   return REST_OK;
 }
+
+// ---------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate device memory.
+//
+// The split partials live in a fixed array that is part of the library image, so the caller
+// passes no workspace.  The array is a device symbol: its name is only meaningful in device
+// code, so host code asks the runtime for its device address once per device (with that
+// device current) and hands that address to the unchanged rest_tree_attention.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticScratchBytes = REST_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device
+
+rest_status static_scratch_pointer(void** out) {
+  int dev = 0;
+  REST_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return REST_UNSUPPORTED;
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    REST_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    g_static_scratch_addr[dev] = p;
+  }
+  *out = g_static_scratch_addr[dev];
+  return REST_OK;
+}
+
+}  // namespace
+
+extern "C" rest_status rest_tree_attention_static_scratch(
+    const void* d_q, const void* d_k, const void* d_v, const int64_t* strides,
+    const int32_t* d_kv_len, const uint32_t* d_mask, int32_t B, int32_t H, int32_t H_kv, int32_t N,
+    int32_t D, int32_t max_kv, float scale, void* d_out, float* d_lse, void* stream) {
+  const size_t need = rest_tree_attention_workspace_bytes(B, H, N, D, max_kv);
+  if (need > kStaticScratchBytes) return REST_WORKSPACE_TOO_SMALL;
+  void* scratch = nullptr;
+  rest_status st = static_scratch_pointer(&scratch);
+  if (st != REST_OK) return st;
+  return rest_tree_attention(d_q, d_k, d_v, strides, d_kv_len, d_mask, B, H, H_kv, N, D, max_kv,
+                             scale, d_out, d_lse, scratch, kStaticScratchBytes, stream);
+}
