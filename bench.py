@@ -226,6 +226,7 @@ def main():
 
     import torch
     import paper_2311_08252_b200 as rest
+    from paper_2311_08252_b200.sharding import max_over_ranks, shard_bounds, whole_job_throughput
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -256,7 +257,10 @@ def main():
 
     B, N, H, D, L, layers = w.B, w.N, w.H, w.D, w.L, w.layers
     pool = N_CTX_POOL
-    ctx_np = datagen.make_contexts(w, T, B=pool * B, Lc=w.Lc, salt=rank).reshape(pool, B, w.Lc)
+    # the global batch of every pooled step is world*B contexts; this rank owns one slice
+    all_ctx = datagen.make_contexts(w, T, B=pool * B * world, Lc=w.Lc).reshape(pool, B * world, w.Lc)
+    c0, c1 = shard_bounds(B * world, rank, world)
+    ctx_np = np.ascontiguousarray(all_ctx[:, c0:c1])
     ctx_len_np = np.full(B, w.Lc, np.int32)
     d_ctx = torch.from_numpy(ctx_np).to(dev)
     d_ctx_len = torch.from_numpy(ctx_len_np).to(dev)
@@ -332,12 +336,7 @@ def main():
             fn(i)
         e1.record(stream)
         barrier()
-        sec = e0.elapsed_time(e1) / 1e3
-        if dist is not None:
-            t = torch.tensor([sec], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            sec = float(t.item())
-        return sec
+        return max_over_ranks(e0.elapsed_time(e1) / 1e3, dist, dev)
 
     for j in range(3):          # plain calls first (also sets kernel attributes before capture)
         step_calls(j)
@@ -422,7 +421,7 @@ def main():
     a_bytes = attention_bytes(B, H, H, N, D, L)
     d_bytes = draft_bytes(w.n_tokens, w.sa_bytes, w.n_min, w.n_max, kp_sum / (pool * B), w.m, N) * B
     line = {
-        "metric": METRIC, "value": world * B * args.steps / sec, "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_throughput(B, args.steps, world, sec), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": sec / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(w, args),
