@@ -358,7 +358,7 @@ def main():
     draft_graphs = [capture(draft_calls, j)[0] for j in range(pool)]
     attn_graph, _ = capture(attn_calls, 0)
     accept_graphs = [capture(accept_calls, j)[0] for j in range(pool)]
-    n_part = max(args.steps, 50)
+    n_part = max(args.steps, 3)
     for i in range(3):
         draft_graphs[i].replay(); attn_graph.replay(); accept_graphs[i].replay()
     t_draft = timed(lambda i: draft_graphs[i % pool].replay(), n_part) / n_part
@@ -408,7 +408,7 @@ def main():
 
     for i in range(3):
         e2e_step(i)
-    n_e2e = max(20, args.steps // 4)
+    n_e2e = max(3, args.steps // 4)
     t_e2e = timed(e2e_step, n_e2e) / n_e2e
     clocks = sampler.stop() if rank == 0 else None
 

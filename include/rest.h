@@ -169,15 +169,16 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  * a serving process that handed every free byte of device memory to its own KV-cache pool at
  * start-up, or a decode loop whose rules forbid allocation calls because cudaMalloc/cudaFree
  * may stall the whole device.  For them the split-KV partials live in a fixed array of
- * REST_STATIC_SCRATCH_BYTES (16 MiB) inside the library image.  Every GPU that loads the
+ * REST_STATIC_SCRATCH_BYTES (1 MiB) inside the library image.  Every GPU that loads the
  * library holds that array until the process exits, whether or not this call is used.
  *
  *   - Arguments, layouts, results and limits are those of rest_tree_attention, without
  *     d_ws / ws_bytes.  The call itself performs no device or host allocation.
  *   - Returns REST_WORKSPACE_TOO_SMALL, launching nothing, when
- *     rest_tree_attention_workspace_bytes(B, H, N, D, max_kv) exceeds REST_STATIC_SCRATCH_BYTES
- *     (e.g. B = 1, H = 32, N = 64, max_kv = 2112 needs 10.2 MiB and fits; shapes with enough
- *     (context, head) pairs to fill the GPU need no scratch at all and always fit).
+ *     rest_tree_attention_workspace_bytes(B, H, N, D, max_kv) exceeds REST_STATIC_SCRATCH_BYTES.
+ *     Scratch is only needed when one (context, head) pair is cut into more than 8 key ranges,
+ *     i.e. for very few pairs with long caches: B*H = 2, N = 64, max_kv = 4160 needs 0.51 MiB
+ *     and fits; B*H = 2, N = 64, max_kv = 8256 needs 1.02 MiB and is refused.
  *   - The first call on each device looks up the array's device address (one runtime query,
  *     with that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.
@@ -185,7 +186,7 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  *     start at zero.  But two calls whose kernels may overlap on the GPU (different streams)
  *     race on the array: serialise them.
  */
-enum { REST_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024 };
+enum { REST_STATIC_SCRATCH_BYTES = 1024 * 1024 };
 rest_status rest_tree_attention_static_scratch(
     const void* d_q, const void* d_k, const void* d_v, const int64_t* strides,
     const int32_t* d_kv_len, const uint32_t* d_mask, int32_t B, int32_t H, int32_t H_kv, int32_t N,

@@ -251,7 +251,7 @@ def rest_tree_attention(q, k, v, kv_len, mask, scale, max_kv=None, out=None, lse
 def rest_tree_attention_static_scratch(q, k, v, kv_len, mask, scale, out, max_kv=None, lse=None,
                                        stream=None):
     """rest_tree_attention without a workspace argument, for callers that must not allocate:
-    the split partials go to a fixed 16 MiB array inside the library.  `out` (bf16 [B,N,H,D])
+    the split partials go to a fixed 1 MiB array inside the library.  `out` (bf16 [B,N,H,D])
     is supplied by the caller, so this wrapper allocates nothing on the device either.
     Raises RestError (workspace too small) when the shape needs more than the fixed array.
     Calls share that array: do not let two of them overlap on the GPU."""

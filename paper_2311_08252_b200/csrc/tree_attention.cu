@@ -3,12 +3,17 @@
 //
 // Split-KV flash-decode layout: one thread block per (context, head, key split).  A block
 // holds the N x 128 query tile as tensor-core A fragments in registers (16 rows per warp)
-// and streams 64-key K/V tiles through a double-buffered, XOR-swizzled shared-memory ring
-// filled with 16-byte asynchronous copies.  Per tile: S = Q K^T (bf16 tensor-core MMA, fp32
+// and streams 64-key K/V tiles through a three-deep, XOR-swizzled shared-memory ring filled
+// with 16-byte asynchronous copies.  Per tile: S = Q K^T (bf16 tensor-core MMA, fp32
 // accumulate), tree mask on the tiles that reach past the prefix, online softmax in base 2,
-// O += P V.  With one split the block normalises and writes bf16 output directly; otherwise
-// it writes un-normalised fp32 partials (plus running max and sum) and a second kernel merges
-// the splits.
+// O += P V.
+//
+// The splits of one (context, head) form a thread-block cluster (up to 8 blocks): each block
+// parks its un-normalised partial in its own shared memory, and after a cluster barrier every
+// block merges a slice of the rows straight out of its peers' shared memory (distributed
+// shared memory) and writes bf16 output.  Only when more than 8 splits are needed do the
+// cluster-merged partials go to the caller's workspace for a second, small merge kernel.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -17,11 +22,15 @@
 #include "common.cuh"
 #include "rest.h"
 
+namespace cg = cooperative_groups;
+
 namespace {
 
 constexpr int kD = REST_HEAD_DIM;     // 128
 constexpr int kBN = 64;               // keys per tile
-constexpr int kStages = 2;
+constexpr int kStages = 3;
+constexpr int kOStride = kD + 4;         // floats per row of a parked partial (bank spread)
+constexpr int kMaxCluster = 8;
 constexpr int kRowBytes = kD * 2;     // 256
 constexpr int kTileBytes = kBN * kRowBytes;   // 16 KB
 constexpr float kLog2e = 1.4426950408889634f;
@@ -34,10 +43,13 @@ struct AttnArgs {
   float* lse;
   const int32_t* kv_len;
   const uint32_t* mask;
-  float* ws_o;      // [B,H,S,N,128] fp32 partial numerators
-  float* ws_ml;     // [B,H,S,N,2]   running max (base-2 units) and sum
+  float* ws_o;      // [B,H,Sp,N,128] fp32 partial numerators (Sp = clusters per (b,h))
+  float* ws_ml;     // [B,H,Sp,N,2]   running max (base-2 units) and sum
   int64_t q_b, q_n, q_h, kv_b, kv_h, kv_l, o_b, o_n, o_h;
-  int B, H, group, N, Wm, S;
+  int B, H, group, N, Wm;
+  int S;            // key splits per (context, head) = C * Sp
+  int C;            // blocks per cluster
+  int Sp;           // clusters per (context, head); > 1 needs the merge kernel
   float scale_log2;
 };
 
@@ -103,9 +115,8 @@ tree_attention_kernel(AttnArgs a) {
   const int L = a.kv_len[b];
   const int total = L + N;
   const int ntiles = (total + kBN - 1) / kBN;
-  const int tps = (ntiles + a.S - 1) / a.S;
-  const int t0 = split * tps;
-  const int t1 = min(ntiles, t0 + tps);
+  const int t0 = (int)(((int64_t)split * ntiles) / a.S);         // balanced partition of the tiles
+  const int t1 = (int)(((int64_t)(split + 1) * ntiles) / a.S);
 
   const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h;
   const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
@@ -135,6 +146,8 @@ tree_attention_kernel(AttnArgs a) {
   };
   if (t0 < t1) load_tile(t0, 0);
   cp_async_commit();
+  if (t0 + 1 < t1) load_tile(t0 + 1, 1);
+  cp_async_commit();
 
   float o[16][4];
 #pragma unroll
@@ -144,14 +157,10 @@ tree_attention_kernel(AttnArgs a) {
   const int r0 = warp * 16 + g, r1 = r0 + 8;
 
   for (int t = t0; t < t1; ++t) {
-    const int stage = (t - t0) & 1;
-    if (t + 1 < t1) {
-      load_tile(t + 1, stage ^ 1);
-      cp_async_commit();
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
+    const int stage = (t - t0) % kStages;
+    if (t + 2 < t1) load_tile(t + 2, (t - t0 + 2) % kStages);   // that slot was drained at t - 1
+    cp_async_commit();                                          // one group per iteration, maybe empty
+    cp_async_wait<2>();                                         // tile t (and Q) have landed
     __syncthreads();
     if (t == t0) {
 #pragma unroll
@@ -246,7 +255,8 @@ tree_attention_kernel(AttnArgs a) {
     }
     __syncthreads();
   }
-  if (t0 >= t1) { cp_async_wait<0>(); }
+  cp_async_wait<0>();
+  __syncthreads();   // every warp is done with the K/V ring (and Q tile): reuse it below
 
   l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1);
   l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
@@ -267,21 +277,72 @@ tree_attention_kernel(AttnArgs a) {
       lp[r0] = (m0 + log2f(l0)) * kLn2;
       lp[r1] = (m1 + log2f(l1)) * kLn2;
     }
-  } else {
-    const int64_t base = (((int64_t)b * a.H + h) * a.S + split) * N;
-    float* po = a.ws_o + base * kD;
+    return;
+  }
+
+  // Park this block's partial in its own shared memory: O [N][kOStride] fp32, then (max, sum).
+  float* sO = reinterpret_cast<float*>(smem);
+  float* sML = sO + N * kOStride;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      int col = i * 8 + t4 * 2;
-      *reinterpret_cast<float2*>(po + (int64_t)r0 * kD + col) = make_float2(o[i][0], o[i][1]);
-      *reinterpret_cast<float2*>(po + (int64_t)r1 * kD + col) = make_float2(o[i][2], o[i][3]);
+  for (int i = 0; i < 16; ++i) {
+    int col = i * 8 + t4 * 2;
+    *reinterpret_cast<float2*>(sO + r0 * kOStride + col) = make_float2(o[i][0], o[i][1]);
+    *reinterpret_cast<float2*>(sO + r1 * kOStride + col) = make_float2(o[i][2], o[i][3]);
+  }
+  if (t4 == 0) {
+    sML[r0 * 2] = m0; sML[r0 * 2 + 1] = l0;
+    sML[r1 * 2] = m1; sML[r1 * 2 + 1] = l1;
+  }
+  cg::cluster_group cluster = cg::this_cluster();
+  cluster.sync();
+
+  // Merge rows [rank*R, rank*R + R) over the C blocks of the cluster, 4 output dims per thread.
+  const int C = a.C;
+  const int rank = (int)cluster.block_rank();
+  const int R = (N + C - 1) / C;
+  const int sup = split / C;
+  for (int idx = tid; idx < R * 32; idx += nthreads) {
+    const int row = rank * R + (idx >> 5), c4 = idx & 31;
+    if (row >= N) continue;
+    // issue every remote read before using any of them (one round trip, not 2*C of them);
+    // an empty split parked zeros with max = -inf, so its weight is 0 and its data harmless
+    float2 ml[kMaxCluster];
+    float4 ov[kMaxCluster];
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p) {
+      if (p < C) {
+        ml[p] = *reinterpret_cast<const float2*>(cluster.map_shared_rank(sML, p) + row * 2);
+        ov[p] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sO, p) + row * kOStride + c4 * 4);
+      }
     }
-    if (t4 == 0) {
-      float* pm = a.ws_ml + base * 2;
-      pm[r0 * 2] = m0; pm[r0 * 2 + 1] = l0;
-      pm[r1 * 2] = m1; pm[r1 * 2 + 1] = l1;
+    float M = -INFINITY;
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p)
+      if (p < C) M = fmaxf(M, ml[p].x);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lsum = 0.f;
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p) {
+      if (p < C) {
+        const float w = (ml[p].x == -INFINITY) ? 0.f : exp2f(ml[p].x - M);
+        lsum += ml[p].y * w;
+        acc.x += ov[p].x * w; acc.y += ov[p].y * w; acc.z += ov[p].z * w; acc.w += ov[p].w * w;
+      }
+    }
+    if (a.Sp == 1) {
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      uint2 pk;
+      pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+      pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2*>(a.out + b * a.o_b + row * a.o_n + h * a.o_h + c4 * 4) = pk;
+      if (a.lse && c4 == 0) a.lse[((int64_t)b * a.H + h) * N + row] = (M + log2f(lsum)) * kLn2;
+    } else {
+      const int64_t base = ((((int64_t)b * a.H + h) * a.Sp + sup) * N + row);
+      *reinterpret_cast<float4*>(a.ws_o + base * kD + c4 * 4) = acc;
+      if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
     }
   }
+  cluster.sync();   // nobody leaves while a peer may still read its shared memory
 }
 
 // Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
@@ -295,18 +356,18 @@ tree_attention_combine_kernel(AttnArgs a) {
   const int64_t bh = unit / a.N;
   const int h = (int)(bh % a.H);
   const int64_t b = bh / a.H;
-  const float* pm = a.ws_ml + (bh * a.S * a.N + row) * 2;
+  const float* pm = a.ws_ml + (bh * a.Sp * a.N + row) * 2;
   float M = -INFINITY;
-  for (int s = 0; s < a.S; ++s) M = fmaxf(M, pm[(int64_t)s * a.N * 2]);
+  for (int s = 0; s < a.Sp; ++s) M = fmaxf(M, pm[(int64_t)s * a.N * 2]);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float lsum = 0.f;
-  for (int s = 0; s < a.S; ++s) {
+  for (int s = 0; s < a.Sp; ++s) {
     float ms = pm[(int64_t)s * a.N * 2], ls = pm[(int64_t)s * a.N * 2 + 1];
     float w = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
     lsum += ls * w;
     if (w != 0.f) {
       const float4 v = *reinterpret_cast<const float4*>(
-          a.ws_o + ((bh * a.S + s) * a.N + row) * kD + lane * 4);
+          a.ws_o + ((bh * a.Sp + s) * a.N + row) * kD + lane * 4);
       acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
     }
   }
@@ -319,16 +380,24 @@ tree_attention_combine_kernel(AttnArgs a) {
   if (a.lse && lane == 0) a.lse[bh * a.N + row] = (M + log2f(lsum)) * kLn2;
 }
 
-int choose_splits(int B, int H, int max_kv) {
+struct SplitPlan { int S, C, Sp; };
+
+// Key splits per (context, head): enough blocks to fill the GPU once (never a partial second
+// wave), at most one split per tile, rounded down to a whole number of clusters.
+SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
   const int64_t units = (int64_t)B * H;
-  int S = (int)((2 * kNumSMs + units - 1) / units);
-  const int cap = (ntiles + 1) / 2;   // at least two tiles per split
-  if (S > cap) S = cap;
-  if (S > 64) S = 64;
-  if (units >= 2 * kNumSMs) S = 1;
-  if (S < 1) S = 1;
-  return S;
+  const int blocks_per_sm = N <= 64 ? 2 : 1;
+  int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
+  if (S > ntiles) S = ntiles;
+  SplitPlan p;
+  if (S >= kMaxCluster) { p.C = kMaxCluster; p.S = (int)(S / kMaxCluster) * kMaxCluster; }
+  else if (S >= 4) { p.C = 4; p.S = 4; }
+  else if (S >= 2) { p.C = 2; p.S = 2; }
+  else { p.C = 1; p.S = 1; }
+  if (p.S > 512) p.S = 512;
+  p.Sp = p.S / p.C;
+  return p;
 }
 
 size_t attn_smem_bytes(int N) {
@@ -340,9 +409,9 @@ size_t attn_smem_bytes(int N) {
 extern "C" size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
                                                       int32_t max_kv) {
   if (B <= 0 || H <= 0 || N <= 0 || D != kD || max_kv <= 0) return 0;
-  const int S = choose_splits(B, H, max_kv);
-  if (S == 1) return 0;
-  return (size_t)B * H * S * N * (kD + 2) * sizeof(float);
+  const SplitPlan p = plan_splits(B, H, N, max_kv);
+  if (p.Sp == 1) return 0;
+  return (size_t)B * H * p.Sp * N * (kD + 2) * sizeof(float);
 }
 
 extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_v,
@@ -372,24 +441,36 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   a.kv_b = strides[3]; a.kv_h = strides[4]; a.kv_l = strides[5];
   a.o_b = strides[6]; a.o_n = strides[7]; a.o_h = strides[8];
   a.B = B; a.H = H; a.group = H / H_kv; a.N = N; a.Wm = (N + 31) / 32;
-  a.S = choose_splits(B, H, max_kv);
+  const SplitPlan plan = plan_splits(B, H, N, max_kv);
+  a.S = plan.S; a.C = plan.C; a.Sp = plan.Sp;
   a.scale_log2 = scale * kLog2e;
   a.ws_o = nullptr; a.ws_ml = nullptr;
-  if (a.S > 1) {
+  if (a.Sp > 1) {
     size_t need = rest_tree_attention_workspace_bytes(B, H, N, D, max_kv);
     if (!d_ws) return REST_INVALID_ARG;
     if (ws_bytes < need) return REST_WORKSPACE_TOO_SMALL;
     a.ws_o = static_cast<float*>(d_ws);
-    a.ws_ml = a.ws_o + (size_t)B * H * a.S * N * kD;
+    a.ws_ml = a.ws_o + (size_t)B * H * a.Sp * N * kD;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t smem = attn_smem_bytes(N);
   REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_kernel),
                                           2, smem));
-  tree_attention_kernel<<<B * H * a.S, (N / 16) * 32, smem, st>>>(a);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(B * H * a.S), 1, 1);
+  cfg.blockDim = dim3((unsigned)((N / 16) * 32), 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)a.C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_kernel, a));
   rest::count_launch();
-  REST_CUDA_TRY(cudaGetLastError());
-  if (a.S > 1) {
+  if (a.Sp > 1) {
     const int64_t units = (int64_t)B * H * N;
     tree_attention_combine_kernel<<<(unsigned)((units + 3) / 4), 128, 0, st>>>(a);
     rest::count_launch();

@@ -32,9 +32,11 @@ def test_status_strings_and_size_queries_without_a_gpu():
     assert L.rest_datastore_aux_bytes(64, 4, 10) == 2 * 4 + 256
     # many (context, head) units -> a single key split, no scratch
     assert rest.tree_attention_workspace_bytes(256, 32, 64, 128, 4160) == 0
-    # single stream -> split keys, fp32 partials of N*(D+2) floats per split
-    n = rest.tree_attention_workspace_bytes(1, 32, 64, 128, 2112)
-    assert n > 0 and n % (32 * 64 * 130 * 4) == 0
+    # single stream, 32 heads -> one 8-block cluster per head merges on chip, no scratch
+    assert rest.tree_attention_workspace_bytes(1, 32, 64, 128, 2112) == 0
+    # very few heads, long cache -> several clusters per head, fp32 partials of N*(D+2) floats
+    n = rest.tree_attention_workspace_bytes(1, 2, 64, 128, 8256)
+    assert n > 0 and n % (2 * 64 * 130 * 4) == 0
     assert rest.tree_attention_workspace_bytes(1, 32, 64, 64, 2112) == 0   # unsupported D
 
 
@@ -68,7 +70,8 @@ def test_host_argument_checks_return_status_codes():
     assert att(64, 64, 4, 4) == 2
     assert att(40, 128, 4, 4) == 2
     assert att(64, 128, 4, 3) == 2
-    assert att(64, 128, 32, 32) == 1       # needs a workspace, none given
+    assert L.rest_tree_attention(256, 256, 256, strides, 256, 256, 1, 2, 2, 64, 128, 8256, 1.0, 256,
+                                 None, None, 0, None) == 1       # needs a workspace, none given
     odd = (ctypes.c_int64 * 9)(*([124] * 9))
     assert att(64, 128, 4, 4, odd) == 1
     assert L.rest_accept(None, None, None, None, 1, 64, 10, None, None, None, None) == 1
