@@ -212,6 +212,15 @@ rest_status rest_accept(const int32_t* d_tokens, const int32_t* d_parents,
                         int32_t N, int32_t max_depth, int32_t* d_accept_len,
                         int32_t* d_accept_nodes, int32_t* d_out_tokens, void* stream);
 
+/*
+ * Device-side trouble that no per-call status can carry.  Every wait inside the kernels is
+ * bounded; a kernel that gives up sets a bit here instead of spinning, and its output is then
+ * undefined.  Reads and clears the flags of the current device (synchronises the device).
+ *   bit 0: tree attention gave up waiting for its tensor-core work
+ *   bit 1: tree attention found its shared-memory window misaligned and did nothing
+ */
+rest_status rest_device_error_flags(uint32_t* h_flags);
+
 const char* rest_status_string(rest_status s);
 /* Text of the last CUDA runtime error seen by this library on the calling thread. */
 const char* rest_last_cuda_error(void);

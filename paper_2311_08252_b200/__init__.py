@@ -29,6 +29,7 @@ EXPORTS = (
     "rest_draft_workspace_bytes", "rest_draft",
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
     "rest_tree_attention_static_scratch",
+    "rest_device_error_flags",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -81,6 +82,8 @@ def lib():
                                                      vp, vp]
     L.rest_accept.restype = i32
     L.rest_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    L.rest_device_error_flags.restype = i32
+    L.rest_device_error_flags.argtypes = [ctypes.POINTER(u32)]
     L.rest_status_string.restype = ctypes.c_char_p
     L.rest_status_string.argtypes = [i32]
     L.rest_last_cuda_error.restype = ctypes.c_char_p
@@ -114,6 +117,13 @@ def _dev_i32(t, name):
     if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
         raise RestError(f"{name} must be a contiguous int32 CUDA tensor")
     return t
+
+
+def device_error_flags() -> int:
+    """Reads and clears the device-side error bits (0 = no kernel ever gave up on a wait)."""
+    v = ctypes.c_uint32(0)
+    _check(lib().rest_device_error_flags(ctypes.byref(v)), "rest_device_error_flags")
+    return int(v.value)
 
 
 def launch_count() -> int:

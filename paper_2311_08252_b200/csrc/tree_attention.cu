@@ -18,6 +18,8 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "rest.h"
@@ -98,7 +100,7 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
 // Shared memory: Q tile [N][256 B] | K ring [stages][16 KB] | V ring [stages][16 KB] | mask [N][4]
 __global__ void __launch_bounds__(256)
 tree_attention_kernel(AttnArgs a) {
-  extern __shared__ __align__(128) unsigned char smem[];
+  extern __shared__ __align__(1024) unsigned char smem[];
   const int N = a.N;
   unsigned char* sQ = smem;
   unsigned char* sK = sQ + N * kRowBytes;
@@ -345,6 +347,439 @@ tree_attention_kernel(AttnArgs a) {
   cluster.sync();   // nobody leaves while a peer may still read its shared memory
 }
 
+// =======================================================================================
+// tcgen05 version: QK^T and PV on the 5th-generation tensor cores, accumulators in TMEM.
+//
+// One block = 4 warps.  Query rows are handled in blocks of 64 (NB = 1 for N <= 64, 2 for
+// N <= 128; rows past N are padding) because an M = 64 accumulator spreads its rows over all
+// four TMEM lane quadrants (16 rows each), so every warp - and every warp scheduler - gets an
+// equal share of the softmax.  The second row block lives in lanes 16..31 of each quadrant,
+// in the same TMEM columns.
+//
+// Q (NB x [64 x 128]), the K/V tiles ([64 x 128]) and P (NB x [64 x 64]) sit in shared memory
+// in the tensor core's canonical 128-byte-swizzled layout (8-row groups of 1024 B, the two
+// 64-element halves of the head dimension side by side), so a K tile is a K-major B operand
+// and the very same bytes of a V tile are an MN-major B operand: no transpose anywhere.
+// Per 64-key tile and row block:
+//   one thread issues 8 tcgen05.mma (M=64, N=64, K=16)   ->  S in TMEM columns [0, 64)
+//   each warp reads its 16 rows with the 16x256b pattern (same register layout as an
+//   mma.sync accumulator: a row is shared by a quad), applies scale / tree mask / base-2
+//   online softmax, and writes P (bf16) into shared memory
+//   one thread issues 4 tcgen05.mma (M=64, N=128, K=16)  ->  P V in TMEM columns [64, 192)
+//   each warp folds its rows of P V into fp32 register accumulators with the usual rescale.
+// Completion of each MMA group is signalled through an mbarrier (tcgen05.commit); waits are
+// bounded and report through g_attn_error instead of spinning forever.  Two blocks share an
+// SM (2 x 256 TMEM columns), so one block's softmax overlaps the other's MMAs and copies.
+// Split merge: same cluster / workspace scheme as above.
+// =======================================================================================
+constexpr int kTcThreads = 128;
+constexpr int kTcStages = 2;
+constexpr int kQBlockBytes = 64 * kRowBytes;            // 16 KB: 64 rows x 128 dims
+constexpr int kPBlockBytes = 64 * 128;                  //  8 KB: 64 rows x 64 keys
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kTmemColS = 0, kTmemColO = 64;
+constexpr long long kWaitCycles = 400000000ll;          // ~0.2 s: give up, flag, clean up
+
+__host__ __device__ constexpr int tc_bar_offset(int NB) { return NB * kQBlockBytes + 2 * kTcStages * kTileBytes + NB * kPBlockBytes; }
+__host__ __device__ constexpr int tc_smem_bytes(int NB) { return tc_bar_offset(NB) + 64; }
+
+__device__ unsigned int g_attn_error;                   // bit 0: wait gave up, bit 1: smem misaligned
+
+// shared-memory matrix descriptor: 128-byte swizzle, descriptor version 1
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major (0) or MN-major (1)
+__device__ __forceinline__ constexpr uint32_t umma_idesc(int M, int N, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                         uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// 16 TMEM lanes x 64 columns: r[4k..4k+3] = {row g: cols 8k+2t, 8k+2t+1; row g+8: same cols}
+__device__ __forceinline__ void tmem_ld_16x64(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Bounded wait on an mbarrier phase; false when the time limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  const long long start = clock64();
+  for (;;) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (clock64() - start > kWaitCycles) return false;
+  }
+}
+
+template <int NB>
+__global__ void __launch_bounds__(kTcThreads, 2)
+tree_attention_tc_kernel(AttnArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int N = a.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = lane >> 2, t4 = lane & 3;
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t sQ = sbase;
+  const uint32_t sK = sQ + NB * kQBlockBytes;
+  const uint32_t sV = sK + kTcStages * kTileBytes;
+  const uint32_t sP = sV + kTcStages * kTileBytes;
+  const uint32_t bar_s = sbase + tc_bar_offset(NB), bar_o = bar_s + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + tc_bar_offset(NB) + 16);
+
+  int bid = blockIdx.x;
+  const int split = bid % a.S; bid /= a.S;
+  const int h = bid % a.H;
+  const int b = bid / a.H;
+  const int hk = h / a.group;
+  const int L = a.kv_len[b];
+  const int total = L + N;
+  const int ntiles = (total + kBN - 1) / kBN;
+  const int t0 = (int)(((int64_t)split * ntiles) / a.S);
+  const int t1 = (int)(((int64_t)(split + 1) * ntiles) / a.S);
+  const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h;
+  const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
+  const __nv_bfloat16* vb = a.v + b * a.kv_b + hk * a.kv_h;
+
+  if ((sbase & 1023u) != 0) {   // the swizzled operand layout needs a 1024-byte aligned base
+    if (tid == 0) atomicOr(&g_attn_error, 2u);
+    return;                     // uniform over the grid: every block sees the same offset
+  }
+
+  // barriers + TMEM
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // Copy pattern: thread handles 16-byte chunk (tid & 15) of rows (tid >> 4) + 8 i.  In the
+  // operand layout a row's 8-row group is 1024 B apart and (row & 7) is fixed per thread, so
+  // source and destination both advance by a constant per step.
+  const int crow = tid >> 4, cchunk = tid & 15;
+  const uint32_t coff = (uint32_t)((cchunk >> 3) * (64 * 128) + crow * 128 + (((cchunk & 7) ^ crow) << 4));
+#pragma unroll
+  for (int i = 0; i < NB * 8; ++i) {     // Q rows crow + 8 i; rows >= N zero-filled
+    const int row = crow + 8 * i;
+    const bool ok = row < N;
+    cp_async16(sQ + (i >> 3) * kQBlockBytes + coff + (i & 7) * 1024,
+               qb + (int64_t)(ok ? row : 0) * a.q_n + cchunk * 8, ok);
+  }
+  auto load_tile = [&](int tile, int stage) {
+    const int key0 = tile * kBN + crow;
+    const uint32_t dK = sK + stage * kTileBytes + coff, dV = sV + stage * kTileBytes + coff;
+    const int64_t src0 = (int64_t)key0 * a.kv_l + cchunk * 8;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const bool ok = key0 + 8 * i < total;
+      const int64_t off = ok ? src0 + (int64_t)(8 * i) * a.kv_l : 0;
+      cp_async16(dK + i * 1024, kb + off, ok);
+      cp_async16(dV + i * 1024, vb + off, ok);
+    }
+  };
+  if (t0 < t1) load_tile(t0, 0);
+  cp_async_commit();
+
+  // rows of this thread: block rb, rows 16 warp + g and + 8
+  uint32_t mrow[NB][2][4];
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb)
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = rb * 64 + warp * 16 + g + 8 * hh;
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+        mrow[rb][hh][w] = (row < N && w < a.Wm) ? a.mask[((int64_t)b * N + row) * a.Wm + w] : 0u;
+    }
+  float o[NB][16][4];
+  float m_run[NB][2], l_run[NB][2];
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[rb][i][0] = o[rb][i][1] = o[rb][i][2] = o[rb][i][3] = 0.f; }
+    m_run[rb][0] = m_run[rb][1] = -INFINITY;
+    l_run[rb][0] = l_run[rb][1] = 0.f;
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_warp = tmem_base + ((uint32_t)(warp * 32) << 16);
+  constexpr uint32_t idesc_s = umma_idesc(64, kBN, 0);
+  constexpr uint32_t idesc_o = umma_idesc(64, kD, 1);
+  // descriptor bases; k-steps add (bytes >> 4) to the low word
+  const uint64_t dq0 = umma_desc(sQ, 16, 1024);
+  const uint64_t dk0 = umma_desc(sK, 16, 1024);
+  const uint64_t dp0 = umma_desc(sP, 16, 1024);
+  const uint64_t dv0 = umma_desc(sV, kBN * 128, 1024);
+
+  int timed_out = 0;
+  for (int t = t0; t < t1; ++t) {
+    const int it = t - t0, stage = it & 1;
+    const uint32_t phase = (uint32_t)(it & 1);
+    if (t + 1 < t1) load_tile(t + 1, stage ^ 1);   // that slot's MMAs were waited for at t - 1
+    cp_async_commit();
+    cp_async_wait<1>();                            // tile t (and Q) have landed
+    fence_async_smem();                            // make them visible to the tensor core
+    tc_fence_before();
+    if (__syncthreads_or(timed_out)) break;        // uniform exit if any thread gave up on a wait
+
+    if (tid == 0) {                                // S = Q K^T : 8 k-steps of 16 over the head dim
+      tc_fence_after();
+#pragma unroll
+      for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t koff = (uint32_t)((ks >> 2) * (64 * 128) + (ks & 3) * 32);
+          umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kTmemColS,
+                   dq0 + ((rb * kQBlockBytes + koff) >> 4),
+                   dk0 + ((stage * kTileBytes + koff) >> 4), idesc_s, ks > 0);
+        }
+      }
+      umma_commit(bar_s);
+    }
+    if (!mbar_wait(bar_s, phase)) timed_out = 1;
+    tc_fence_after();
+
+    const int key0 = t * kBN;
+    const bool need_mask = key0 + kBN > L;
+    float alpha[NB][2];
+#pragma unroll
+    for (int rb = 0; rb < NB; ++rb) {
+      uint32_t sr[32];
+      tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kTmemColS, sr);
+      tmem_wait_ld();
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v = __uint_as_float(sr[4 * k + e]) * a.scale_log2;
+          if (need_mask) {
+            const int key = key0 + k * 8 + t4 * 2 + (e & 1);
+            bool ok = key < L;
+            if (!ok && key < total) {
+              const int jj = key - L;
+              const int hh = e >> 1;
+              const uint32_t wsel = (jj >> 5) == 0 ? mrow[rb][hh][0] : (jj >> 5) == 1 ? mrow[rb][hh][1]
+                                    : (jj >> 5) == 2 ? mrow[rb][hh][2] : mrow[rb][hh][3];
+              ok = (wsel >> (jj & 31)) & 1u;
+            }
+            if (!ok) v = -INFINITY;
+          }
+          sr[4 * k + e] = __float_as_uint(v);
+        }
+        mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sr[4 * k]), __uint_as_float(sr[4 * k + 1])));
+        mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sr[4 * k + 2]), __uint_as_float(sr[4 * k + 3])));
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+      const float mn0 = fmaxf(m_run[rb][0], mx0), mn1 = fmaxf(m_run[rb][1], mx1);
+      const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+      alpha[rb][0] = ex2(m_run[rb][0] - ms0);      // m = -inf gives 0
+      alpha[rb][1] = ex2(m_run[rb][1] - ms1);
+      m_run[rb][0] = mn0; m_run[rb][1] = mn1;
+      float ps0 = 0.f, ps1 = 0.f;
+      // P (bf16) -> shared memory, K-major 128-byte-swizzled [64 rows x 64 keys]
+      const int rr0 = warp * 16 + g, rr1 = rr0 + 8;
+      const uint32_t p0 = sP + rb * kPBlockBytes + (rr0 >> 3) * 1024 + (rr0 & 7) * 128 + t4 * 4;
+      const uint32_t p1 = sP + rb * kPBlockBytes + (rr1 >> 3) * 1024 + (rr1 & 7) * 128 + t4 * 4;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float e0 = ex2(__uint_as_float(sr[4 * k]) - ms0), e1 = ex2(__uint_as_float(sr[4 * k + 1]) - ms0);
+        const float e2 = ex2(__uint_as_float(sr[4 * k + 2]) - ms1), e3 = ex2(__uint_as_float(sr[4 * k + 3]) - ms1);
+        ps0 += e0 + e1;
+        ps1 += e2 + e3;
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(p0 + ((k ^ (rr0 & 7)) << 4)), "r"(pack_bf16(e0, e1)) : "memory");
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(p1 + ((k ^ (rr1 & 7)) << 4)), "r"(pack_bf16(e2, e3)) : "memory");
+      }
+      l_run[rb][0] = l_run[rb][0] * alpha[rb][0] + ps0;
+      l_run[rb][1] = l_run[rb][1] * alpha[rb][1] + ps1;
+    }
+    fence_async_smem();
+    tc_fence_before();
+    if (__syncthreads_or(timed_out)) break;
+
+    if (tid == 0) {                                // O_t = P V : 4 k-steps of 16 keys
+      tc_fence_after();
+#pragma unroll
+      for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kTmemColO,
+                   dp0 + ((rb * kPBlockBytes + kk * 32) >> 4),
+                   dv0 + ((stage * kTileBytes + kk * 2048) >> 4), idesc_o, kk > 0);
+        }
+      }
+      umma_commit(bar_o);
+    }
+    if (!mbar_wait(bar_o, phase)) timed_out = 1;
+    tc_fence_after();
+
+#pragma unroll
+    for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {             // 64 output dims at a time
+        uint32_t orr[32];
+        tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kTmemColO + hf * 64, orr);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          float* oo = o[rb][hf * 8 + k];
+          oo[0] = oo[0] * alpha[rb][0] + __uint_as_float(orr[4 * k]);
+          oo[1] = oo[1] * alpha[rb][0] + __uint_as_float(orr[4 * k + 1]);
+          oo[2] = oo[2] * alpha[rb][1] + __uint_as_float(orr[4 * k + 2]);
+          oo[3] = oo[3] * alpha[rb][1] + __uint_as_float(orr[4 * k + 3]);
+        }
+      }
+    }
+    tc_fence_before();
+  }
+  cp_async_wait<0>();
+  tc_fence_before();
+  if (__syncthreads_or(timed_out) && tid == 0) atomicOr(&g_attn_error, 1u);
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
+                 : "memory");
+  }
+
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      l_run[rb][hh] += __shfl_xor_sync(0xFFFFFFFFu, l_run[rb][hh], 1);
+      l_run[rb][hh] += __shfl_xor_sync(0xFFFFFFFFu, l_run[rb][hh], 2);
+    }
+  }
+
+  if (a.S == 1) {
+#pragma unroll
+    for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int row = rb * 64 + warp * 16 + g + 8 * hh;
+        if (row >= N) continue;
+        const float l = l_run[rb][hh];
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)row * a.o_n + h * a.o_h;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          *reinterpret_cast<uint32_t*>(op + i * 8 + t4 * 2) =
+              pack_bf16(o[rb][i][2 * hh] * inv, o[rb][i][2 * hh + 1] * inv);
+        if (a.lse && t4 == 0)
+          a.lse[((int64_t)b * a.H + h) * N + row] = (m_run[rb][hh] + log2f(l)) * kLn2;
+      }
+    }
+    return;
+  }
+
+  // Park the partial (operand tiles are dead now) and merge across the cluster.
+  float* sO = reinterpret_cast<float*>(smem);
+  float* sML = sO + N * kOStride;
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = rb * 64 + warp * 16 + g + 8 * hh;
+      if (row >= N) continue;
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        *reinterpret_cast<float2*>(sO + row * kOStride + i * 8 + t4 * 2) =
+            make_float2(o[rb][i][2 * hh], o[rb][i][2 * hh + 1]);
+      if (t4 == 0) { sML[row * 2] = m_run[rb][hh]; sML[row * 2 + 1] = l_run[rb][hh]; }
+    }
+  }
+  cg::cluster_group cluster = cg::this_cluster();
+  cluster.sync();
+  const int C = a.C;
+  const int rank = (int)cluster.block_rank();
+  const int R = (N + C - 1) / C;
+  const int sup = split / C;
+  for (int idx = tid; idx < R * 32; idx += kTcThreads) {
+    const int mr = rank * R + (idx >> 5), c4 = idx & 31;
+    if (mr >= N) continue;
+    float2 ml[kMaxCluster];
+    float4 ov[kMaxCluster];
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p) {
+      if (p < C) {
+        ml[p] = *reinterpret_cast<const float2*>(cluster.map_shared_rank(sML, p) + mr * 2);
+        ov[p] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sO, p) + mr * kOStride + c4 * 4);
+      }
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p)
+      if (p < C) M = fmaxf(M, ml[p].x);
+    float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lsum = 0.f;
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p) {
+      if (p < C) {
+        const float w = (ml[p].x == -INFINITY) ? 0.f : exp2f(ml[p].x - M);
+        lsum += ml[p].y * w;
+        o4.x += ov[p].x * w; o4.y += ov[p].y * w; o4.z += ov[p].z * w; o4.w += ov[p].w * w;
+      }
+    }
+    if (a.Sp == 1) {
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      uint2 pk2;
+      pk2.x = pack_bf16(o4.x * inv, o4.y * inv);
+      pk2.y = pack_bf16(o4.z * inv, o4.w * inv);
+      *reinterpret_cast<uint2*>(a.out + b * a.o_b + (int64_t)mr * a.o_n + h * a.o_h + c4 * 4) = pk2;
+      if (a.lse && c4 == 0) a.lse[((int64_t)b * a.H + h) * N + mr] = (M + log2f(lsum)) * kLn2;
+    } else {
+      const int64_t base = ((((int64_t)b * a.H + h) * a.Sp + sup) * N + mr);
+      *reinterpret_cast<float4*>(a.ws_o + base * kD + c4 * 4) = o4;
+      if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
+    }
+  }
+  cluster.sync();
+}
+
 // Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
 __global__ void __launch_bounds__(128)
 tree_attention_combine_kernel(AttnArgs a) {
@@ -384,10 +819,20 @@ struct SplitPlan { int S, C, Sp; };
 
 // Key splits per (context, head): enough blocks to fill the GPU once (never a partial second
 // wave), at most one split per tile, rounded down to a whole number of clusters.
+// REST_ATTENTION_IMPL=mma_sync selects the older mma.sync kernel (kept for comparison runs);
+// anything else, or unset, runs the tcgen05 kernel.
+bool use_tcgen05() {
+  static const bool v = [] {
+    const char* e = getenv("REST_ATTENTION_IMPL");
+    return !(e && strcmp(e, "mma_sync") == 0);
+  }();
+  return v;
+}
+
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
   const int64_t units = (int64_t)B * H;
-  const int blocks_per_sm = N <= 64 ? 2 : 1;
+  const int blocks_per_sm = (use_tcgen05() || N <= 64) ? 2 : 1;
   int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
   if (S > ntiles) S = ntiles;
   SplitPlan p;
@@ -405,6 +850,15 @@ size_t attn_smem_bytes(int N) {
 }
 
 }  // namespace
+
+extern "C" rest_status rest_device_error_flags(uint32_t* h_flags) {
+  if (!h_flags) return REST_INVALID_ARG;
+  unsigned int v = 0, zero = 0;
+  REST_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_attn_error, sizeof(v)));
+  if (v != 0) REST_CUDA_TRY(cudaMemcpyToSymbol(g_attn_error, &zero, sizeof(zero)));
+  *h_flags = v;
+  return REST_OK;
+}
 
 extern "C" size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
                                                       int32_t max_kv) {
@@ -453,12 +907,21 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
     a.ws_ml = a.ws_o + (size_t)B * H * a.Sp * N * kD;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t smem = attn_smem_bytes(N);
-  REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_kernel),
-                                          2, smem));
+  const bool tc = use_tcgen05();
+  const bool two_blocks = N > 64;
+  const size_t smem = tc ? (size_t)tc_smem_bytes(two_blocks ? 2 : 1) : attn_smem_bytes(N);
+  if (tc && two_blocks)
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_tc_kernel<2>),
+                                            4, smem));
+  else if (tc)
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_tc_kernel<1>),
+                                            3, smem));
+  else
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_kernel),
+                                            2, smem));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(B * H * a.S), 1, 1);
-  cfg.blockDim = dim3((unsigned)((N / 16) * 32), 1, 1);
+  cfg.blockDim = dim3((unsigned)(tc ? kTcThreads : (N / 16) * 32), 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -468,7 +931,12 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_kernel, a));
+  if (tc && two_blocks)
+    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<2>, a));
+  else if (tc)
+    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<1>, a));
+  else
+    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_kernel, a));
   rest::count_launch();
   if (a.Sp > 1) {
     const int64_t units = (int64_t)B * H * N;
