@@ -367,21 +367,33 @@ tree_attention_kernel(AttnArgs a) {
 //   online softmax, and writes P (bf16) into shared memory
 //   one thread issues 4 tcgen05.mma (M=64, N=128, K=16)  ->  P V in TMEM columns [64, 192)
 //   each warp folds its rows of P V into fp32 register accumulators with the usual rescale.
+// The loop is software-pipelined: a fifth warp only issues MMAs, S is double-buffered in TMEM,
+// and Q K(t+1)^T runs on the tensor core while the four softmax warps work on tile t; P V of
+// tile t is folded into the register accumulators one iteration later, when it has long
+// finished.  K and V slots are refilled (16-byte cp.async, committed in a fixed group order)
+// as soon as the MMA that read them has completed.
 // Completion of each MMA group is signalled through an mbarrier (tcgen05.commit); waits are
-// bounded and report through g_attn_error instead of spinning forever.  Two blocks share an
-// SM (2 x 256 TMEM columns), so one block's softmax overlaps the other's MMAs and copies.
-// Split merge: same cluster / workspace scheme as above.
+// bounded and report through g_attn_error instead of spinning forever.  For N <= 64 two
+// blocks share an SM (2 x 256 TMEM columns).
+// Split merge: the splits of one (context, head) form a cluster; every block pushes its
+// partial rows into the shared memory of the block that owns those rows (posted stores, no
+// remote round trips), and after a cluster barrier each owner reduces locally.
 // =======================================================================================
-constexpr int kTcThreads = 128;
+constexpr int kTcThreads = 160;             // 4 softmax / copy warps + 1 MMA-issuing warp
 constexpr int kTcStages = 2;
 constexpr int kQBlockBytes = 64 * kRowBytes;            // 16 KB: 64 rows x 128 dims
 constexpr int kPBlockBytes = 64 * 128;                  //  8 KB: 64 rows x 64 keys
 constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kTmemColS = 0, kTmemColO = 64;
+constexpr uint32_t kColS = 0, kColO = 128;      // S double-buffered in [0,64) and [64,128); P V in [128,256)
 constexpr long long kWaitCycles = 400000000ll;          // ~0.2 s: give up, flag, clean up
 
 __host__ __device__ constexpr int tc_bar_offset(int NB) { return NB * kQBlockBytes + 2 * kTcStages * kTileBytes + NB * kPBlockBytes; }
 __host__ __device__ constexpr int tc_smem_bytes(int NB) { return tc_bar_offset(NB) + 64; }
+// Tiles are dealt so that the first splits take the spare ones: the last split, which holds
+// the masked tree tiles, never gets an extra tile.
+__host__ __device__ inline int tc_tile_begin(int split, int ntiles, int S) {
+  return (int)(((long long)split * ntiles + S - 1) / S);
+}
 
 __device__ unsigned int g_attn_error;                   // bit 0: wait gave up, bit 1: smem misaligned
 
@@ -447,19 +459,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 }
 
 template <int NB>
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, NB == 1 ? 2 : 1)
 tree_attention_tc_kernel(AttnArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   const int N = a.N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool is_mma_warp = warp == 4;          // warps 0..3: copies + softmax; warp 4: issues MMAs
   const int g = lane >> 2, t4 = lane & 3;
   const uint32_t sbase = smem_u32(smem);
   const uint32_t sQ = sbase;
   const uint32_t sK = sQ + NB * kQBlockBytes;
   const uint32_t sV = sK + kTcStages * kTileBytes;
   const uint32_t sP = sV + kTcStages * kTileBytes;
-  const uint32_t bar_s = sbase + tc_bar_offset(NB), bar_o = bar_s + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + tc_bar_offset(NB) + 16);
+  const uint32_t bar_s0 = sbase + tc_bar_offset(NB), bar_o = bar_s0 + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + tc_bar_offset(NB) + 24);
 
   int bid = blockIdx.x;
   const int split = bid % a.S; bid /= a.S;
@@ -469,8 +482,8 @@ tree_attention_tc_kernel(AttnArgs a) {
   const int L = a.kv_len[b];
   const int total = L + N;
   const int ntiles = (total + kBN - 1) / kBN;
-  const int t0 = (int)(((int64_t)split * ntiles) / a.S);
-  const int t1 = (int)(((int64_t)(split + 1) * ntiles) / a.S);
+  const int t0 = tc_tile_begin(split, ntiles, a.S);
+  const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
   const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h;
   const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
   const __nv_bfloat16* vb = a.v + b * a.kv_b + hk * a.kv_h;
@@ -482,7 +495,8 @@ tree_attention_tc_kernel(AttnArgs a) {
 
   // barriers + TMEM
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s0) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s0 + 8) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -493,59 +507,66 @@ tree_attention_tc_kernel(AttnArgs a) {
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
-  // Copy pattern: thread handles 16-byte chunk (tid & 15) of rows (tid >> 4) + 8 i.  In the
-  // operand layout a row's 8-row group is 1024 B apart and (row & 7) is fixed per thread, so
-  // source and destination both advance by a constant per step.
-  const int crow = tid >> 4, cchunk = tid & 15;
+  // Copy pattern (threads 0..127): thread handles 16-byte chunk (tid & 15) of rows
+  // (tid >> 4) + 8 i.  In the operand layout a row's 8-row group is 1024 B apart and
+  // (row & 7) is fixed per thread, so source and destination advance by constants.
+  const int crow = (tid >> 4) & 7, cchunk = tid & 15;
   const uint32_t coff = (uint32_t)((cchunk >> 3) * (64 * 128) + crow * 128 + (((cchunk & 7) ^ crow) << 4));
-#pragma unroll
-  for (int i = 0; i < NB * 8; ++i) {     // Q rows crow + 8 i; rows >= N zero-filled
-    const int row = crow + 8 * i;
-    const bool ok = row < N;
-    cp_async16(sQ + (i >> 3) * kQBlockBytes + coff + (i & 7) * 1024,
-               qb + (int64_t)(ok ? row : 0) * a.q_n + cchunk * 8, ok);
-  }
-  auto load_tile = [&](int tile, int stage) {
+  auto load_rows = [&](const __nv_bfloat16* base, uint32_t dst, int tile) {
     const int key0 = tile * kBN + crow;
-    const uint32_t dK = sK + stage * kTileBytes + coff, dV = sV + stage * kTileBytes + coff;
     const int64_t src0 = (int64_t)key0 * a.kv_l + cchunk * 8;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const bool ok = key0 + 8 * i < total;
-      const int64_t off = ok ? src0 + (int64_t)(8 * i) * a.kv_l : 0;
-      cp_async16(dK + i * 1024, kb + off, ok);
-      cp_async16(dV + i * 1024, vb + off, ok);
+      cp_async16(dst + coff + i * 1024, base + (ok ? src0 + (int64_t)(8 * i) * a.kv_l : 0), ok);
     }
   };
-  if (t0 < t1) load_tile(t0, 0);
-  cp_async_commit();
-
-  // rows of this thread: block rb, rows 16 warp + g and + 8
-  uint32_t mrow[NB][2][4];
+  // Copy groups are committed in a fixed order so that wait_group counts stay constant:
+  //   prologue: {Q, K(t0)}, {K(t0+1)}, {V(t0)};  iteration t: {K(t+2)}, {V(t+1)}.
+  if (!is_mma_warp) {
 #pragma unroll
-  for (int rb = 0; rb < NB; ++rb)
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int row = rb * 64 + warp * 16 + g + 8 * hh;
-#pragma unroll
-      for (int w = 0; w < 4; ++w)
-        mrow[rb][hh][w] = (row < N && w < a.Wm) ? a.mask[((int64_t)b * N + row) * a.Wm + w] : 0u;
+    for (int i = 0; i < NB * 8; ++i) {     // Q rows crow + 8 i; rows >= N zero-filled
+      const int row = crow + 8 * i;
+      const bool ok = row < N;
+      cp_async16(sQ + (i >> 3) * kQBlockBytes + coff + (i & 7) * 1024,
+                 qb + (int64_t)(ok ? row : 0) * a.q_n + cchunk * 8, ok);
     }
+    if (t0 < t1) load_rows(kb, sK, t0);
+    cp_async_commit();
+    if (t0 + 1 < t1) load_rows(kb, sK + kTileBytes, t0 + 1);
+    cp_async_commit();
+    if (t0 < t1) load_rows(vb, sV, t0);
+    cp_async_commit();
+  }
+
+  // rows of this thread: block rb, rows 16 (warp & 3) + g and + 8; mask row as two 64-bit halves
+  unsigned long long mlo[NB][2], mhi[NB][2];
   float o[NB][16][4];
-  float m_run[NB][2], l_run[NB][2];
+  float m_run[NB][2], l_run[NB][2], alpha[NB][2];
 #pragma unroll
   for (int rb = 0; rb < NB; ++rb) {
 #pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = rb * 64 + (warp & 3) * 16 + g + 8 * hh;
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (!is_mma_warp && row < N) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row) * a.Wm + i];
+      }
+      mlo[rb][hh] = (unsigned long long)w[0] | ((unsigned long long)w[1] << 32);
+      mhi[rb][hh] = (unsigned long long)w[2] | ((unsigned long long)w[3] << 32);
+      m_run[rb][hh] = -INFINITY; l_run[rb][hh] = 0.f; alpha[rb][hh] = 1.f;
+    }
+#pragma unroll
     for (int i = 0; i < 16; ++i) { o[rb][i][0] = o[rb][i][1] = o[rb][i][2] = o[rb][i][3] = 0.f; }
-    m_run[rb][0] = m_run[rb][1] = -INFINITY;
-    l_run[rb][0] = l_run[rb][1] = 0.f;
   }
 
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_warp = tmem_base + ((uint32_t)(warp * 32) << 16);
+  const uint32_t tmem_warp = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
   constexpr uint32_t idesc_s = umma_idesc(64, kBN, 0);
   constexpr uint32_t idesc_o = umma_idesc(64, kD, 1);
   // descriptor bases; k-steps add (bytes >> 4) to the low word
@@ -554,117 +575,27 @@ tree_attention_tc_kernel(AttnArgs a) {
   const uint64_t dp0 = umma_desc(sP, 16, 1024);
   const uint64_t dv0 = umma_desc(sV, kBN * 128, 1024);
 
-  int timed_out = 0;
-  for (int t = t0; t < t1; ++t) {
-    const int it = t - t0, stage = it & 1;
-    const uint32_t phase = (uint32_t)(it & 1);
-    if (t + 1 < t1) load_tile(t + 1, stage ^ 1);   // that slot's MMAs were waited for at t - 1
-    cp_async_commit();
-    cp_async_wait<1>();                            // tile t (and Q) have landed
-    fence_async_smem();                            // make them visible to the tensor core
-    tc_fence_before();
-    if (__syncthreads_or(timed_out)) break;        // uniform exit if any thread gave up on a wait
-
-    if (tid == 0) {                                // S = Q K^T : 8 k-steps of 16 over the head dim
-      tc_fence_after();
-#pragma unroll
-      for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t koff = (uint32_t)((ks >> 2) * (64 * 128) + (ks & 3) * 32);
-          umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kTmemColS,
-                   dq0 + ((rb * kQBlockBytes + koff) >> 4),
-                   dk0 + ((stage * kTileBytes + koff) >> 4), idesc_s, ks > 0);
-        }
-      }
-      umma_commit(bar_s);
-    }
-    if (!mbar_wait(bar_s, phase)) timed_out = 1;
-    tc_fence_after();
-
-    const int key0 = t * kBN;
-    const bool need_mask = key0 + kBN > L;
-    float alpha[NB][2];
-#pragma unroll
-    for (int rb = 0; rb < NB; ++rb) {
-      uint32_t sr[32];
-      tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kTmemColS, sr);
-      tmem_wait_ld();
-      float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float v = __uint_as_float(sr[4 * k + e]) * a.scale_log2;
-          if (need_mask) {
-            const int key = key0 + k * 8 + t4 * 2 + (e & 1);
-            bool ok = key < L;
-            if (!ok && key < total) {
-              const int jj = key - L;
-              const int hh = e >> 1;
-              const uint32_t wsel = (jj >> 5) == 0 ? mrow[rb][hh][0] : (jj >> 5) == 1 ? mrow[rb][hh][1]
-                                    : (jj >> 5) == 2 ? mrow[rb][hh][2] : mrow[rb][hh][3];
-              ok = (wsel >> (jj & 31)) & 1u;
-            }
-            if (!ok) v = -INFINITY;
-          }
-          sr[4 * k + e] = __float_as_uint(v);
-        }
-        mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sr[4 * k]), __uint_as_float(sr[4 * k + 1])));
-        mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sr[4 * k + 2]), __uint_as_float(sr[4 * k + 3])));
-      }
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
-      mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
-      mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
-      const float mn0 = fmaxf(m_run[rb][0], mx0), mn1 = fmaxf(m_run[rb][1], mx1);
-      const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-      alpha[rb][0] = ex2(m_run[rb][0] - ms0);      // m = -inf gives 0
-      alpha[rb][1] = ex2(m_run[rb][1] - ms1);
-      m_run[rb][0] = mn0; m_run[rb][1] = mn1;
-      float ps0 = 0.f, ps1 = 0.f;
-      // P (bf16) -> shared memory, K-major 128-byte-swizzled [64 rows x 64 keys]
-      const int rr0 = warp * 16 + g, rr1 = rr0 + 8;
-      const uint32_t p0 = sP + rb * kPBlockBytes + (rr0 >> 3) * 1024 + (rr0 & 7) * 128 + t4 * 4;
-      const uint32_t p1 = sP + rb * kPBlockBytes + (rr1 >> 3) * 1024 + (rr1 & 7) * 128 + t4 * 4;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const float e0 = ex2(__uint_as_float(sr[4 * k]) - ms0), e1 = ex2(__uint_as_float(sr[4 * k + 1]) - ms0);
-        const float e2 = ex2(__uint_as_float(sr[4 * k + 2]) - ms1), e3 = ex2(__uint_as_float(sr[4 * k + 3]) - ms1);
-        ps0 += e0 + e1;
-        ps1 += e2 + e3;
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(p0 + ((k ^ (rr0 & 7)) << 4)), "r"(pack_bf16(e0, e1)) : "memory");
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(p1 + ((k ^ (rr1 & 7)) << 4)), "r"(pack_bf16(e2, e3)) : "memory");
-      }
-      l_run[rb][0] = l_run[rb][0] * alpha[rb][0] + ps0;
-      l_run[rb][1] = l_run[rb][1] * alpha[rb][1] + ps1;
-    }
-    fence_async_smem();
-    tc_fence_before();
-    if (__syncthreads_or(timed_out)) break;
-
-    if (tid == 0) {                                // O_t = P V : 4 k-steps of 16 keys
-      tc_fence_after();
-#pragma unroll
-      for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kTmemColO,
-                   dp0 + ((rb * kPBlockBytes + kk * 32) >> 4),
-                   dv0 + ((stage * kTileBytes + kk * 2048) >> 4), idesc_o, kk > 0);
-        }
-      }
-      umma_commit(bar_o);
-    }
-    if (!mbar_wait(bar_o, phase)) timed_out = 1;
-    tc_fence_after();
-
+  auto issue_qk = [&](int it) {    // S[it & 1] = Q K(t)^T : 8 k-steps of 16 over the head dim
+    const int stage = it & 1;
 #pragma unroll
     for (int rb = 0; rb < NB; ++rb) {
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {             // 64 output dims at a time
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t koff = (uint32_t)((ks >> 2) * (64 * 128) + (ks & 3) * 32);
+        umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kColS + stage * 64,
+                 dq0 + ((rb * kQBlockBytes + koff) >> 4),
+                 dk0 + ((stage * kTileBytes + koff) >> 4), idesc_s, ks > 0);
+      }
+    }
+    umma_commit(bar_s0 + stage * 8);
+  };
+  auto fold_pv = [&]() {           // o = o * alpha + (P V of the previous tile)
+#pragma unroll
+    for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
         uint32_t orr[32];
-        tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kTmemColO + hf * 64, orr);
+        tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kColO + hf * 64, orr);
         tmem_wait_ld();
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -676,11 +607,156 @@ tree_attention_tc_kernel(AttnArgs a) {
         }
       }
     }
+  };
+
+  // pipeline prologue: S(t0) is in flight before the loop starts
+  int timed_out = 0;
+  if (t0 < t1) {
+    cp_async_wait<2>();
+    fence_async_smem();
     tc_fence_before();
+    __syncthreads();
+    if (is_mma_warp && lane == 0) { tc_fence_after(); issue_qk(0); }
+  }
+
+  for (int t = t0; t < t1; ++t) {
+    const int it = t - t0;
+    cp_async_wait<1>();                            // K(t+1) has landed
+    fence_async_smem();
+    tc_fence_before();
+    if (__syncthreads_or(timed_out)) break;        // uniform exit if any thread gave up on a wait
+    if (is_mma_warp) {
+      if (lane == 0 && t + 1 < t1) { tc_fence_after(); issue_qk(it + 1); }   // overlaps softmax(t)
+    } else {
+      if (!mbar_wait(bar_s0 + (it & 1) * 8, (uint32_t)((it >> 1) & 1))) timed_out = 1;
+      tc_fence_after();
+      const int key0 = t * kBN;
+      const bool need_mask = key0 + kBN > L;
+      uint32_t pk[NB][16];
+      float alpha_new[NB][2];
+#pragma unroll
+      for (int rb = 0; rb < NB; ++rb) {
+        uint32_t sr[32];
+        tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kColS + (it & 1) * 64, sr);
+        tmem_wait_ld();
+        if (rb == NB - 1) {                        // K(t) is dead (its MMAs completed): refill the slot
+          if (t + 2 < t1) load_rows(kb, sK + (it & 1) * kTileBytes, t + 2);
+          cp_async_commit();
+        }
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+        if (!need_mask) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float v0 = __uint_as_float(sr[4 * k]) * a.scale_log2, v1 = __uint_as_float(sr[4 * k + 1]) * a.scale_log2;
+            const float v2 = __uint_as_float(sr[4 * k + 2]) * a.scale_log2, v3 = __uint_as_float(sr[4 * k + 3]) * a.scale_log2;
+            sr[4 * k] = __float_as_uint(v0); sr[4 * k + 1] = __float_as_uint(v1);
+            sr[4 * k + 2] = __float_as_uint(v2); sr[4 * k + 3] = __float_as_uint(v3);
+            mx0 = fmaxf(mx0, fmaxf(v0, v1));
+            mx1 = fmaxf(mx1, fmaxf(v2, v3));
+          }
+        } else {
+          // 64-bit "key j of this tile is visible" masks of the thread's two rows: prefix keys,
+          // then the row's tree bits moved to where key L sits in this tile
+          unsigned long long am[2];
+          const int off = L - key0;                // position of key L in this tile (may be < 0)
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            unsigned long long pre = off >= 64 ? ~0ull : (off <= 0 ? 0ull : ((1ull << off) - 1ull));
+            unsigned long long tb;
+            if (off >= 64) tb = 0ull;
+            else if (off >= 0) tb = mlo[rb][hh] << off;
+            else if (off > -64) tb = (mlo[rb][hh] >> (-off)) | (mhi[rb][hh] << (64 + off));
+            else if (off > -128) tb = mhi[rb][hh] >> (-off - 64);
+            else tb = 0ull;
+            am[hh] = (pre | tb) >> (2 * t4);
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const bool ok = (am[e >> 1] >> (8 * k + (e & 1))) & 1ull;
+              const float v = ok ? __uint_as_float(sr[4 * k + e]) * a.scale_log2 : -INFINITY;
+              sr[4 * k + e] = __float_as_uint(v);
+            }
+            mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sr[4 * k]), __uint_as_float(sr[4 * k + 1])));
+            mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sr[4 * k + 2]), __uint_as_float(sr[4 * k + 3])));
+          }
+        }
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+        const float mn0 = fmaxf(m_run[rb][0], mx0), mn1 = fmaxf(m_run[rb][1], mx1);
+        const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+        alpha_new[rb][0] = ex2(m_run[rb][0] - ms0);  // m = -inf gives 0
+        alpha_new[rb][1] = ex2(m_run[rb][1] - ms1);
+        m_run[rb][0] = mn0; m_run[rb][1] = mn1;
+        float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float e0 = ex2(__uint_as_float(sr[4 * k]) - ms0), e1 = ex2(__uint_as_float(sr[4 * k + 1]) - ms0);
+          const float e2 = ex2(__uint_as_float(sr[4 * k + 2]) - ms1), e3 = ex2(__uint_as_float(sr[4 * k + 3]) - ms1);
+          ps0 += e0 + e1;
+          ps1 += e2 + e3;
+          pk[rb][2 * k] = pack_bf16(e0, e1);
+          pk[rb][2 * k + 1] = pack_bf16(e2, e3);
+        }
+        l_run[rb][0] = l_run[rb][0] * alpha_new[rb][0] + ps0;
+        l_run[rb][1] = l_run[rb][1] * alpha_new[rb][1] + ps1;
+      }
+      // P V of the previous tile finished a while ago: fold it in (with the previous rescale),
+      // which also frees the P buffer, the O columns and the previous V slot.
+      if (it > 0) {
+        if (!mbar_wait(bar_o, (uint32_t)((it - 1) & 1))) timed_out = 1;
+        tc_fence_after();
+        fold_pv();
+      }
+      if (t + 1 < t1) load_rows(vb, sV + ((it + 1) & 1) * kTileBytes, t + 1);
+      cp_async_commit();
+#pragma unroll
+      for (int rb = 0; rb < NB; ++rb) {
+        alpha[rb][0] = alpha_new[rb][0]; alpha[rb][1] = alpha_new[rb][1];
+        // P (bf16) -> shared memory, K-major 128-byte-swizzled [64 rows x 64 keys]
+        const int rr0 = warp * 16 + g, rr1 = rr0 + 8;
+        const uint32_t p0 = sP + rb * kPBlockBytes + (rr0 >> 3) * 1024 + (rr0 & 7) * 128 + t4 * 4;
+        const uint32_t p1 = sP + rb * kPBlockBytes + (rr1 >> 3) * 1024 + (rr1 & 7) * 128 + t4 * 4;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(p0 + ((k ^ (rr0 & 7)) << 4)), "r"(pk[rb][2 * k]) : "memory");
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(p1 + ((k ^ (rr1 & 7)) << 4)), "r"(pk[rb][2 * k + 1]) : "memory");
+        }
+      }
+      cp_async_wait<2>();                          // V(t) has landed
+      fence_async_smem();
+      tc_fence_before();
+    }
+    if (__syncthreads_or(timed_out)) break;
+    if (is_mma_warp && lane == 0) {                // O = P V : 4 k-steps of 16 keys
+      tc_fence_after();
+      const int stage = it & 1;
+#pragma unroll
+      for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kColO,
+                   dp0 + ((rb * kPBlockBytes + kk * 32) >> 4),
+                   dv0 + ((stage * kTileBytes + kk * 2048) >> 4), idesc_o, kk > 0);
+        }
+      }
+      umma_commit(bar_o);
+    }
+  }
+  if (!is_mma_warp && t0 < t1 && !timed_out) {     // the last tile's P V
+    if (!mbar_wait(bar_o, (uint32_t)((t1 - t0 - 1) & 1))) timed_out = 1;
+    tc_fence_after();
+    fold_pv();
   }
   cp_async_wait<0>();
   tc_fence_before();
   if (__syncthreads_or(timed_out) && tid == 0) atomicOr(&g_attn_error, 1u);
+  // This block no longer touches its operand tiles: tell the cluster (peers will write their
+  // partial rows into this block's shared memory once every block has said so).
+  if (a.S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
                  : "memory");
@@ -701,7 +777,7 @@ tree_attention_tc_kernel(AttnArgs a) {
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
         const int row = rb * 64 + warp * 16 + g + 8 * hh;
-        if (row >= N) continue;
+        if (is_mma_warp || row >= N) continue;
         const float l = l_run[rb][hh];
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)row * a.o_n + h * a.o_h;
@@ -716,38 +792,47 @@ tree_attention_tc_kernel(AttnArgs a) {
     return;
   }
 
-  // Park the partial (operand tiles are dead now) and merge across the cluster.
-  float* sO = reinterpret_cast<float*>(smem);
-  float* sML = sO + N * kOStride;
+  // Merge across the cluster by pushing: rows [r*R, r*R + R) belong to block r.  Every block
+  // stores its partial rows (fp32 O, max, sum) into the owner's shared memory, slot = its own
+  // rank; stores are posted, so nobody waits on a remote round trip.  After the second
+  // cluster barrier each owner reduces its C slots locally and writes the output.
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = a.C;
+  const int rank = (int)cluster.block_rank();
+  const int R = (N + C - 1) / C;
+  float* sO = reinterpret_cast<float*>(smem);          // [C][R][kOStride]
+  float* sML = sO + C * R * kOStride;                   // [C][R][2]
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every block's tiles are dead
 #pragma unroll
   for (int rb = 0; rb < NB; ++rb) {
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       const int row = rb * 64 + warp * 16 + g + 8 * hh;
-      if (row >= N) continue;
+      if (is_mma_warp || row >= N) continue;
+      const int owner = row / R, slot = rank * R + (row - owner * R);
+      float* ro = cluster.map_shared_rank(sO, owner) + slot * kOStride;
 #pragma unroll
       for (int i = 0; i < 16; ++i)
-        *reinterpret_cast<float2*>(sO + row * kOStride + i * 8 + t4 * 2) =
-            make_float2(o[rb][i][2 * hh], o[rb][i][2 * hh + 1]);
-      if (t4 == 0) { sML[row * 2] = m_run[rb][hh]; sML[row * 2 + 1] = l_run[rb][hh]; }
+        *reinterpret_cast<float2*>(ro + i * 8 + t4 * 2) = make_float2(o[rb][i][2 * hh], o[rb][i][2 * hh + 1]);
+      if (t4 == 0)
+        *reinterpret_cast<float2*>(cluster.map_shared_rank(sML, owner) + slot * 2) =
+            make_float2(m_run[rb][hh], l_run[rb][hh]);
     }
   }
-  cg::cluster_group cluster = cg::this_cluster();
-  cluster.sync();
-  const int C = a.C;
-  const int rank = (int)cluster.block_rank();
-  const int R = (N + C - 1) / C;
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+
   const int sup = split / C;
   for (int idx = tid; idx < R * 32; idx += kTcThreads) {
-    const int mr = rank * R + (idx >> 5), c4 = idx & 31;
+    const int lr = idx >> 5, mr = rank * R + lr, c4 = idx & 31;
     if (mr >= N) continue;
     float2 ml[kMaxCluster];
     float4 ov[kMaxCluster];
 #pragma unroll
     for (int p = 0; p < kMaxCluster; ++p) {
       if (p < C) {
-        ml[p] = *reinterpret_cast<const float2*>(cluster.map_shared_rank(sML, p) + mr * 2);
-        ov[p] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sO, p) + mr * kOStride + c4 * 4);
+        ml[p] = *reinterpret_cast<const float2*>(sML + (p * R + lr) * 2);
+        ov[p] = *reinterpret_cast<const float4*>(sO + (p * R + lr) * kOStride + c4 * 4);
       }
     }
     float M = -INFINITY;
@@ -759,7 +844,7 @@ tree_attention_tc_kernel(AttnArgs a) {
 #pragma unroll
     for (int p = 0; p < kMaxCluster; ++p) {
       if (p < C) {
-        const float w = (ml[p].x == -INFINITY) ? 0.f : exp2f(ml[p].x - M);
+        const float w = (ml[p].x == -INFINITY) ? 0.f : ex2(ml[p].x - M);
         lsum += ml[p].y * w;
         o4.x += ov[p].x * w; o4.y += ov[p].y * w; o4.z += ov[p].z * w; o4.w += ov[p].w * w;
       }
@@ -777,7 +862,6 @@ tree_attention_tc_kernel(AttnArgs a) {
       if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
     }
   }
-  cluster.sync();
 }
 
 // Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
@@ -832,7 +916,7 @@ bool use_tcgen05() {
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
   const int64_t units = (int64_t)B * H;
-  const int blocks_per_sm = (use_tcgen05() || N <= 64) ? 2 : 1;
+  const int blocks_per_sm = N <= 64 ? 2 : 1;
   int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
   if (S > ntiles) S = ntiles;
   SplitPlan p;
