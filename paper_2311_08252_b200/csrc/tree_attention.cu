@@ -387,7 +387,14 @@ constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;      // S double-buffered in [0,64) and [64,128); P V in [128,256)
 constexpr long long kWaitCycles = 400000000ll;          // ~0.2 s: give up, flag, clean up
 
-__host__ __device__ constexpr int tc_bar_offset(int NB) { return NB * kQBlockBytes + 2 * kTcStages * kTileBytes + NB * kPBlockBytes; }
+// Shared memory of the tcgen05 kernel: operand tiles (Q blocks, K ring, V ring, P blocks), later
+// reused by the split merge, which stages 64 NB partial rows and receives up to 64 NB + 8 rows
+// of kOStride floats; the mbarriers and the TMEM slot sit behind whichever is larger.
+__host__ __device__ constexpr int tc_operand_bytes(int NB) { return NB * kQBlockBytes + 2 * kTcStages * kTileBytes + NB * kPBlockBytes; }
+__host__ __device__ constexpr int tc_merge_bytes(int NB) { return (2 * 64 * NB + 8) * kOStride * 4; }
+__host__ __device__ constexpr int tc_bar_offset(int NB) {
+  return tc_operand_bytes(NB) > tc_merge_bytes(NB) ? tc_operand_bytes(NB) : tc_merge_bytes(NB);
+}
 __host__ __device__ constexpr int tc_smem_bytes(int NB) { return tc_bar_offset(NB) + 64; }
 // Tiles are dealt so that the first splits take the spare ones: the last split, which holds
 // the masked tree tiles, never gets an extra tile.
@@ -471,7 +478,7 @@ tree_attention_tc_kernel(AttnArgs a) {
   const uint32_t sK = sQ + NB * kQBlockBytes;
   const uint32_t sV = sK + kTcStages * kTileBytes;
   const uint32_t sP = sV + kTcStages * kTileBytes;
-  const uint32_t bar_s0 = sbase + tc_bar_offset(NB), bar_o = bar_s0 + 16;
+  const uint32_t bar_s0 = sbase + tc_bar_offset(NB), bar_o = bar_s0 + 16, bar_m = bar_s0 + 32;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + tc_bar_offset(NB) + 24);
 
   int bid = blockIdx.x;
@@ -498,7 +505,15 @@ tree_attention_tc_kernel(AttnArgs a) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s0) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s0 + 8) : "memory");
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_m) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (a.S > 1) {   // merge: this block will receive its rows of every peer's partial
+      const int Rm = (N + a.C - 1) / a.C;
+      const int mine = max(0, min(Rm, N - (split % a.C) * Rm));
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_m),
+                   "r"((uint32_t)(a.C * mine * kOStride * 4))
+                   : "memory");
+    }
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -754,9 +769,6 @@ tree_attention_tc_kernel(AttnArgs a) {
   cp_async_wait<0>();
   tc_fence_before();
   if (__syncthreads_or(timed_out) && tid == 0) atomicOr(&g_attn_error, 1u);
-  // This block no longer touches its operand tiles: tell the cluster (peers will write their
-  // partial rows into this block's shared memory once every block has said so).
-  if (a.S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
                  : "memory");
@@ -792,47 +804,62 @@ tree_attention_tc_kernel(AttnArgs a) {
     return;
   }
 
-  // Merge across the cluster by pushing: rows [r*R, r*R + R) belong to block r.  Every block
-  // stores its partial rows (fp32 O, max, sum) into the owner's shared memory, slot = its own
-  // rank; stores are posted, so nobody waits on a remote round trip.  After the second
-  // cluster barrier each owner reduces its C slots locally and writes the output.
-  cg::cluster_group cluster = cg::this_cluster();
+  // Merge across the cluster by pushing.  Rows [r*R, r*R + R) belong to block r.  A partial
+  // row is 132 floats: 128 of O, then (max, sum).  Each block stages its rows in its own
+  // shared memory and, once every block of the cluster is done with its operand tiles, sends
+  // each owner its rows with ONE bulk shared-to-shared copy that signals the owner's mbarrier
+  // (armed at start-up with the byte count it will receive).  Nobody waits on a remote round
+  // trip; the owner reduces its C slots locally as soon as its mbarrier completes.
   const int C = a.C;
-  const int rank = (int)cluster.block_rank();
+  const int rank = split % C;
   const int R = (N + C - 1) / C;
-  float* sO = reinterpret_cast<float*>(smem);          // [C][R][kOStride]
-  float* sML = sO + C * R * kOStride;                   // [C][R][2]
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every block's tiles are dead
+  float* sStage = reinterpret_cast<float*>(smem);                    // [N][kOStride]
+  float* sRecv = sStage + (size_t)N * kOStride;                      // [C][R][kOStride]
 #pragma unroll
   for (int rb = 0; rb < NB; ++rb) {
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       const int row = rb * 64 + warp * 16 + g + 8 * hh;
       if (is_mma_warp || row >= N) continue;
-      const int owner = row / R, slot = rank * R + (row - owner * R);
-      float* ro = cluster.map_shared_rank(sO, owner) + slot * kOStride;
+      float* ro = sStage + row * kOStride;
 #pragma unroll
       for (int i = 0; i < 16; ++i)
         *reinterpret_cast<float2*>(ro + i * 8 + t4 * 2) = make_float2(o[rb][i][2 * hh], o[rb][i][2 * hh + 1]);
-      if (t4 == 0)
-        *reinterpret_cast<float2*>(cluster.map_shared_rank(sML, owner) + slot * 2) =
-            make_float2(m_run[rb][hh], l_run[rb][hh]);
+      if (t4 == 0) *reinterpret_cast<float2*>(ro + kD) = make_float2(m_run[rb][hh], l_run[rb][hh]);
     }
   }
+  fence_async_smem();                          // staged rows -> visible to the bulk-copy engine
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every block's tiles are dead
+  if (tid < C) {
+    const int owner = tid;
+    const int rows = max(0, min(R, N - owner * R));
+    if (rows > 0) {
+      const uint32_t src = smem_u32(sStage + (size_t)owner * R * kOStride);
+      const uint32_t dst_local = smem_u32(sRecv + (size_t)rank * R * kOStride);
+      uint32_t dst, rbar;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(dst_local), "r"(owner));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(bar_m), "r"(owner));
+      asm volatile(
+          "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+          ::"r"(dst), "r"(src), "r"((uint32_t)(rows * kOStride * 4)), "r"(rbar)
+          : "memory");
+    }
+  }
+  int merge_timeout = mbar_wait(bar_m, 0u) ? 0 : 1;
 
   const int sup = split / C;
-  for (int idx = tid; idx < R * 32; idx += kTcThreads) {
+  const int my_rows = max(0, min(R, N - rank * R));
+  for (int idx = tid; idx < my_rows * 32; idx += kTcThreads) {
     const int lr = idx >> 5, mr = rank * R + lr, c4 = idx & 31;
-    if (mr >= N) continue;
     float2 ml[kMaxCluster];
     float4 ov[kMaxCluster];
 #pragma unroll
     for (int p = 0; p < kMaxCluster; ++p) {
       if (p < C) {
-        ml[p] = *reinterpret_cast<const float2*>(sML + (p * R + lr) * 2);
-        ov[p] = *reinterpret_cast<const float4*>(sO + (p * R + lr) * kOStride + c4 * 4);
+        const float* rr = sRecv + (size_t)(p * R + lr) * kOStride;
+        ml[p] = *reinterpret_cast<const float2*>(rr + kD);
+        ov[p] = *reinterpret_cast<const float4*>(rr + c4 * 4);
       }
     }
     float M = -INFINITY;
@@ -862,6 +889,10 @@ tree_attention_tc_kernel(AttnArgs a) {
       if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
     }
   }
+  if (merge_timeout && tid == 0) atomicOr(&g_attn_error, 1u);
+  // stay until every peer has received what this block sent (its staged rows are the source)
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
