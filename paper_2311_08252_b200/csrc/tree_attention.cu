@@ -50,6 +50,7 @@ struct AttnArgs {
   int64_t q_b, q_n, q_h, kv_b, kv_h, kv_l, o_b, o_n, o_h;
   int B, H, group, N, Wm;
   int S;            // key splits per (context, head) = C * Sp
+  int NBLK;         // 64-row query blocks per (context, head): each gets its own thread blocks
   int C;            // blocks per cluster
   int Sp;           // clusters per (context, head); > 1 needs the merge kernel
   float scale_log2;
@@ -350,11 +351,14 @@ tree_attention_kernel(AttnArgs a) {
 // =======================================================================================
 // tcgen05 version: QK^T and PV on the 5th-generation tensor cores, accumulators in TMEM.
 //
-// One block = 4 warps.  Query rows are handled in blocks of 64 (NB = 1 for N <= 64, 2 for
-// N <= 128; rows past N are padding) because an M = 64 accumulator spreads its rows over all
-// four TMEM lane quadrants (16 rows each), so every warp - and every warp scheduler - gets an
-// equal share of the softmax.  The second row block lives in lanes 16..31 of each quadrant,
-// in the same TMEM columns.
+// One block = 4 softmax warps + 1 MMA-issuing warp.  Query rows are handled in blocks of 64:
+// every 64-row block of the N draft rows gets its own thread blocks (grid index: row block
+// fastest after the split, so the blocks of one (context, head) stream the same K/V tiles at
+// the same time and the second reader hits L2).  M = 64 rather than 128 because an M = 64
+// accumulator spreads its rows over all four TMEM lane quadrants (16 rows each), so every
+// warp - and every warp scheduler - gets an equal share of the softmax.  (The kernel is
+// written for NB row blocks per thread block, the second one in lanes 16..31 of each
+// quadrant; it is instantiated with NB = 1, which keeps two blocks resident per SM.)
 //
 // Q (NB x [64 x 128]), the K/V tiles ([64 x 128]) and P (NB x [64 x 64]) sit in shared memory
 // in the tensor core's canonical 128-byte-swizzled layout (8-row groups of 1024 B, the two
@@ -483,6 +487,7 @@ tree_attention_tc_kernel(AttnArgs a) {
 
   int bid = blockIdx.x;
   const int split = bid % a.S; bid /= a.S;
+  const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 64-row block of the N draft rows
   const int h = bid % a.H;
   const int b = bid / a.H;
   const int hk = h / a.group;
@@ -491,7 +496,9 @@ tree_attention_tc_kernel(AttnArgs a) {
   const int ntiles = (total + kBN - 1) / kBN;
   const int t0 = tc_tile_begin(split, ntiles, a.S);
   const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
-  const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h;
+  const int row0 = rblk * (64 * NB);                 // first draft row of this thread block
+  const int Nl = min(64 * NB, N - row0);             // its number of real rows
+  const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h + (int64_t)row0 * a.q_n;
   const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
   const __nv_bfloat16* vb = a.v + b * a.kv_b + hk * a.kv_h;
 
@@ -508,8 +515,8 @@ tree_attention_tc_kernel(AttnArgs a) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_m) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (a.S > 1) {   // merge: this block will receive its rows of every peer's partial
-      const int Rm = (N + a.C - 1) / a.C;
-      const int mine = max(0, min(Rm, N - (split % a.C) * Rm));
+      const int Rm = (Nl + a.C - 1) / a.C;
+      const int mine = max(0, min(Rm, Nl - (split % a.C) * Rm));
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_m),
                    "r"((uint32_t)(a.C * mine * kOStride * 4))
                    : "memory");
@@ -542,7 +549,7 @@ tree_attention_tc_kernel(AttnArgs a) {
 #pragma unroll
     for (int i = 0; i < NB * 8; ++i) {     // Q rows crow + 8 i; rows >= N zero-filled
       const int row = crow + 8 * i;
-      const bool ok = row < N;
+      const bool ok = row < Nl;
       cp_async16(sQ + (i >> 3) * kQBlockBytes + coff + (i & 7) * 1024,
                  qb + (int64_t)(ok ? row : 0) * a.q_n + cchunk * 8, ok);
     }
@@ -564,10 +571,10 @@ tree_attention_tc_kernel(AttnArgs a) {
     for (int hh = 0; hh < 2; ++hh) {
       const int row = rb * 64 + (warp & 3) * 16 + g + 8 * hh;
       uint32_t w[4] = {0u, 0u, 0u, 0u};
-      if (!is_mma_warp && row < N) {
+      if (!is_mma_warp && row < Nl) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row) * a.Wm + i];
+          if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row0 + row) * a.Wm + i];
       }
       mlo[rb][hh] = (unsigned long long)w[0] | ((unsigned long long)w[1] << 32);
       mhi[rb][hh] = (unsigned long long)w[2] | ((unsigned long long)w[3] << 32);
@@ -789,16 +796,16 @@ tree_attention_tc_kernel(AttnArgs a) {
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
         const int row = rb * 64 + warp * 16 + g + 8 * hh;
-        if (is_mma_warp || row >= N) continue;
+        if (is_mma_warp || row >= Nl) continue;
         const float l = l_run[rb][hh];
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)row * a.o_n + h * a.o_h;
+        __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)(row0 + row) * a.o_n + h * a.o_h;
 #pragma unroll
         for (int i = 0; i < 16; ++i)
           *reinterpret_cast<uint32_t*>(op + i * 8 + t4 * 2) =
               pack_bf16(o[rb][i][2 * hh] * inv, o[rb][i][2 * hh + 1] * inv);
         if (a.lse && t4 == 0)
-          a.lse[((int64_t)b * a.H + h) * N + row] = (m_run[rb][hh] + log2f(l)) * kLn2;
+          a.lse[((int64_t)b * a.H + h) * N + row0 + row] = (m_run[rb][hh] + log2f(l)) * kLn2;
       }
     }
     return;
@@ -812,15 +819,15 @@ tree_attention_tc_kernel(AttnArgs a) {
   // trip; the owner reduces its C slots locally as soon as its mbarrier completes.
   const int C = a.C;
   const int rank = split % C;
-  const int R = (N + C - 1) / C;
-  float* sStage = reinterpret_cast<float*>(smem);                    // [N][kOStride]
-  float* sRecv = sStage + (size_t)N * kOStride;                      // [C][R][kOStride]
+  const int R = (Nl + C - 1) / C;
+  float* sStage = reinterpret_cast<float*>(smem);                    // [Nl][kOStride]
+  float* sRecv = sStage + (size_t)Nl * kOStride;                     // [C][R][kOStride]
 #pragma unroll
   for (int rb = 0; rb < NB; ++rb) {
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       const int row = rb * 64 + warp * 16 + g + 8 * hh;
-      if (is_mma_warp || row >= N) continue;
+      if (is_mma_warp || row >= Nl) continue;
       float* ro = sStage + row * kOStride;
 #pragma unroll
       for (int i = 0; i < 16; ++i)
@@ -833,7 +840,7 @@ tree_attention_tc_kernel(AttnArgs a) {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every block's tiles are dead
   if (tid < C) {
     const int owner = tid;
-    const int rows = max(0, min(R, N - owner * R));
+    const int rows = max(0, min(R, Nl - owner * R));
     if (rows > 0) {
       const uint32_t src = smem_u32(sStage + (size_t)owner * R * kOStride);
       const uint32_t dst_local = smem_u32(sRecv + (size_t)rank * R * kOStride);
@@ -849,9 +856,9 @@ tree_attention_tc_kernel(AttnArgs a) {
   int merge_timeout = mbar_wait(bar_m, 0u) ? 0 : 1;
 
   const int sup = split / C;
-  const int my_rows = max(0, min(R, N - rank * R));
+  const int my_rows = max(0, min(R, Nl - rank * R));
   for (int idx = tid; idx < my_rows * 32; idx += kTcThreads) {
-    const int lr = idx >> 5, mr = rank * R + lr, c4 = idx & 31;
+    const int lr = idx >> 5, mr = row0 + rank * R + lr, c4 = idx & 31;   // mr: global draft row
     float2 ml[kMaxCluster];
     float4 ov[kMaxCluster];
 #pragma unroll
@@ -946,8 +953,9 @@ bool use_tcgen05() {
 
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
-  const int64_t units = (int64_t)B * H;
-  const int blocks_per_sm = N <= 64 ? 2 : 1;
+  // the tcgen05 kernel gives every 64-row block of the draft rows its own thread blocks
+  const int64_t units = (int64_t)B * H * (use_tcgen05() ? (N + 63) / 64 : 1);
+  const int blocks_per_sm = (use_tcgen05() || N <= 64) ? 2 : 1;
   int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
   if (S > ntiles) S = ntiles;
   SplitPlan p;
@@ -1023,19 +1031,17 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool tc = use_tcgen05();
-  const bool two_blocks = N > 64;
-  const size_t smem = tc ? (size_t)tc_smem_bytes(two_blocks ? 2 : 1) : attn_smem_bytes(N);
-  if (tc && two_blocks)
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_tc_kernel<2>),
-                                            4, smem));
-  else if (tc)
+  a.NBLK = tc ? (N + 63) / 64 : 1;
+  const size_t smem = tc ? (size_t)tc_smem_bytes(1) : attn_smem_bytes(N);
+  if (tc)
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_tc_kernel<1>),
                                             3, smem));
   else
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_kernel),
                                             2, smem));
+  if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(B * H * a.S), 1, 1);
+  cfg.gridDim = dim3((unsigned)(B * H * a.NBLK * a.S), 1, 1);
   cfg.blockDim = dim3((unsigned)(tc ? kTcThreads : (N / 16) * 32), 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
@@ -1046,9 +1052,7 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (tc && two_blocks)
-    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<2>, a));
-  else if (tc)
+  if (tc)
     REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<1>, a));
   else
     REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_kernel, a));
