@@ -14,6 +14,7 @@
 // shared memory) and writes bf16 output.  Only when more than 8 splits are needed do the
 // cluster-merged partials go to the caller's workspace for a second, small merge kernel.
 #include <cooperative_groups.h>
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -51,6 +52,7 @@ struct AttnArgs {
   int B, H, group, N, Wm;
   int S;            // key splits per (context, head) = C * Sp
   int NBLK;         // 64-row query blocks per (context, head): each gets its own thread blocks
+  int q_slot[3], kv_slot[3];   // tensor-map coordinate index (1..3) of rows, head, batch
   int C;            // blocks per cluster
   int Sp;           // clusters per (context, head); > 1 needs the merge kernel
   float scale_log2;
@@ -902,6 +904,502 @@ tree_attention_tc_kernel(AttnArgs a) {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// =======================================================================================
+// Warp-specialised version of the tcgen05 kernel (the default).
+//
+// Same arithmetic, same shared-memory operand layout and same split merge as the kernel
+// above, but the three kinds of work run in their own warps and talk through mbarriers only;
+// there is no block-wide barrier inside the loop:
+//   warp 4, one thread: TMA producer.  K and V tiles (and Q once) arrive as 64 x 64 boxes of
+//           a 4-D tensor map with 128-byte swizzle, which is exactly the operand layout; rows
+//           past the tensor's extent are zero-filled by the copy engine.  A slot is refilled
+//           as soon as the MMA that read it has completed (tcgen05.commit on its "free" barrier).
+//   warp 5, one thread: MMA issuer.  Q K(t+2)^T is issued right after P V(t), so the tensor
+//           core always has the next S tile ready while the softmax warps work on this one.
+//   warps 0..3: softmax.  Wait for S(t), read it from TMEM, scale / mask / online softmax, fold
+//           P V(t-1) into the register accumulators, store P(t), signal the MMA warp.
+// Every wait is bounded; a wait that gives up raises a block-wide abort word that every other
+// wait polls, so all roles leave their loops and the block still frees its TMEM.
+// =======================================================================================
+constexpr int kWsThreads = 192;
+constexpr int kWsBarBytes = 192;
+// barrier slots (8 bytes each) behind the operand tiles
+enum {
+  kBarKFull = 0, kBarVFull = 16, kBarSFull = 32, kBarOFull = 48, kBarKFree = 56, kBarVFree = 72,
+  kBarPFull = 88, kBarQFull = 96, kBarMerge = 104, kBarTmemSlot = 112, kBarAbort = 116
+};
+__host__ __device__ constexpr int ws_smem_bytes() { return tc_bar_offset(1) + kWsBarBytes; }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait that also gives up when another thread of the block has raised the abort word.
+__device__ __forceinline__ bool mbar_wait_abortable(uint32_t bar, uint32_t parity, volatile uint32_t* abort_word) {
+  const long long start = clock64();
+  for (;;) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (*abort_word != 0u) return false;
+    if (clock64() - start > kWaitCycles) { *abort_word = 1u; return false; }
+  }
+}
+// one 64 x 64 bf16 box (8 KB) of a 4-D tensor map -> shared memory, completion on an mbarrier
+// (row, head, batch) sit at tensor-map coordinates slot[0], slot[1], slot[2] (each 1..3): the map
+// orders its outer dimensions by increasing stride, whatever the caller's layout is.
+__device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* map, int c0, int row, int head,
+                                             int batch, const int (&slot)[3], uint32_t bar) {
+  const int c1 = slot[0] == 1 ? row : slot[1] == 1 ? head : batch;
+  const int c2 = slot[0] == 2 ? row : slot[1] == 2 ? head : batch;
+  const int c3 = slot[0] == 3 ? row : slot[1] == 3 ? head : batch;
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kWsThreads, 2)
+tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
+                         const __grid_constant__ CUtensorMap tm_k,
+                         const __grid_constant__ CUtensorMap tm_v) {
+  constexpr int NB = 1;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int N = a.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool is_softmax = warp < 4;
+  const int g = lane >> 2, t4 = lane & 3;
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t sQ = sbase;
+  const uint32_t sK = sQ + kQBlockBytes;
+  const uint32_t sV = sK + kTcStages * kTileBytes;
+  const uint32_t sP = sV + kTcStages * kTileBytes;
+  const uint32_t bars = sbase + tc_bar_offset(1);
+  const uint32_t bar_m = bars + kBarMerge;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + tc_bar_offset(1) + kBarTmemSlot);
+  volatile uint32_t* abort_word = reinterpret_cast<volatile uint32_t*>(smem + tc_bar_offset(1) + kBarAbort);
+
+  int bid = blockIdx.x;
+  const int split = bid % a.S; bid /= a.S;
+  const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 64-row block of the N draft rows
+  const int h = bid % a.H;
+  const int b = bid / a.H;
+  const int hk = h / a.group;
+  const int L = a.kv_len[b];
+  const int total = L + N;
+  const int ntiles = (total + kBN - 1) / kBN;
+  const int t0 = tc_tile_begin(split, ntiles, a.S);
+  const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
+  const int nt = t1 - t0;
+  const int row0 = rblk * 64;                        // first draft row of this thread block
+  const int Nl = min(64, N - row0);                  // its number of real rows
+
+  if ((sbase & 1023u) != 0) {   // the swizzled operand layout needs a 1024-byte aligned base
+    if (tid == 0) atomicOr(&g_attn_error, 2u);
+    return;                     // uniform over the grid: every block sees the same offset
+  }
+
+  if (tid == 0) {
+    mbar_init(bars + kBarKFull, 1); mbar_init(bars + kBarKFull + 8, 1);
+    mbar_init(bars + kBarVFull, 1); mbar_init(bars + kBarVFull + 8, 1);
+    mbar_init(bars + kBarSFull, 1); mbar_init(bars + kBarSFull + 8, 1);
+    mbar_init(bars + kBarOFull, 1);
+    mbar_init(bars + kBarKFree, 1); mbar_init(bars + kBarKFree + 8, 1);
+    mbar_init(bars + kBarVFree, 1); mbar_init(bars + kBarVFree + 8, 1);
+    mbar_init(bars + kBarPFull, 4);            // one arrival per softmax warp
+    mbar_init(bars + kBarQFull, 1);
+    mbar_init(bar_m, 1);
+    *abort_word = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (a.S > 1) {   // merge: this block will receive its rows of every peer's partial
+      const int Rm = (Nl + a.C - 1) / a.C;
+      const int mine = max(0, min(Rm, Nl - (split % a.C) * Rm));
+      mbar_expect_tx(bar_m, (uint32_t)(a.C * mine * kOStride * 4));
+    }
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // rows of this thread (softmax warps): rows 16 warp + g and + 8; mask row as two 64-bit halves
+  unsigned long long mlo[NB][2], mhi[NB][2];
+  float o[NB][16][4];
+  float m_run[NB][2], l_run[NB][2], alpha[NB][2];
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = (warp & 3) * 16 + g + 8 * hh;
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (is_softmax && row < Nl) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row0 + row) * a.Wm + i];
+      }
+      mlo[rb][hh] = (unsigned long long)w[0] | ((unsigned long long)w[1] << 32);
+      mhi[rb][hh] = (unsigned long long)w[2] | ((unsigned long long)w[3] << 32);
+      m_run[rb][hh] = -INFINITY; l_run[rb][hh] = 0.f; alpha[rb][hh] = 1.f;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) { o[rb][i][0] = o[rb][i][1] = o[rb][i][2] = o[rb][i][3] = 0.f; }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_warp = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+
+  if (warp == 4) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(bars + kBarQFull, (uint32_t)kQBlockBytes);
+      tma_load_box(sQ, &tm_q, 0, row0, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 64 * 128, &tm_q, 64, row0, h, b, a.q_slot, bars + kBarQFull);
+      int issued_k = 0, issued_v = 0;
+      for (int it = 0; it < nt; ++it) {
+        const int slot = it & 1, key0 = (t0 + it) * kBN;
+        const uint32_t free_parity = (uint32_t)(((it >> 1) + 1) & 1);
+        if (it >= 2 && !mbar_wait_abortable(bars + kBarKFree + slot * 8, free_parity, abort_word)) break;
+        mbar_expect_tx(bars + kBarKFull + slot * 8, (uint32_t)kTileBytes);
+        tma_load_box(sK + slot * kTileBytes, &tm_k, 0, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
+        tma_load_box(sK + slot * kTileBytes + 64 * 128, &tm_k, 64, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
+        ++issued_k;
+        if (it >= 2 && !mbar_wait_abortable(bars + kBarVFree + slot * 8, free_parity, abort_word)) break;
+        mbar_expect_tx(bars + kBarVFull + slot * 8, (uint32_t)kTileBytes);
+        tma_load_box(sV + slot * kTileBytes, &tm_v, 0, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
+        tma_load_box(sV + slot * kTileBytes + 64 * 128, &tm_v, 64, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
+        ++issued_v;
+      }
+      if (*abort_word != 0u) {
+        // giving up: let the copies already in flight land before this block goes away
+        mbar_wait(bars + kBarQFull, 0u);
+        for (int it = max(0, issued_k - 2); it < issued_k; ++it)
+          mbar_wait(bars + kBarKFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
+        for (int it = max(0, issued_v - 2); it < issued_v; ++it)
+          mbar_wait(bars + kBarVFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma_idesc(64, kBN, 0);
+      constexpr uint32_t idesc_o = umma_idesc(64, kD, 1);
+      const uint64_t dq0 = umma_desc(sQ, 16, 1024);
+      const uint64_t dk0 = umma_desc(sK, 16, 1024);
+      const uint64_t dp0 = umma_desc(sP, 16, 1024);
+      const uint64_t dv0 = umma_desc(sV, kBN * 128, 1024);
+      bool ok = mbar_wait_abortable(bars + kBarQFull, 0u, abort_word);
+      // S[it & 1] = Q K(t)^T.  The S buffer is free: its previous reader stored P(it - 2) only
+      // after reading it, and P(it - 2) was waited for before this call.
+      auto issue_qk = [&](int it) -> bool {
+        const int slot = it & 1;
+        if (!mbar_wait_abortable(bars + kBarKFull + slot * 8, (uint32_t)((it >> 1) & 1), abort_word)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t koff = (uint32_t)((ks >> 2) * (64 * 128) + (ks & 3) * 32);
+          umma_f16(tmem_base + kColS + slot * 64, dq0 + (koff >> 4),
+                   dk0 + ((slot * kTileBytes + koff) >> 4), idesc_s, ks > 0);
+        }
+        umma_commit(bars + kBarSFull + slot * 8);
+        umma_commit(bars + kBarKFree + slot * 8);
+        return true;
+      };
+      if (ok && nt > 0) ok = issue_qk(0);
+      if (ok && nt > 1) ok = issue_qk(1);
+      for (int it = 0; ok && it < nt; ++it) {
+        const int slot = it & 1;
+        // P(it) is in shared memory; its writers had folded P V(it - 1) before, so O is free
+        if (!mbar_wait_abortable(bars + kBarPFull, (uint32_t)(it & 1), abort_word)) break;
+        if (!mbar_wait_abortable(bars + kBarVFull + slot * 8, (uint32_t)((it >> 1) & 1), abort_word)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          umma_f16(tmem_base + kColO, dp0 + ((kk * 32) >> 4),
+                   dv0 + ((slot * kTileBytes + kk * 2048) >> 4), idesc_o, kk > 0);
+        umma_commit(bars + kBarOFull);
+        umma_commit(bars + kBarVFree + slot * 8);
+        if (it + 2 < nt) ok = issue_qk(it + 2);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax warps
+    auto fold_pv = [&]() {           // o = o * alpha + (P V of the previous tile)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t orr[32];
+        tmem_ld_16x64(tmem_warp + kColO + hf * 64, orr);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          float* oo = o[0][hf * 8 + k];
+          oo[0] = oo[0] * alpha[0][0] + __uint_as_float(orr[4 * k]);
+          oo[1] = oo[1] * alpha[0][0] + __uint_as_float(orr[4 * k + 1]);
+          oo[2] = oo[2] * alpha[0][1] + __uint_as_float(orr[4 * k + 2]);
+          oo[3] = oo[3] * alpha[0][1] + __uint_as_float(orr[4 * k + 3]);
+        }
+      }
+    };
+    bool ok = true;
+    for (int it = 0; ok && it < nt; ++it) {
+      const int t = t0 + it;
+      if (!mbar_wait_abortable(bars + kBarSFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1), abort_word)) break;
+      tc_fence_after();
+      const int key0 = t * kBN;
+      const bool need_mask = key0 + kBN > L;
+      uint32_t pk[NB][16];
+      float alpha_new[NB][2];
+#pragma unroll
+      for (int rb = 0; rb < NB; ++rb) {
+        uint32_t sr[32];
+        tmem_ld_16x64(tmem_warp + kColS + (it & 1) * 64, sr);
+        tmem_wait_ld();
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+        if (!need_mask) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float v0 = __uint_as_float(sr[4 * k]) * a.scale_log2, v1 = __uint_as_float(sr[4 * k + 1]) * a.scale_log2;
+            const float v2 = __uint_as_float(sr[4 * k + 2]) * a.scale_log2, v3 = __uint_as_float(sr[4 * k + 3]) * a.scale_log2;
+            sr[4 * k] = __float_as_uint(v0); sr[4 * k + 1] = __float_as_uint(v1);
+            sr[4 * k + 2] = __float_as_uint(v2); sr[4 * k + 3] = __float_as_uint(v3);
+            mx0 = fmaxf(mx0, fmaxf(v0, v1));
+            mx1 = fmaxf(mx1, fmaxf(v2, v3));
+          }
+        } else {
+          // 64-bit "key j of this tile is visible" masks of the thread's two rows: prefix keys,
+          // then the row's tree bits moved to where key L sits in this tile
+          unsigned long long am[2];
+          const int off = L - key0;                // position of key L in this tile (may be < 0)
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            unsigned long long pre = off >= 64 ? ~0ull : (off <= 0 ? 0ull : ((1ull << off) - 1ull));
+            unsigned long long tb;
+            if (off >= 64) tb = 0ull;
+            else if (off >= 0) tb = mlo[rb][hh] << off;
+            else if (off > -64) tb = (mlo[rb][hh] >> (-off)) | (mhi[rb][hh] << (64 + off));
+            else if (off > -128) tb = mhi[rb][hh] >> (-off - 64);
+            else tb = 0ull;
+            am[hh] = (pre | tb) >> (2 * t4);
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const bool ok = (am[e >> 1] >> (8 * k + (e & 1))) & 1ull;
+              const float v = ok ? __uint_as_float(sr[4 * k + e]) * a.scale_log2 : -INFINITY;
+              sr[4 * k + e] = __float_as_uint(v);
+            }
+            mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sr[4 * k]), __uint_as_float(sr[4 * k + 1])));
+            mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sr[4 * k + 2]), __uint_as_float(sr[4 * k + 3])));
+          }
+        }
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+        const float mn0 = fmaxf(m_run[rb][0], mx0), mn1 = fmaxf(m_run[rb][1], mx1);
+        const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+        alpha_new[rb][0] = ex2(m_run[rb][0] - ms0);  // m = -inf gives 0
+        alpha_new[rb][1] = ex2(m_run[rb][1] - ms1);
+        m_run[rb][0] = mn0; m_run[rb][1] = mn1;
+        float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float e0 = ex2(__uint_as_float(sr[4 * k]) - ms0), e1 = ex2(__uint_as_float(sr[4 * k + 1]) - ms0);
+          const float e2 = ex2(__uint_as_float(sr[4 * k + 2]) - ms1), e3 = ex2(__uint_as_float(sr[4 * k + 3]) - ms1);
+          ps0 += e0 + e1;
+          ps1 += e2 + e3;
+          pk[rb][2 * k] = pack_bf16(e0, e1);
+          pk[rb][2 * k + 1] = pack_bf16(e2, e3);
+        }
+        l_run[rb][0] = l_run[rb][0] * alpha_new[rb][0] + ps0;
+        l_run[rb][1] = l_run[rb][1] * alpha_new[rb][1] + ps1;
+      }
+      if (it > 0) {
+        if (!mbar_wait_abortable(bars + kBarOFull, (uint32_t)((it - 1) & 1), abort_word)) break;
+        tc_fence_after();
+        fold_pv();
+      }
+      alpha[0][0] = alpha_new[0][0]; alpha[0][1] = alpha_new[0][1];
+      if (key0 + kBN > total) {
+        // Ragged last tile: rows of V past the last real key hold whatever the cache holds
+        // there.  Their probabilities are zero, but 0 x NaN is NaN: clear them.
+        if (!mbar_wait_abortable(bars + kBarVFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1), abort_word)) break;
+        const int first = total - key0;            // 0 < first < 64
+        for (int c = tid; c < (kBN - first) * 16; c += 128) {
+          const int row = first + (c >> 4), chunk = c & 15;
+          const uint32_t dst = sV + (it & 1) * kTileBytes + (chunk >> 3) * (64 * 128) + (row >> 3) * 1024 +
+                               (row & 7) * 128 + (((chunk & 7) ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+        }
+      }
+      {
+        // P (bf16) -> shared memory, K-major 128-byte-swizzled [64 rows x 64 keys]
+        const int rr0 = warp * 16 + g, rr1 = rr0 + 8;
+        const uint32_t p0 = sP + (rr0 >> 3) * 1024 + (rr0 & 7) * 128 + t4 * 4;
+        const uint32_t p1 = sP + (rr1 >> 3) * 1024 + (rr1 & 7) * 128 + t4 * 4;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(p0 + ((k ^ (rr0 & 7)) << 4)), "r"(pk[0][2 * k]) : "memory");
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(p1 + ((k ^ (rr1 & 7)) << 4)), "r"(pk[0][2 * k + 1]) : "memory");
+        }
+      }
+      fence_async_smem();                          // P (and cleared V rows) -> visible to the tensor core
+      tc_fence_before();                           // this warp's TMEM reads are done
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + kBarPFull);
+    }
+    if (nt > 0 && *abort_word == 0u) {             // the last tile's P V
+      if (mbar_wait_abortable(bars + kBarOFull, (uint32_t)((nt - 1) & 1), abort_word)) {
+        tc_fence_after();
+        fold_pv();
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_word != 0u && tid == 0) atomicOr(&g_attn_error, 1u);
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
+                 : "memory");
+  }
+
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      l_run[rb][hh] += __shfl_xor_sync(0xFFFFFFFFu, l_run[rb][hh], 1);
+      l_run[rb][hh] += __shfl_xor_sync(0xFFFFFFFFu, l_run[rb][hh], 2);
+    }
+  }
+
+  if (a.S == 1) {
+#pragma unroll
+    for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int row = rb * 64 + warp * 16 + g + 8 * hh;
+        if (!is_softmax || row >= Nl) continue;
+        const float l = l_run[rb][hh];
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)(row0 + row) * a.o_n + h * a.o_h;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          *reinterpret_cast<uint32_t*>(op + i * 8 + t4 * 2) =
+              pack_bf16(o[rb][i][2 * hh] * inv, o[rb][i][2 * hh + 1] * inv);
+        if (a.lse && t4 == 0)
+          a.lse[((int64_t)b * a.H + h) * N + row0 + row] = (m_run[rb][hh] + log2f(l)) * kLn2;
+      }
+    }
+    return;
+  }
+
+  // Merge across the cluster by pushing.  Rows [r*R, r*R + R) belong to block r.  A partial
+  // row is 132 floats: 128 of O, then (max, sum).  Each block stages its rows in its own
+  // shared memory and, once every block of the cluster is done with its operand tiles, sends
+  // each owner its rows with ONE bulk shared-to-shared copy that signals the owner's mbarrier
+  // (armed at start-up with the byte count it will receive).  Nobody waits on a remote round
+  // trip; the owner reduces its C slots locally as soon as its mbarrier completes.
+  const int C = a.C;
+  const int rank = split % C;
+  const int R = (Nl + C - 1) / C;
+  float* sStage = reinterpret_cast<float*>(smem);                    // [Nl][kOStride]
+  float* sRecv = sStage + (size_t)Nl * kOStride;                     // [C][R][kOStride]
+#pragma unroll
+  for (int rb = 0; rb < NB; ++rb) {
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = rb * 64 + warp * 16 + g + 8 * hh;
+      if (!is_softmax || row >= Nl) continue;
+      float* ro = sStage + row * kOStride;
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        *reinterpret_cast<float2*>(ro + i * 8 + t4 * 2) = make_float2(o[rb][i][2 * hh], o[rb][i][2 * hh + 1]);
+      if (t4 == 0) *reinterpret_cast<float2*>(ro + kD) = make_float2(m_run[rb][hh], l_run[rb][hh]);
+    }
+  }
+  fence_async_smem();                          // staged rows -> visible to the bulk-copy engine
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every block's tiles are dead
+  if (tid < C) {
+    const int owner = tid;
+    const int rows = max(0, min(R, Nl - owner * R));
+    if (rows > 0) {
+      const uint32_t src = smem_u32(sStage + (size_t)owner * R * kOStride);
+      const uint32_t dst_local = smem_u32(sRecv + (size_t)rank * R * kOStride);
+      uint32_t dst, rbar;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(dst_local), "r"(owner));
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(bar_m), "r"(owner));
+      asm volatile(
+          "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+          ::"r"(dst), "r"(src), "r"((uint32_t)(rows * kOStride * 4)), "r"(rbar)
+          : "memory");
+    }
+  }
+  int merge_timeout = mbar_wait(bar_m, 0u) ? 0 : 1;
+
+  const int sup = split / C;
+  const int my_rows = max(0, min(R, Nl - rank * R));
+  for (int idx = tid; idx < my_rows * 32; idx += kWsThreads) {
+    const int lr = idx >> 5, mr = row0 + rank * R + lr, c4 = idx & 31;   // mr: global draft row
+    float2 ml[kMaxCluster];
+    float4 ov[kMaxCluster];
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p) {
+      if (p < C) {
+        const float* rr = sRecv + (size_t)(p * R + lr) * kOStride;
+        ml[p] = *reinterpret_cast<const float2*>(rr + kD);
+        ov[p] = *reinterpret_cast<const float4*>(rr + c4 * 4);
+      }
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p)
+      if (p < C) M = fmaxf(M, ml[p].x);
+    float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lsum = 0.f;
+#pragma unroll
+    for (int p = 0; p < kMaxCluster; ++p) {
+      if (p < C) {
+        const float w = (ml[p].x == -INFINITY) ? 0.f : ex2(ml[p].x - M);
+        lsum += ml[p].y * w;
+        o4.x += ov[p].x * w; o4.y += ov[p].y * w; o4.z += ov[p].z * w; o4.w += ov[p].w * w;
+      }
+    }
+    if (a.Sp == 1) {
+      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+      uint2 pk2;
+      pk2.x = pack_bf16(o4.x * inv, o4.y * inv);
+      pk2.y = pack_bf16(o4.z * inv, o4.w * inv);
+      *reinterpret_cast<uint2*>(a.out + b * a.o_b + (int64_t)mr * a.o_n + h * a.o_h + c4 * 4) = pk2;
+      if (a.lse && c4 == 0) a.lse[((int64_t)b * a.H + h) * N + mr] = (M + log2f(lsum)) * kLn2;
+    } else {
+      const int64_t base = ((((int64_t)b * a.H + h) * a.Sp + sup) * N + mr);
+      *reinterpret_cast<float4*>(a.ws_o + base * kD + c4 * 4) = o4;
+      if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
+    }
+  }
+  if (merge_timeout && tid == 0) atomicOr(&g_attn_error, 1u);
+  // stay until every peer has received what this block sent (its staged rows are the source)
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
 __global__ void __launch_bounds__(128)
 tree_attention_combine_kernel(AttnArgs a) {
@@ -937,19 +1435,74 @@ tree_attention_combine_kernel(AttnArgs a) {
   if (a.lse && lane == 0) a.lse[bh * a.N + row] = (M + log2f(lsum)) * kLn2;
 }
 
+// cuTensorMapEncodeTiled is reached through the runtime's driver entry point (no link against
+// libcuda).  The maps describe bf16 tensors (d = 128, rows, heads, batch) with arbitrary 16-byte
+// aligned strides; a box is 64 elements x 64 rows with 128-byte swizzle; out-of-range rows read
+// as zeros.
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult st;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &st) != cudaSuccess ||
+        st != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+bool encode_box_map(CUtensorMap* map, const void* base, int64_t rows, int64_t heads, int64_t batch,
+                    int64_t row_stride, int64_t head_stride, int64_t batch_stride, int (&slot)[3]) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  // outer dimensions in order of increasing stride (size-1 dimensions last: their stride is unused)
+  int64_t size[3] = {rows, heads, batch}, stride[3] = {row_stride, head_stride, batch_stride};
+  int order[3] = {0, 1, 2};
+  auto key = [&](int i) { return size[i] > 1 ? stride[i] : (int64_t)1 << 60; };
+  for (int i = 0; i < 3; ++i)
+    for (int j = i + 1; j < 3; ++j)
+      if (key(order[j]) < key(order[i])) { int t = order[i]; order[i] = order[j]; order[j] = t; }
+  cuuint64_t dims[4] = {(cuuint64_t)kD, 1, 1, 1};
+  cuuint64_t strides[3] = {0, 0, 0};
+  cuuint32_t box[4] = {64, 1, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  cuuint64_t prev = (cuuint64_t)kD * 2;
+  for (int i = 0; i < 3; ++i) {
+    const int which = order[i];
+    slot[which] = i + 1;
+    dims[i + 1] = (cuuint64_t)size[which];
+    // the stride of a size-1 dimension never addresses anything: keep it legal and non-decreasing
+    cuuint64_t st = size[which] > 1 ? (cuuint64_t)stride[which] * 2 : prev * dims[i];
+    if (st < prev) st = prev;
+    strides[i] = st;
+    prev = st;
+    if (which == 0) box[i + 1] = 64;
+  }
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct SplitPlan { int S, C, Sp; };
 
 // Key splits per (context, head): enough blocks to fill the GPU once (never a partial second
 // wave), at most one split per tile, rounded down to a whole number of clusters.
-// REST_ATTENTION_IMPL=mma_sync selects the older mma.sync kernel (kept for comparison runs);
-// anything else, or unset, runs the tcgen05 kernel.
-bool use_tcgen05() {
-  static const bool v = [] {
+// REST_ATTENTION_IMPL selects an older kernel for comparison runs: "cp_async" = the tcgen05
+// kernel fed by cp.async, "mma_sync" = the mma.sync kernel.  Unset or anything else: the
+// warp-specialised tcgen05 + TMA kernel.
+int attention_impl() {
+  static const int v = [] {
     const char* e = getenv("REST_ATTENTION_IMPL");
-    return !(e && strcmp(e, "mma_sync") == 0);
+    if (e && strcmp(e, "mma_sync") == 0) return 2;
+    if (e && strcmp(e, "cp_async") == 0) return 1;
+    return 0;
   }();
   return v;
 }
+bool use_tcgen05() { return attention_impl() != 2; }
 
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
@@ -1030,10 +1583,13 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
     a.ws_ml = a.ws_o + (size_t)B * H * a.Sp * N * kD;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool tc = use_tcgen05();
+  const int impl = attention_impl();
+  const bool tc = impl != 2;
   a.NBLK = tc ? (N + 63) / 64 : 1;
-  const size_t smem = tc ? (size_t)tc_smem_bytes(1) : attn_smem_bytes(N);
-  if (tc)
+  const size_t smem = impl == 0 ? (size_t)ws_smem_bytes() : impl == 1 ? (size_t)tc_smem_bytes(1) : attn_smem_bytes(N);
+  if (impl == 0)
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 4, smem));
+  else if (impl == 1)
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_tc_kernel<1>),
                                             3, smem));
   else
@@ -1042,7 +1598,7 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(B * H * a.NBLK * a.S), 1, 1);
-  cfg.blockDim = dim3((unsigned)(tc ? kTcThreads : (N / 16) * 32), 1, 1);
+  cfg.blockDim = dim3((unsigned)(impl == 0 ? kWsThreads : impl == 1 ? kTcThreads : (N / 16) * 32), 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -1052,10 +1608,20 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (tc)
+  if (impl == 0) {
+    // tensor maps: Q (d, N rows, H, B); K and V (d, max_kv rows, H_kv, B)
+    CUtensorMap tm_q, tm_k, tm_v;
+    int v_slot[3];
+    if (!encode_box_map(&tm_q, d_q, N, H, B, a.q_n, a.q_h, a.q_b, a.q_slot) ||
+        !encode_box_map(&tm_k, d_k, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, a.kv_slot) ||
+        !encode_box_map(&tm_v, d_v, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, v_slot))
+      return rest::note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, a, tm_q, tm_k, tm_v));
+  } else if (impl == 1) {
     REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<1>, a));
-  else
+  } else {
     REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_kernel, a));
+  }
   rest::count_launch();
   if (a.Sp > 1) {
     const int64_t units = (int64_t)B * H * N;
