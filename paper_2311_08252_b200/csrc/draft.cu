@@ -123,11 +123,13 @@ __device__ __forceinline__ int64_t sample_slot(int64_t lo, int64_t cnt, int K, i
 }
 
 // Smallest set bit strictly after position j (the bitmap carries a sentinel past the rows).
-__device__ __forceinline__ int next_set(const uint32_t* __restrict__ row, int j) {
-  int w = j >> 5;
-  uint32_t bits = row[w] & ~((2u << (j & 31)) - 1u);
-  while (bits == 0) bits = row[++w];
-  return (w << 5) + __ffs(bits) - 1;
+// jump[w] holds the position of the first set bit in the words after w, so a run that spans
+// many words costs one more load, not one per word.
+__device__ __forceinline__ int next_set(const uint32_t* __restrict__ row,
+                                        const uint16_t* __restrict__ jump, int j) {
+  const int w = j >> 5;
+  const uint32_t bits = row[w] & ~((2u << (j & 31)) - 1u);
+  return bits ? (w << 5) + __ffs(bits) - 1 : (int)jump[w];
 }
 
 // Largest set bit at or before position j (bit 0 is always set).
@@ -168,6 +170,7 @@ struct Smem {
   int q[16];
   long long lb[17], ub[17];
   uint32_t e1[kMaxM + 1];      // nodes of weight 1 per depth
+  int e1diff[kMaxM + 2];       // the same as a difference array over depths, before the prefix sum
   uint32_t heavy_total;        // nodes of weight >= 2
   int err;
   int bin_hi;
@@ -191,6 +194,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   Smem& s = *reinterpret_cast<Smem*>(smem_raw);
   uint16_t* lenlcp = reinterpret_cast<uint16_t*>(smem_raw + sizeof(Smem));          // [kcap]
   uint32_t* bm = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Smem) + 2 * a.kcap); // [m][nwords]
+  uint16_t* jump = reinterpret_cast<uint16_t*>(bm + a.m * a.nwords);                // [m][nwords]
 
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -212,6 +216,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   if (tid == 0) { s.err = 0; s.heavy_total = 0; s.nsel = 0; }
   if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; }
   if (tid <= kMaxM) s.e1[tid] = 0;
+  if (tid <= kMaxM + 1) s.e1diff[tid] = 0;
   for (int i = tid; i < kHistHi; i += kThreads) s.hist_hi[i] = 0;
   for (int i = tid; i < kHistLo; i += kThreads) s.hist_lo[i] = 0;
   __syncthreads();
@@ -280,16 +285,28 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   const int niter = (Kp + kThreads - 1) / kThreads;
 
   // ---- phase 2: gather rows, common-prefix lengths, node-start bitmaps --------------------
+  // the suffix-array entry of the next iteration's row is fetched one iteration ahead, so
+  // that the two dependent reads (entry, then tokens) of consecutive iterations overlap
+  // (lane 0 also needs the row before its own, which another warp holds: it fetches that
+  // entry ahead as well and reads both rows' tokens side by side)
+  int64_t p_next = 0, pp_next = 0;
+  if (tid < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid));
+  if (lane == 0 && tid > 0 && tid <= Kp)
+    pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid - 1));
   for (int it = 0; it < niter; ++it) {
     const int jbase = it * kThreads + warp * 32;
-    if (jbase >= Kp) continue;   // warp-uniform
     const int j = jbase + lane;
+    int64_t p = p_next;
+    const int64_t pp = pp_next;
+    if (j + kThreads < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + kThreads));
+    if (lane == 0 && j + kThreads <= Kp)
+      pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + kThreads - 1));
+    if (jbase >= Kp) continue;   // warp-uniform
     const bool valid = j < Kp;
     int row[kMaxM], prev[kMaxM];
     int len = 0, plen = 0;
     bool bad = false;
     if (valid) {
-      int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
       if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
       int64_t base = p + n_win;
       int64_t rem = n_tokens - base;
@@ -304,7 +321,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
     for (int d = 0; d < kMaxM; ++d) prev[d] = __shfl_up_sync(kFull, row[d], 1);
     plen = __shfl_up_sync(kFull, len, 1);
     if (lane == 0 && j > 0) {   // previous row belongs to another warp: fetch it again
-      int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j - 1));
+      int64_t p = pp;
       if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
       int64_t base = p + n_win;
       int64_t rem = n_tokens - base;
@@ -352,6 +369,30 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
     return;
   }
 
+  // jump table: for every depth (one warp each) a suffix scan over the bitmap words, last chunk
+  // of 32 words first: jump[w] = position of the first set bit in any word after w
+  if (warp < m) {
+    const uint32_t* row = bm + warp * nwords;
+    uint16_t* jrow = jump + warp * nwords;
+    const int last = (Kp + 31) >> 5;              // the sentinel word
+    int carry = 0x7FFFFFFF;
+    for (int c = last >> 5; c >= 0; --c) {
+      const int wi = c * 32 + lane;
+      const uint32_t bits = wi <= last ? row[wi] : 0u;
+      int v = bits ? (wi << 5) + __ffs(bits) - 1 : 0x7FFFFFFF;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {          // inclusive suffix minimum over the lanes
+        const int u = __shfl_down_sync(kFull, v, o);
+        if (lane + o < 32) v = min(v, u);
+      }
+      v = min(v, carry);
+      const int after = __shfl_down_sync(kFull, v, 1);
+      if (wi <= last) jrow[wi] = (uint16_t)min(lane < 31 ? after : carry, 0xFFFF);
+      carry = __shfl_sync(kFull, v, 0);
+    }
+  }
+  __syncthreads();
+
   // ---- phase 3a: histogram of (weight, depth) over all Trie nodes --------------------------
   // key = weight << 5 | (16 - depth): larger key = better node.
   for (int it = 0; it < niter; ++it) {
@@ -361,21 +402,33 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
     const bool valid = j < Kp;
     const int ll = valid ? lenlcp[j] : 0;
     const int lcp = ll & 0xFF, len = ll >> 8;
+    // Weights along a row never grow with depth: walk down from the first depth at which the
+    // row starts a node until the weight drops to 1; every deeper node of the row weighs 1.
     uint32_t nheavy = 0;
-    for (int d = 1; d <= m; ++d) {
-      const bool act = valid && d > lcp && d <= len;
-      int c = 0;
-      if (act) c = next_set(bm + (d - 1) * nwords, j) - j;
-      uint32_t ones = __ballot_sync(kFull, act && c == 1);
-      if (lane == 0 && ones) atomicAdd(&s.e1[d], __popc(ones));
-      if (act && c >= 2) {
+    int d1 = len + 1;                      // first depth of weight 1 (len + 1: none)
+    if (valid) {
+      for (int d = lcp + 1; d <= len; ++d) {
+        const int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
+        if (c < 2) { d1 = d; break; }
         atomicAdd(&s.hist_hi[((c << 5) | (16 - d)) >> 10], 1u);
         ++nheavy;
       }
     }
+    // weight-1 nodes per depth: d1 <= d <= len, counted as starts minus ends per warp
+    for (int d = 1; d <= m + 1; ++d) {
+      const uint32_t st = __ballot_sync(kFull, valid && d1 == d && d1 <= len);
+      const uint32_t en = __ballot_sync(kFull, valid && d1 <= len && len + 1 == d);
+      if (lane == 0 && (st | en)) atomicAdd(&s.e1diff[d], __popc(st) - __popc(en));
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) nheavy += __shfl_xor_sync(kFull, nheavy, o);
     if (lane == 0 && nheavy) atomicAdd(&s.heavy_total, nheavy);
+  }
+  __syncthreads();
+
+  if (tid == 0) {
+    int run = 0;
+    for (int d = 1; d <= m; ++d) { run += s.e1diff[d]; s.e1[d] = (uint32_t)run; }
   }
   __syncthreads();
 
@@ -395,7 +448,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       const int ll = lenlcp[j];
       const int lcp = ll & 0xFF, len = ll >> 8;
       for (int d = lcp + 1; d <= len; ++d) {
-        int c = next_set(bm + (d - 1) * nwords, j) - j;
+        int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
         if (c < 2) break;   // weights do not grow with depth
         uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
         if ((int)(key >> 10) == bin_hi) atomicAdd(&s.hist_lo[key & 1023u], 1u);
@@ -430,13 +483,14 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       const int ll = lenlcp[j];
       const int lcp = ll & 0xFF, len = ll >> 8;
       for (int d = lcp + 1; d <= len; ++d) {
-        int c = next_set(bm + (d - 1) * nwords, j) - j;
+        int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
         uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
         if (key > tstar) {
           uint32_t slot = atomicAdd(&s.nsel, 1u);
           if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)j; s.selcnt[slot] = c; }
-        } else if (key == tstar) {
-          tie = true;
+        } else {
+          tie = key == tstar;
+          break;                           // keys only fall with depth along a row
         }
       }
     }
@@ -530,7 +584,7 @@ size_t draft_smem_bytes(int K, int m, int* kcap_out, int* nwords_out) {
   int nwords = kcap / 32 + 1;
   if (kcap_out) *kcap_out = kcap;
   if (nwords_out) *nwords_out = nwords;
-  size_t bytes = sizeof(Smem) + 2 * (size_t)kcap + 4 * (size_t)m * nwords;
+  size_t bytes = sizeof(Smem) + 2 * (size_t)kcap + (4 + 2) * (size_t)m * nwords;
   return (bytes + 15) / 16 * 16;
 }
 
