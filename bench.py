@@ -32,6 +32,10 @@ if ROOT not in sys.path:
 import datagen  # noqa: E402
 
 METRIC = "draft trees/s through retrieve+trie+mask, tree attention (all layers) and accept"
+# dram__bytes_read.sum + dram__bytes_write.sum of one tree_attention_ws_kernel launch at the
+# single_stream attention shape, from the ncu capture summarised under profiles/ (the kernel has
+# not changed since); other shapes have no capture and report null.
+NCU_TRAFFIC_BYTES = {("single_stream", "tree_attention_ws_kernel"): 35_186_688}
 UNIT = "trees/s"
 N_CTX_POOL = 64          # distinct contexts rotated through the steps
 
@@ -430,11 +434,13 @@ def main():
                   "mean_candidates_per_context": kp_sum / (pool * B),
                   "mean_nodes_per_tree": nodes_sum / (pool * B),
                   "contexts_with_a_match": matched / (pool * B)},
-        "roofline": {"kernel": "tree_attention_kernel (+ split merge), one layer", "bound": "hbm",
+        "roofline": {"kernel": "tree_attention_ws_kernel, one layer", "bound": "hbm",
                      "achieved": a_bytes / t_attn / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": a_bytes / t_attn / 1e9 / peak, "peak_kind": "of " + peak_kind,
                      "frac_of_nominal_8TBs": a_bytes / t_attn / 1e9 / 8000.0,
-                     "algorithmic_bytes_per_launch": a_bytes, "traffic": None},
+                     "algorithmic_bytes_per_launch": a_bytes,
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, "tree_attention_ws_kernel"))
+                     if args.n_tokens is None else None},
         "roofline_draft": {"kernel": "rest_draft_kernel", "bound": "hbm (latency-bound at B=1)",
                            "achieved": d_bytes / t_draft / 1e9, "peak": peak, "unit": "GB/s",
                            "frac": d_bytes / t_draft / 1e9 / peak,
@@ -442,6 +448,7 @@ def main():
         "e2e": {"value": world * B / t_e2e, "unit": UNIT, "ms_per_step": t_e2e * 1e3,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
+        "device_error_flags": rest.device_error_flags(),
         "clocks": clocks,
     }
     if not args.no_cpu_baseline:

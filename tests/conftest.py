@@ -24,3 +24,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _no_device_side_give_ups(request):
+    """After every GPU test: no kernel may have given up on a bounded wait."""
+    yield
+    if "gpu" in request.keywords:
+        import paper_2311_08252_b200 as rest
+        assert rest.device_error_flags() == 0
