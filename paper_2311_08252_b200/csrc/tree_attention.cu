@@ -996,14 +996,12 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   const int h = bid % a.H;
   const int b = bid / a.H;
   const int hk = h / a.group;
-  const int L = a.kv_len[b];
-  const int total = L + N;
-  const int ntiles = (total + kBN - 1) / kBN;
-  const int t0 = tc_tile_begin(split, ntiles, a.S);
-  const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
-  const int nt = t1 - t0;
   const int row0 = rblk * 64;                        // first draft row of this thread block
   const int Nl = min(64, N - row0);                  // its number of real rows
+
+  // Programmatic dependent launch: the next kernel in the stream may start its own set-up now;
+  // this kernel touches no global memory until the one before it has fully completed.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if ((sbase & 1023u) != 0) {   // the swizzled operand layout needs a 1024-byte aligned base
     if (tid == 0) atomicOr(&g_attn_error, 2u);
@@ -1034,6 +1032,15 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+
+  // everything above is independent of the inputs; from here on global memory is read
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int L = a.kv_len[b];
+  const int total = L + N;
+  const int ntiles = (total + kBN - 1) / kBN;
+  const int t0 = tc_tile_begin(split, ntiles, a.S);
+  const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
+  const int nt = t1 - t0;
 
   // rows of this thread (softmax warps): rows 16 warp + g and + 8; mask row as two 64-bit halves
   unsigned long long mlo[NB][2], mhi[NB][2];
@@ -1601,13 +1608,17 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   cfg.blockDim = dim3((unsigned)(impl == 0 ? kWsThreads : impl == 1 ? kTcThreads : (N / 16) * 32), 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)a.C;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // the warp-specialised kernel waits (griddepcontrol.wait) before its first global access, so it
+  // may be launched while the kernel before it in the stream is still draining
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = impl == 0 ? 2 : 1;
   if (impl == 0) {
     // tensor maps: Q (d, N rows, H, B); K and V (d, max_kv rows, H_kv, B)
     CUtensorMap tm_q, tm_k, tm_v;
