@@ -18,6 +18,9 @@ rest_accept_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict
                    int32_t* __restrict__ accept_nodes, int32_t* __restrict__ out_tokens) {
   const int lane = threadIdx.x & 31;
   const int b = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  // launched with programmatic stream serialisation: wait for the kernel before it in the
+  // stream to complete before touching global memory
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (b >= B) return;   // warp-uniform
   const int32_t* tok = tokens + (int64_t)b * N;
   const int32_t* par = parents + (int64_t)b * N;
@@ -60,10 +63,18 @@ extern "C" rest_status rest_accept(const int32_t* d_tokens, const int32_t* d_par
       (!d_accept_nodes && max_depth > 0) || !d_out_tokens)
     return REST_INVALID_ARG;
   int blocks = (B + kWarpsPerBlock - 1) / kWarpsPerBlock;
-  rest_accept_kernel<<<blocks, kWarpsPerBlock * 32, 0, static_cast<cudaStream_t>(stream)>>>(
-      d_tokens, d_parents, d_n_nodes, d_verifier_tokens, B, N, max_depth, d_accept_len,
-      d_accept_nodes, d_out_tokens);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+  cfg.blockDim = dim3(kWarpsPerBlock * 32, 1, 1);
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, rest_accept_kernel, d_tokens, d_parents, d_n_nodes,
+                                   d_verifier_tokens, (int)B, (int)N, (int)max_depth, d_accept_len,
+                                   d_accept_nodes, d_out_tokens));
   rest::count_launch();
-  REST_CUDA_TRY(cudaGetLastError());
   return REST_OK;
 }

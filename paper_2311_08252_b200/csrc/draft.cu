@@ -199,6 +199,9 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   const int b = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = a.N, m = a.m, Wm = (N + 31) >> 5;
+  // a kernel launched behind this one with programmatic stream serialisation may begin its
+  // set-up now (it still waits for this grid to complete before it reads anything)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int32_t* __restrict__ T = a.T;
   const SaT* __restrict__ sa = static_cast<const SaT*>(a.sa);
   const int64_t n_tokens = a.n_tokens;
