@@ -1359,6 +1359,10 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
     }
   }
   int merge_timeout = mbar_wait(bar_m, 0u) ? 0 : 1;
+  // "I have received everything sent to me": once every block of the cluster has said so, all
+  // copies out of this block's staged rows are complete too and it may leave (waited for at
+  // the very end, after the reduction, when it has normally long completed)
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
   const int sup = split / C;
   const int my_rows = max(0, min(R, Nl - rank * R));
@@ -1402,8 +1406,6 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
     }
   }
   if (merge_timeout && tid == 0) atomicOr(&g_attn_error, 1u);
-  // stay until every peer has received what this block sent (its staged rows are the source)
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
