@@ -213,6 +213,28 @@ rest_status rest_accept(const int32_t* d_tokens, const int32_t* d_parents,
                         int32_t* d_accept_nodes, int32_t* d_out_tokens, void* stream);
 
 /*
+ * rest_kv_commit - make the accepted draft path part of the prefix KV cache.
+ *
+ * The paper does not describe the cache; any implementation of its loop (Sec. 3.2: draft,
+ * verify, accept, repeat with the longer context) has to do this between two steps.  For
+ * context b with L = kv_len[b] and len = accept_len[b]: K/V row L + accept_nodes[b][i] of every
+ * kv head is copied to row L + i, i = 0..len-1, in place (accept_nodes[b][i] >= i always holds
+ * for trees written by rest_draft, and the kernel reads all source rows before it writes).
+ *
+ *   d_k, d_v        bf16, element (b,hk,l,d) at b*kv_strides[0] + hk*kv_strides[1] + l*kv_strides[2] + d,
+ *                   same layout rules as rest_tree_attention (D = 128, 16-byte aligned rows)
+ *   d_accept_nodes  int32[B,max_depth], d_accept_len int32[B]: as written by rest_accept
+ *   N               number of tree slots (node indices are clamped to [0, N))
+ *   d_new_kv_len    optional int32[B]: receives L + len (may alias d_kv_len)
+ *   Limits: max_depth <= 16.  The token the verifier produced at the stop (out_tokens[len]) has
+ *   no K/V yet: it is the next step's first input token.
+ */
+rest_status rest_kv_commit(void* d_k, void* d_v, const int64_t* kv_strides, const int32_t* d_kv_len,
+                           const int32_t* d_accept_nodes, const int32_t* d_accept_len, int32_t B,
+                           int32_t H_kv, int32_t N, int32_t D, int32_t max_depth,
+                           int32_t* d_new_kv_len, void* stream);
+
+/*
  * Device-side trouble that no per-call status can carry.  Every wait inside the kernels is
  * bounded; a kernel that gives up sets a bit here instead of spinning, and its output is then
  * undefined.  Reads and clears the flags of the current device (synchronises the device).

@@ -138,3 +138,18 @@ def accept(tokens, parents, n_nodes, verifier_tokens, max_depth):
                         ctypes.c_int32(B), ctypes.c_int32(N), ctypes.c_int32(max_depth),
                         _p(al), _p(an), _p(ot))
     return al, an, ot
+
+
+def kv_commit(k_bits, v_bits, kv_len, accept_nodes, accept_len):
+    """Plain restatement of "the accepted path becomes part of the prefix": returns copies of
+    the uint16 K/V arrays [B,H_kv,Lcap,D] in which row kv_len[b] + i holds what row
+    kv_len[b] + accept_nodes[b][i] held, i < accept_len[b], and the new lengths."""
+    k2, v2 = k_bits.copy(), v_bits.copy()
+    new_len = np.asarray(kv_len, np.int32).copy()
+    for b in range(k_bits.shape[0]):
+        L = int(kv_len[b])
+        for i in range(int(accept_len[b])):
+            k2[b, :, L + i] = k_bits[b, :, L + int(accept_nodes[b, i])]
+            v2[b, :, L + i] = v_bits[b, :, L + int(accept_nodes[b, i])]
+        new_len[b] = L + int(accept_len[b])
+    return k2, v2, new_len

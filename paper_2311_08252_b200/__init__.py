@@ -29,7 +29,7 @@ EXPORTS = (
     "rest_draft_workspace_bytes", "rest_draft",
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
     "rest_tree_attention_static_scratch",
-    "rest_device_error_flags",
+    "rest_device_error_flags", "rest_kv_commit",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -82,6 +82,8 @@ def lib():
                                                      vp, vp]
     L.rest_accept.restype = i32
     L.rest_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    L.rest_kv_commit.restype = i32
+    L.rest_kv_commit.argtypes = [vp, vp, ctypes.POINTER(i64), vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
     L.rest_device_error_flags.restype = i32
     L.rest_device_error_flags.argtypes = [ctypes.POINTER(u32)]
     L.rest_status_string.restype = ctypes.c_char_p
@@ -298,3 +300,26 @@ def rest_accept(tokens, parents, n_nodes, verifier_tokens, max_depth, out=None, 
                        out[1].data_ptr(), out[2].data_ptr(), _stream(stream))
     _check(rc, "rest_accept")
     return out
+
+
+def rest_kv_commit(k, v, kv_len, accept_nodes, accept_len, N, new_kv_len=None, stream=None):
+    """Moves the K/V rows of the accepted draft nodes (tree slots kv_len[b] + node) to the
+    contiguous slots kv_len[b] .. kv_len[b] + accept_len[b] - 1 of k, v bf16 [B,H_kv,Lcap,D], in
+    place.  new_kv_len (optional int32[B]) receives kv_len + accept_len."""
+    import torch
+    L = lib()
+    for t, nm in ((k, "k"), (v, "v")):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.stride(-1) == 1):
+            raise RestError(f"{nm} must be a bf16 CUDA tensor with a contiguous last dimension")
+    if k.stride() != v.stride() or k.shape != v.shape:
+        raise RestError("k and v must have the same shape and strides")
+    for t, nm in ((kv_len, "kv_len"), (accept_nodes, "accept_nodes"), (accept_len, "accept_len")):
+        _dev_i32(t, nm)
+    B, H_kv, _, D = k.shape
+    max_depth = accept_nodes.shape[1]
+    strides = (ctypes.c_int64 * 3)(k.stride(0), k.stride(1), k.stride(2))
+    rc = L.rest_kv_commit(k.data_ptr(), v.data_ptr(), strides, kv_len.data_ptr(), _ptr(accept_nodes),
+                          accept_len.data_ptr(), B, H_kv, N, D, max_depth, _ptr(new_kv_len),
+                          _stream(stream))
+    _check(rc, "rest_kv_commit")
+    return new_kv_len
