@@ -1,19 +1,34 @@
 // rest_tree_attention: masked attention of the N draft positions over the prefix KV cache
 // and over their own ancestors (Sec. 3.2 "Draft verification").
 //
-// Split-KV flash-decode layout: one thread block per (context, head, key split).  A block
-// holds the N x 128 query tile as tensor-core A fragments in registers (16 rows per warp)
-// and streams 64-key K/V tiles through a three-deep, XOR-swizzled shared-memory ring filled
-// with 16-byte asynchronous copies.  Per tile: S = Q K^T (bf16 tensor-core MMA, fp32
-// accumulate), tree mask on the tiles that reach past the prefix, online softmax in base 2,
-// O += P V.
+// Split-KV flash-decode layout on the 5th-generation tensor cores.  One thread block per
+// (context, head, 64-row block of the draft rows, key split) streams 64-key K/V tiles:
+// S = Q K^T and O += P V are tcgen05.mma with the accumulators in TMEM, the operand tiles
+// arrive by TMA, and the tree mask / base-2 online softmax runs in registers in between.
 //
-// The splits of one (context, head) form a thread-block cluster (up to 8 blocks): each block
-// parks its un-normalised partial in its own shared memory, and after a cluster barrier every
-// block merges a slice of the rows straight out of its peers' shared memory (distributed
-// shared memory) and writes bf16 output.  Only when more than 8 splits are needed do the
-// cluster-merged partials go to the caller's workspace for a second, small merge kernel.
-#include <cooperative_groups.h>
+// M = 64 rather than 128 because an M = 64 accumulator spreads its rows over all four TMEM
+// lane quadrants (16 rows each), so every softmax warp - and every warp scheduler - gets an
+// equal share.  Every 64-row block of the N draft rows gets its own thread blocks (grid
+// index: row block fastest after the split, so the blocks of one (context, head) stream the
+// same K/V tiles at the same time and the second reader hits L2).
+//
+// Q ([64 x 128]), the K/V tiles ([64 x 128]) and P ([64 x 64]) sit in shared memory in the
+// tensor core's canonical 128-byte-swizzled layout (8-row groups of 1024 B, the two
+// 64-element halves of the head dimension side by side), so a K tile is a K-major B operand
+// and the very same bytes of a V tile are an MN-major B operand: no transpose anywhere.
+// Per 64-key tile:
+//   8 tcgen05.mma (M=64, N=64, K=16)   ->  S in TMEM columns [0, 64) or [64, 128)
+//   each softmax warp reads its 16 rows with the 16x256b pattern (a row is shared by a quad),
+//   applies scale / tree mask / online softmax, and writes P (bf16) into shared memory
+//   4 tcgen05.mma (M=64, N=128, K=16)  ->  P V in TMEM columns [128, 256)
+//   each warp folds its rows of P V into fp32 register accumulators with the usual rescale.
+//
+// The splits of one (context, head, row block) form a thread-block cluster (up to 8 blocks).
+// Every block stages its un-normalised partial rows in its own shared memory and sends each
+// owner its slice with one bulk shared-to-shared copy that completes on the owner's
+// mbarrier; the owner reduces locally and writes bf16 output.  Only when more than 8 splits
+// are needed do the cluster-merged partials go to the caller's workspace for a second, small
+// merge kernel.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -25,14 +40,11 @@
 #include "common.cuh"
 #include "rest.h"
 
-namespace cg = cooperative_groups;
-
 namespace {
 
 constexpr int kD = REST_HEAD_DIM;     // 128
 constexpr int kBN = 64;               // keys per tile
-constexpr int kStages = 3;
-constexpr int kOStride = kD + 4;         // floats per row of a parked partial (bank spread)
+constexpr int kOStride = kD + 4;      // floats per row of a staged partial: 128 O + m, l (+2 pad)
 constexpr int kMaxCluster = 8;
 constexpr int kRowBytes = kD * 2;     // 256
 constexpr int kTileBytes = kBN * kRowBytes;   // 16 KB
@@ -61,347 +73,27 @@ struct AttnArgs {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool pred) {
-  int sz = pred ? 16 : 0;   // size 0: nothing is read, destination is zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz)
-               : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
-                                        uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
-                                          uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
-                                         uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
-      "{%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-// byte offset of 16-byte chunk `chunk` of row `row` in a swizzled [rows][256 B] tile
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {
-  return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
-}
 
-// Shared memory: Q tile [N][256 B] | K ring [stages][16 KB] | V ring [stages][16 KB] | mask [N][4]
-__global__ void __launch_bounds__(256)
-tree_attention_kernel(AttnArgs a) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  const int N = a.N;
-  unsigned char* sQ = smem;
-  unsigned char* sK = sQ + N * kRowBytes;
-  unsigned char* sV = sK + kStages * kTileBytes;
-  uint32_t* sMask = reinterpret_cast<uint32_t*>(sV + kStages * kTileBytes);
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x;
-  const int g = lane >> 2, t4 = lane & 3;
-  int bid = blockIdx.x;
-  const int split = bid % a.S; bid /= a.S;
-  const int h = bid % a.H;
-  const int b = bid / a.H;
-  const int hk = h / a.group;
-  const int L = a.kv_len[b];
-  const int total = L + N;
-  const int ntiles = (total + kBN - 1) / kBN;
-  const int t0 = (int)(((int64_t)split * ntiles) / a.S);         // balanced partition of the tiles
-  const int t1 = (int)(((int64_t)(split + 1) * ntiles) / a.S);
-
-  const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h;
-  const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
-  const __nv_bfloat16* vb = a.v + b * a.kv_b + hk * a.kv_h;
-
-  // Q tile and mask rows
-  for (int c = tid; c < N * 16; c += nthreads) {
-    int row = c >> 4, chunk = c & 15;
-    cp_async16(smem_u32(sQ) + swz(row, chunk), qb + row * a.q_n + chunk * 8, true);
-  }
-  for (int c = tid; c < N * 4; c += nthreads) {
-    int row = c >> 2, w = c & 3;
-    sMask[c] = (w < a.Wm) ? a.mask[((int64_t)b * N + row) * a.Wm + w] : 0u;
-  }
-  auto load_tile = [&](int tile, int stage) {
-    const int key0 = tile * kBN;
-    const uint32_t dK = smem_u32(sK) + stage * kTileBytes;
-    const uint32_t dV = smem_u32(sV) + stage * kTileBytes;
-    for (int c = tid; c < kBN * 16; c += nthreads) {
-      int row = c >> 4, chunk = c & 15;
-      int key = key0 + row;
-      bool ok = key < total;
-      int64_t off = (int64_t)(ok ? key : 0) * a.kv_l + chunk * 8;
-      cp_async16(dK + swz(row, chunk), kb + off, ok);
-      cp_async16(dV + swz(row, chunk), vb + off, ok);
-    }
-  };
-  if (t0 < t1) load_tile(t0, 0);
-  cp_async_commit();
-  if (t0 + 1 < t1) load_tile(t0 + 1, 1);
-  cp_async_commit();
-
-  float o[16][4];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g+8 of this warp
-  uint32_t qf[8][4];
-  const int r0 = warp * 16 + g, r1 = r0 + 8;
-
-  for (int t = t0; t < t1; ++t) {
-    const int stage = (t - t0) % kStages;
-    if (t + 2 < t1) load_tile(t + 2, (t - t0 + 2) % kStages);   // that slot was drained at t - 1
-    cp_async_commit();                                          // one group per iteration, maybe empty
-    cp_async_wait<2>();                                         // tile t (and Q) have landed
-    __syncthreads();
-    if (t == t0) {
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        int chunk = ks * 2 + (lane >> 4);
-        ldsm_x4(smem_u32(sQ) + swz(row, chunk), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
-      }
-    }
-    const uint32_t bK = smem_u32(sK) + stage * kTileBytes;
-    const uint32_t bV = smem_u32(sV) + stage * kTileBytes;
-
-    // S = Q K^T : 16 rows x 64 keys per warp
-    float s[8][4];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-      for (int np = 0; np < 4; ++np) {   // pairs of 8-key tiles
-        uint32_t b0, b1, b2, b3;
-        int key = np * 16 + (lane & 7) + (lane >> 4) * 8;
-        int chunk = ks * 2 + ((lane >> 3) & 1);
-        ldsm_x4(bK + swz(key, chunk), b0, b1, b2, b3);
-        mma_bf16(s[np * 2], qf[ks], b0, b1);
-        mma_bf16(s[np * 2 + 1], qf[ks], b2, b3);
-      }
-    }
-
-    // scale, mask, online softmax (base 2)
-    const int key0 = t * kBN;
-    const bool need_mask = key0 + kBN > L;
-    float mx0 = -INFINITY, mx1 = -INFINITY;
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        float v = s[nt][e] * a.scale_log2;
-        if (need_mask) {
-          int key = key0 + nt * 8 + t4 * 2 + (e & 1);
-          int row = (e < 2) ? r0 : r1;
-          bool ok = key < L;
-          if (!ok && key < total) {
-            int j = key - L;
-            ok = (sMask[row * 4 + (j >> 5)] >> (j & 31)) & 1u;
-          }
-          if (!ok) v = -INFINITY;
-        }
-        s[nt][e] = v;
-      }
-      mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
-      mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
-    }
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
-    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
-    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
-    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-    const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-    const float al0 = exp2f(m0 - ms0), al1 = exp2f(m1 - ms1);   // m = -inf gives 0
-    m0 = mn0; m1 = mn1;
-    float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      s[nt][0] = exp2f(s[nt][0] - ms0); s[nt][1] = exp2f(s[nt][1] - ms0);
-      s[nt][2] = exp2f(s[nt][2] - ms1); s[nt][3] = exp2f(s[nt][3] - ms1);
-      ps0 += s[nt][0] + s[nt][1];
-      ps1 += s[nt][2] + s[nt][3];
-    }
-    l0 = l0 * al0 + ps0;
-    l1 = l1 * al1 + ps1;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { o[i][0] *= al0; o[i][1] *= al0; o[i][2] *= al1; o[i][3] *= al1; }
-
-    // O += P V
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {   // 16 keys per step
-      uint32_t pa[4];
-      pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-      pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-      pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-      pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-#pragma unroll
-      for (int dp = 0; dp < 8; ++dp) {   // pairs of 8-wide output tiles
-        uint32_t b0, b1, b2, b3;
-        int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        int chunk = dp * 2 + (lane >> 4);
-        ldsm_x4_t(bV + swz(key, chunk), b0, b1, b2, b3);
-        mma_bf16(o[dp * 2], pa, b0, b1);
-        mma_bf16(o[dp * 2 + 1], pa, b2, b3);
-      }
-    }
-    __syncthreads();
-  }
-  cp_async_wait<0>();
-  __syncthreads();   // every warp is done with the K/V ring (and Q tile): reuse it below
-
-  l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1);
-  l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
-  l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 1);
-  l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 2);
-
-  if (a.S == 1) {
-    const float inv0 = l0 > 0.f ? 1.f / l0 : 0.f, inv1 = l1 > 0.f ? 1.f / l1 : 0.f;
-    __nv_bfloat16* ob = a.out + b * a.o_b + h * a.o_h;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      int col = i * 8 + t4 * 2;
-      *reinterpret_cast<uint32_t*>(ob + r0 * a.o_n + col) = pack_bf16(o[i][0] * inv0, o[i][1] * inv0);
-      *reinterpret_cast<uint32_t*>(ob + r1 * a.o_n + col) = pack_bf16(o[i][2] * inv1, o[i][3] * inv1);
-    }
-    if (a.lse && t4 == 0) {
-      float* lp = a.lse + ((int64_t)b * a.H + h) * N;
-      lp[r0] = (m0 + log2f(l0)) * kLn2;
-      lp[r1] = (m1 + log2f(l1)) * kLn2;
-    }
-    return;
-  }
-
-  // Park this block's partial in its own shared memory: O [N][kOStride] fp32, then (max, sum).
-  float* sO = reinterpret_cast<float*>(smem);
-  float* sML = sO + N * kOStride;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    int col = i * 8 + t4 * 2;
-    *reinterpret_cast<float2*>(sO + r0 * kOStride + col) = make_float2(o[i][0], o[i][1]);
-    *reinterpret_cast<float2*>(sO + r1 * kOStride + col) = make_float2(o[i][2], o[i][3]);
-  }
-  if (t4 == 0) {
-    sML[r0 * 2] = m0; sML[r0 * 2 + 1] = l0;
-    sML[r1 * 2] = m1; sML[r1 * 2 + 1] = l1;
-  }
-  cg::cluster_group cluster = cg::this_cluster();
-  cluster.sync();
-
-  // Merge rows [rank*R, rank*R + R) over the C blocks of the cluster, 4 output dims per thread.
-  const int C = a.C;
-  const int rank = (int)cluster.block_rank();
-  const int R = (N + C - 1) / C;
-  const int sup = split / C;
-  for (int idx = tid; idx < R * 32; idx += nthreads) {
-    const int row = rank * R + (idx >> 5), c4 = idx & 31;
-    if (row >= N) continue;
-    // issue every remote read before using any of them (one round trip, not 2*C of them);
-    // an empty split parked zeros with max = -inf, so its weight is 0 and its data harmless
-    float2 ml[kMaxCluster];
-    float4 ov[kMaxCluster];
-#pragma unroll
-    for (int p = 0; p < kMaxCluster; ++p) {
-      if (p < C) {
-        ml[p] = *reinterpret_cast<const float2*>(cluster.map_shared_rank(sML, p) + row * 2);
-        ov[p] = *reinterpret_cast<const float4*>(cluster.map_shared_rank(sO, p) + row * kOStride + c4 * 4);
-      }
-    }
-    float M = -INFINITY;
-#pragma unroll
-    for (int p = 0; p < kMaxCluster; ++p)
-      if (p < C) M = fmaxf(M, ml[p].x);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float lsum = 0.f;
-#pragma unroll
-    for (int p = 0; p < kMaxCluster; ++p) {
-      if (p < C) {
-        const float w = (ml[p].x == -INFINITY) ? 0.f : exp2f(ml[p].x - M);
-        lsum += ml[p].y * w;
-        acc.x += ov[p].x * w; acc.y += ov[p].y * w; acc.z += ov[p].z * w; acc.w += ov[p].w * w;
-      }
-    }
-    if (a.Sp == 1) {
-      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-      uint2 pk;
-      pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-      pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-      *reinterpret_cast<uint2*>(a.out + b * a.o_b + row * a.o_n + h * a.o_h + c4 * 4) = pk;
-      if (a.lse && c4 == 0) a.lse[((int64_t)b * a.H + h) * N + row] = (M + log2f(lsum)) * kLn2;
-    } else {
-      const int64_t base = ((((int64_t)b * a.H + h) * a.Sp + sup) * N + row);
-      *reinterpret_cast<float4*>(a.ws_o + base * kD + c4 * 4) = acc;
-      if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
-    }
-  }
-  cluster.sync();   // nobody leaves while a peer may still read its shared memory
-}
-
-// =======================================================================================
-// tcgen05 version: QK^T and PV on the 5th-generation tensor cores, accumulators in TMEM.
-//
-// One block = 4 softmax warps + 1 MMA-issuing warp.  Query rows are handled in blocks of 64:
-// every 64-row block of the N draft rows gets its own thread blocks (grid index: row block
-// fastest after the split, so the blocks of one (context, head) stream the same K/V tiles at
-// the same time and the second reader hits L2).  M = 64 rather than 128 because an M = 64
-// accumulator spreads its rows over all four TMEM lane quadrants (16 rows each), so every
-// warp - and every warp scheduler - gets an equal share of the softmax.  (The kernel is
-// written for NB row blocks per thread block, the second one in lanes 16..31 of each
-// quadrant; it is instantiated with NB = 1, which keeps two blocks resident per SM.)
-//
-// Q (NB x [64 x 128]), the K/V tiles ([64 x 128]) and P (NB x [64 x 64]) sit in shared memory
-// in the tensor core's canonical 128-byte-swizzled layout (8-row groups of 1024 B, the two
-// 64-element halves of the head dimension side by side), so a K tile is a K-major B operand
-// and the very same bytes of a V tile are an MN-major B operand: no transpose anywhere.
-// Per 64-key tile and row block:
-//   one thread issues 8 tcgen05.mma (M=64, N=64, K=16)   ->  S in TMEM columns [0, 64)
-//   each warp reads its 16 rows with the 16x256b pattern (same register layout as an
-//   mma.sync accumulator: a row is shared by a quad), applies scale / tree mask / base-2
-//   online softmax, and writes P (bf16) into shared memory
-//   one thread issues 4 tcgen05.mma (M=64, N=128, K=16)  ->  P V in TMEM columns [64, 192)
-//   each warp folds its rows of P V into fp32 register accumulators with the usual rescale.
-// The loop is software-pipelined: a fifth warp only issues MMAs, S is double-buffered in TMEM,
-// and Q K(t+1)^T runs on the tensor core while the four softmax warps work on tile t; P V of
-// tile t is folded into the register accumulators one iteration later, when it has long
-// finished.  K and V slots are refilled (16-byte cp.async, committed in a fixed group order)
-// as soon as the MMA that read them has completed.
-// Completion of each MMA group is signalled through an mbarrier (tcgen05.commit); waits are
-// bounded and report through g_attn_error instead of spinning forever.  For N <= 64 two
-// blocks share an SM (2 x 256 TMEM columns).
-// Split merge: the splits of one (context, head) form a cluster; every block pushes its
-// partial rows into the shared memory of the block that owns those rows (posted stores, no
-// remote round trips), and after a cluster barrier each owner reduces locally.
-// =======================================================================================
-constexpr int kTcThreads = 160;             // 4 softmax / copy warps + 1 MMA-issuing warp
-constexpr int kTcStages = 2;
+constexpr int kTcStages = 2;                            // K and V ring depth
 constexpr int kQBlockBytes = 64 * kRowBytes;            // 16 KB: 64 rows x 128 dims
 constexpr int kPBlockBytes = 64 * 128;                  //  8 KB: 64 rows x 64 keys
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;      // S double-buffered in [0,64) and [64,128); P V in [128,256)
 constexpr long long kWaitCycles = 400000000ll;          // ~0.2 s: give up, flag, clean up
 
-// Shared memory of the tcgen05 kernel: operand tiles (Q blocks, K ring, V ring, P blocks), later
-// reused by the split merge, which stages 64 NB partial rows and receives up to 64 NB + 8 rows
-// of kOStride floats; the mbarriers and the TMEM slot sit behind whichever is larger.
+// Shared memory: operand tiles (Q blocks, K ring, V ring, P blocks), later reused by the split
+// merge, which stages 64 NB partial rows and receives up to 64 NB + 8 rows of kOStride floats;
+// the mbarriers and the TMEM slot sit behind whichever is larger.  (NB = 64-row blocks per
+// thread block; the kernel uses NB = 1, which keeps two blocks resident per SM.)
 __host__ __device__ constexpr int tc_operand_bytes(int NB) { return NB * kQBlockBytes + 2 * kTcStages * kTileBytes + NB * kPBlockBytes; }
 __host__ __device__ constexpr int tc_merge_bytes(int NB) { return (2 * 64 * NB + 8) * kOStride * 4; }
 __host__ __device__ constexpr int tc_bar_offset(int NB) {
   return tc_operand_bytes(NB) > tc_merge_bytes(NB) ? tc_operand_bytes(NB) : tc_merge_bytes(NB);
 }
-__host__ __device__ constexpr int tc_smem_bytes(int NB) { return tc_bar_offset(NB) + 64; }
 // Tiles are dealt so that the first splits take the spare ones: the last split, which holds
 // the masked tree tiles, never gets an extra tile.
 __host__ __device__ inline int tc_tile_begin(int split, int ntiles, int S) {
@@ -471,445 +163,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
 }
 
-template <int NB>
-__global__ void __launch_bounds__(kTcThreads, NB == 1 ? 2 : 1)
-tree_attention_tc_kernel(AttnArgs a) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  const int N = a.N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const bool is_mma_warp = warp == 4;          // warps 0..3: copies + softmax; warp 4: issues MMAs
-  const int g = lane >> 2, t4 = lane & 3;
-  const uint32_t sbase = smem_u32(smem);
-  const uint32_t sQ = sbase;
-  const uint32_t sK = sQ + NB * kQBlockBytes;
-  const uint32_t sV = sK + kTcStages * kTileBytes;
-  const uint32_t sP = sV + kTcStages * kTileBytes;
-  const uint32_t bar_s0 = sbase + tc_bar_offset(NB), bar_o = bar_s0 + 16, bar_m = bar_s0 + 32;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + tc_bar_offset(NB) + 24);
-
-  int bid = blockIdx.x;
-  const int split = bid % a.S; bid /= a.S;
-  const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 64-row block of the N draft rows
-  const int h = bid % a.H;
-  const int b = bid / a.H;
-  const int hk = h / a.group;
-  const int L = a.kv_len[b];
-  const int total = L + N;
-  const int ntiles = (total + kBN - 1) / kBN;
-  const int t0 = tc_tile_begin(split, ntiles, a.S);
-  const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
-  const int row0 = rblk * (64 * NB);                 // first draft row of this thread block
-  const int Nl = min(64 * NB, N - row0);             // its number of real rows
-  const __nv_bfloat16* qb = a.q + b * a.q_b + h * a.q_h + (int64_t)row0 * a.q_n;
-  const __nv_bfloat16* kb = a.k + b * a.kv_b + hk * a.kv_h;
-  const __nv_bfloat16* vb = a.v + b * a.kv_b + hk * a.kv_h;
-
-  if ((sbase & 1023u) != 0) {   // the swizzled operand layout needs a 1024-byte aligned base
-    if (tid == 0) atomicOr(&g_attn_error, 2u);
-    return;                     // uniform over the grid: every block sees the same offset
-  }
-
-  // barriers + TMEM
-  if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s0) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s0 + 8) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_m) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (a.S > 1) {   // merge: this block will receive its rows of every peer's partial
-      const int Rm = (Nl + a.C - 1) / a.C;
-      const int mine = max(0, min(Rm, Nl - (split % a.C) * Rm));
-      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_m),
-                   "r"((uint32_t)(a.C * mine * kOStride * 4))
-                   : "memory");
-    }
-  }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(tmem_slot)), "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-
-  // Copy pattern (threads 0..127): thread handles 16-byte chunk (tid & 15) of rows
-  // (tid >> 4) + 8 i.  In the operand layout a row's 8-row group is 1024 B apart and
-  // (row & 7) is fixed per thread, so source and destination advance by constants.
-  const int crow = (tid >> 4) & 7, cchunk = tid & 15;
-  const uint32_t coff = (uint32_t)((cchunk >> 3) * (64 * 128) + crow * 128 + (((cchunk & 7) ^ crow) << 4));
-  auto load_rows = [&](const __nv_bfloat16* base, uint32_t dst, int tile) {
-    const int key0 = tile * kBN + crow;
-    const int64_t src0 = (int64_t)key0 * a.kv_l + cchunk * 8;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const bool ok = key0 + 8 * i < total;
-      cp_async16(dst + coff + i * 1024, base + (ok ? src0 + (int64_t)(8 * i) * a.kv_l : 0), ok);
-    }
-  };
-  // Copy groups are committed in a fixed order so that wait_group counts stay constant:
-  //   prologue: {Q, K(t0)}, {K(t0+1)}, {V(t0)};  iteration t: {K(t+2)}, {V(t+1)}.
-  if (!is_mma_warp) {
-#pragma unroll
-    for (int i = 0; i < NB * 8; ++i) {     // Q rows crow + 8 i; rows >= N zero-filled
-      const int row = crow + 8 * i;
-      const bool ok = row < Nl;
-      cp_async16(sQ + (i >> 3) * kQBlockBytes + coff + (i & 7) * 1024,
-                 qb + (int64_t)(ok ? row : 0) * a.q_n + cchunk * 8, ok);
-    }
-    if (t0 < t1) load_rows(kb, sK, t0);
-    cp_async_commit();
-    if (t0 + 1 < t1) load_rows(kb, sK + kTileBytes, t0 + 1);
-    cp_async_commit();
-    if (t0 < t1) load_rows(vb, sV, t0);
-    cp_async_commit();
-  }
-
-  // rows of this thread: block rb, rows 16 (warp & 3) + g and + 8; mask row as two 64-bit halves
-  unsigned long long mlo[NB][2], mhi[NB][2];
-  float o[NB][16][4];
-  float m_run[NB][2], l_run[NB][2], alpha[NB][2];
-#pragma unroll
-  for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int row = rb * 64 + (warp & 3) * 16 + g + 8 * hh;
-      uint32_t w[4] = {0u, 0u, 0u, 0u};
-      if (!is_mma_warp && row < Nl) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row0 + row) * a.Wm + i];
-      }
-      mlo[rb][hh] = (unsigned long long)w[0] | ((unsigned long long)w[1] << 32);
-      mhi[rb][hh] = (unsigned long long)w[2] | ((unsigned long long)w[3] << 32);
-      m_run[rb][hh] = -INFINITY; l_run[rb][hh] = 0.f; alpha[rb][hh] = 1.f;
-    }
-#pragma unroll
-    for (int i = 0; i < 16; ++i) { o[rb][i][0] = o[rb][i][1] = o[rb][i][2] = o[rb][i][3] = 0.f; }
-  }
-
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_warp = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-  constexpr uint32_t idesc_s = umma_idesc(64, kBN, 0);
-  constexpr uint32_t idesc_o = umma_idesc(64, kD, 1);
-  // descriptor bases; k-steps add (bytes >> 4) to the low word
-  const uint64_t dq0 = umma_desc(sQ, 16, 1024);
-  const uint64_t dk0 = umma_desc(sK, 16, 1024);
-  const uint64_t dp0 = umma_desc(sP, 16, 1024);
-  const uint64_t dv0 = umma_desc(sV, kBN * 128, 1024);
-
-  auto issue_qk = [&](int it) {    // S[it & 1] = Q K(t)^T : 8 k-steps of 16 over the head dim
-    const int stage = it & 1;
-#pragma unroll
-    for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const uint32_t koff = (uint32_t)((ks >> 2) * (64 * 128) + (ks & 3) * 32);
-        umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kColS + stage * 64,
-                 dq0 + ((rb * kQBlockBytes + koff) >> 4),
-                 dk0 + ((stage * kTileBytes + koff) >> 4), idesc_s, ks > 0);
-      }
-    }
-    umma_commit(bar_s0 + stage * 8);
-  };
-  auto fold_pv = [&]() {           // o = o * alpha + (P V of the previous tile)
-#pragma unroll
-    for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        uint32_t orr[32];
-        tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kColO + hf * 64, orr);
-        tmem_wait_ld();
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          float* oo = o[rb][hf * 8 + k];
-          oo[0] = oo[0] * alpha[rb][0] + __uint_as_float(orr[4 * k]);
-          oo[1] = oo[1] * alpha[rb][0] + __uint_as_float(orr[4 * k + 1]);
-          oo[2] = oo[2] * alpha[rb][1] + __uint_as_float(orr[4 * k + 2]);
-          oo[3] = oo[3] * alpha[rb][1] + __uint_as_float(orr[4 * k + 3]);
-        }
-      }
-    }
-  };
-
-  // pipeline prologue: S(t0) is in flight before the loop starts
-  int timed_out = 0;
-  if (t0 < t1) {
-    cp_async_wait<2>();
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    if (is_mma_warp && lane == 0) { tc_fence_after(); issue_qk(0); }
-  }
-
-  for (int t = t0; t < t1; ++t) {
-    const int it = t - t0;
-    cp_async_wait<1>();                            // K(t+1) has landed
-    fence_async_smem();
-    tc_fence_before();
-    if (__syncthreads_or(timed_out)) break;        // uniform exit if any thread gave up on a wait
-    if (is_mma_warp) {
-      if (lane == 0 && t + 1 < t1) { tc_fence_after(); issue_qk(it + 1); }   // overlaps softmax(t)
-    } else {
-      if (!mbar_wait(bar_s0 + (it & 1) * 8, (uint32_t)((it >> 1) & 1))) timed_out = 1;
-      tc_fence_after();
-      const int key0 = t * kBN;
-      const bool need_mask = key0 + kBN > L;
-      uint32_t pk[NB][16];
-      float alpha_new[NB][2];
-#pragma unroll
-      for (int rb = 0; rb < NB; ++rb) {
-        uint32_t sr[32];
-        tmem_ld_16x64(tmem_warp + ((uint32_t)(rb * 16) << 16) + kColS + (it & 1) * 64, sr);
-        tmem_wait_ld();
-        if (rb == NB - 1) {                        // K(t) is dead (its MMAs completed): refill the slot
-          if (t + 2 < t1) load_rows(kb, sK + (it & 1) * kTileBytes, t + 2);
-          cp_async_commit();
-        }
-        float mx0 = -INFINITY, mx1 = -INFINITY;
-        if (!need_mask) {
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float v0 = __uint_as_float(sr[4 * k]) * a.scale_log2, v1 = __uint_as_float(sr[4 * k + 1]) * a.scale_log2;
-            const float v2 = __uint_as_float(sr[4 * k + 2]) * a.scale_log2, v3 = __uint_as_float(sr[4 * k + 3]) * a.scale_log2;
-            sr[4 * k] = __float_as_uint(v0); sr[4 * k + 1] = __float_as_uint(v1);
-            sr[4 * k + 2] = __float_as_uint(v2); sr[4 * k + 3] = __float_as_uint(v3);
-            mx0 = fmaxf(mx0, fmaxf(v0, v1));
-            mx1 = fmaxf(mx1, fmaxf(v2, v3));
-          }
-        } else {
-          // 64-bit "key j of this tile is visible" masks of the thread's two rows: prefix keys,
-          // then the row's tree bits moved to where key L sits in this tile
-          unsigned long long am[2];
-          const int off = L - key0;                // position of key L in this tile (may be < 0)
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            unsigned long long pre = off >= 64 ? ~0ull : (off <= 0 ? 0ull : ((1ull << off) - 1ull));
-            unsigned long long tb;
-            if (off >= 64) tb = 0ull;
-            else if (off >= 0) tb = mlo[rb][hh] << off;
-            else if (off > -64) tb = (mlo[rb][hh] >> (-off)) | (mhi[rb][hh] << (64 + off));
-            else if (off > -128) tb = mhi[rb][hh] >> (-off - 64);
-            else tb = 0ull;
-            am[hh] = (pre | tb) >> (2 * t4);
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const bool ok = (am[e >> 1] >> (8 * k + (e & 1))) & 1ull;
-              const float v = ok ? __uint_as_float(sr[4 * k + e]) * a.scale_log2 : -INFINITY;
-              sr[4 * k + e] = __float_as_uint(v);
-            }
-            mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sr[4 * k]), __uint_as_float(sr[4 * k + 1])));
-            mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sr[4 * k + 2]), __uint_as_float(sr[4 * k + 3])));
-          }
-        }
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
-        const float mn0 = fmaxf(m_run[rb][0], mx0), mn1 = fmaxf(m_run[rb][1], mx1);
-        const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        alpha_new[rb][0] = ex2(m_run[rb][0] - ms0);  // m = -inf gives 0
-        alpha_new[rb][1] = ex2(m_run[rb][1] - ms1);
-        m_run[rb][0] = mn0; m_run[rb][1] = mn1;
-        float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const float e0 = ex2(__uint_as_float(sr[4 * k]) - ms0), e1 = ex2(__uint_as_float(sr[4 * k + 1]) - ms0);
-          const float e2 = ex2(__uint_as_float(sr[4 * k + 2]) - ms1), e3 = ex2(__uint_as_float(sr[4 * k + 3]) - ms1);
-          ps0 += e0 + e1;
-          ps1 += e2 + e3;
-          pk[rb][2 * k] = pack_bf16(e0, e1);
-          pk[rb][2 * k + 1] = pack_bf16(e2, e3);
-        }
-        l_run[rb][0] = l_run[rb][0] * alpha_new[rb][0] + ps0;
-        l_run[rb][1] = l_run[rb][1] * alpha_new[rb][1] + ps1;
-      }
-      // P V of the previous tile finished a while ago: fold it in (with the previous rescale),
-      // which also frees the P buffer, the O columns and the previous V slot.
-      if (it > 0) {
-        if (!mbar_wait(bar_o, (uint32_t)((it - 1) & 1))) timed_out = 1;
-        tc_fence_after();
-        fold_pv();
-      }
-      if (t + 1 < t1) load_rows(vb, sV + ((it + 1) & 1) * kTileBytes, t + 1);
-      cp_async_commit();
-#pragma unroll
-      for (int rb = 0; rb < NB; ++rb) {
-        alpha[rb][0] = alpha_new[rb][0]; alpha[rb][1] = alpha_new[rb][1];
-        // P (bf16) -> shared memory, K-major 128-byte-swizzled [64 rows x 64 keys]
-        const int rr0 = warp * 16 + g, rr1 = rr0 + 8;
-        const uint32_t p0 = sP + rb * kPBlockBytes + (rr0 >> 3) * 1024 + (rr0 & 7) * 128 + t4 * 4;
-        const uint32_t p1 = sP + rb * kPBlockBytes + (rr1 >> 3) * 1024 + (rr1 & 7) * 128 + t4 * 4;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          asm volatile("st.shared.b32 [%0], %1;" ::"r"(p0 + ((k ^ (rr0 & 7)) << 4)), "r"(pk[rb][2 * k]) : "memory");
-          asm volatile("st.shared.b32 [%0], %1;" ::"r"(p1 + ((k ^ (rr1 & 7)) << 4)), "r"(pk[rb][2 * k + 1]) : "memory");
-        }
-      }
-      cp_async_wait<2>();                          // V(t) has landed
-      fence_async_smem();
-      tc_fence_before();
-    }
-    if (__syncthreads_or(timed_out)) break;
-    if (is_mma_warp && lane == 0) {                // O = P V : 4 k-steps of 16 keys
-      tc_fence_after();
-      const int stage = it & 1;
-#pragma unroll
-      for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          umma_f16(tmem_base + ((uint32_t)(rb * 16) << 16) + kColO,
-                   dp0 + ((rb * kPBlockBytes + kk * 32) >> 4),
-                   dv0 + ((stage * kTileBytes + kk * 2048) >> 4), idesc_o, kk > 0);
-        }
-      }
-      umma_commit(bar_o);
-    }
-  }
-  if (!is_mma_warp && t0 < t1 && !timed_out) {     // the last tile's P V
-    if (!mbar_wait(bar_o, (uint32_t)((t1 - t0 - 1) & 1))) timed_out = 1;
-    tc_fence_after();
-    fold_pv();
-  }
-  cp_async_wait<0>();
-  tc_fence_before();
-  if (__syncthreads_or(timed_out) && tid == 0) atomicOr(&g_attn_error, 1u);
-  if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
-                 : "memory");
-  }
-
-#pragma unroll
-  for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      l_run[rb][hh] += __shfl_xor_sync(0xFFFFFFFFu, l_run[rb][hh], 1);
-      l_run[rb][hh] += __shfl_xor_sync(0xFFFFFFFFu, l_run[rb][hh], 2);
-    }
-  }
-
-  if (a.S == 1) {
-#pragma unroll
-    for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const int row = rb * 64 + warp * 16 + g + 8 * hh;
-        if (is_mma_warp || row >= Nl) continue;
-        const float l = l_run[rb][hh];
-        const float inv = l > 0.f ? 1.f / l : 0.f;
-        __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)(row0 + row) * a.o_n + h * a.o_h;
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          *reinterpret_cast<uint32_t*>(op + i * 8 + t4 * 2) =
-              pack_bf16(o[rb][i][2 * hh] * inv, o[rb][i][2 * hh + 1] * inv);
-        if (a.lse && t4 == 0)
-          a.lse[((int64_t)b * a.H + h) * N + row0 + row] = (m_run[rb][hh] + log2f(l)) * kLn2;
-      }
-    }
-    return;
-  }
-
-  // Merge across the cluster by pushing.  Rows [r*R, r*R + R) belong to block r.  A partial
-  // row is 132 floats: 128 of O, then (max, sum).  Each block stages its rows in its own
-  // shared memory and, once every block of the cluster is done with its operand tiles, sends
-  // each owner its rows with ONE bulk shared-to-shared copy that signals the owner's mbarrier
-  // (armed at start-up with the byte count it will receive).  Nobody waits on a remote round
-  // trip; the owner reduces its C slots locally as soon as its mbarrier completes.
-  const int C = a.C;
-  const int rank = split % C;
-  const int R = (Nl + C - 1) / C;
-  float* sStage = reinterpret_cast<float*>(smem);                    // [Nl][kOStride]
-  float* sRecv = sStage + (size_t)Nl * kOStride;                     // [C][R][kOStride]
-#pragma unroll
-  for (int rb = 0; rb < NB; ++rb) {
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int row = rb * 64 + warp * 16 + g + 8 * hh;
-      if (is_mma_warp || row >= Nl) continue;
-      float* ro = sStage + row * kOStride;
-#pragma unroll
-      for (int i = 0; i < 16; ++i)
-        *reinterpret_cast<float2*>(ro + i * 8 + t4 * 2) = make_float2(o[rb][i][2 * hh], o[rb][i][2 * hh + 1]);
-      if (t4 == 0) *reinterpret_cast<float2*>(ro + kD) = make_float2(m_run[rb][hh], l_run[rb][hh]);
-    }
-  }
-  fence_async_smem();                          // staged rows -> visible to the bulk-copy engine
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every block's tiles are dead
-  if (tid < C) {
-    const int owner = tid;
-    const int rows = max(0, min(R, Nl - owner * R));
-    if (rows > 0) {
-      const uint32_t src = smem_u32(sStage + (size_t)owner * R * kOStride);
-      const uint32_t dst_local = smem_u32(sRecv + (size_t)rank * R * kOStride);
-      uint32_t dst, rbar;
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(dst_local), "r"(owner));
-      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(bar_m), "r"(owner));
-      asm volatile(
-          "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-          ::"r"(dst), "r"(src), "r"((uint32_t)(rows * kOStride * 4)), "r"(rbar)
-          : "memory");
-    }
-  }
-  int merge_timeout = mbar_wait(bar_m, 0u) ? 0 : 1;
-
-  const int sup = split / C;
-  const int my_rows = max(0, min(R, Nl - rank * R));
-  for (int idx = tid; idx < my_rows * 32; idx += kTcThreads) {
-    const int lr = idx >> 5, mr = row0 + rank * R + lr, c4 = idx & 31;   // mr: global draft row
-    float2 ml[kMaxCluster];
-    float4 ov[kMaxCluster];
-#pragma unroll
-    for (int p = 0; p < kMaxCluster; ++p) {
-      if (p < C) {
-        const float* rr = sRecv + (size_t)(p * R + lr) * kOStride;
-        ml[p] = *reinterpret_cast<const float2*>(rr + kD);
-        ov[p] = *reinterpret_cast<const float4*>(rr + c4 * 4);
-      }
-    }
-    float M = -INFINITY;
-#pragma unroll
-    for (int p = 0; p < kMaxCluster; ++p)
-      if (p < C) M = fmaxf(M, ml[p].x);
-    float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    float lsum = 0.f;
-#pragma unroll
-    for (int p = 0; p < kMaxCluster; ++p) {
-      if (p < C) {
-        const float w = (ml[p].x == -INFINITY) ? 0.f : ex2(ml[p].x - M);
-        lsum += ml[p].y * w;
-        o4.x += ov[p].x * w; o4.y += ov[p].y * w; o4.z += ov[p].z * w; o4.w += ov[p].w * w;
-      }
-    }
-    if (a.Sp == 1) {
-      const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-      uint2 pk2;
-      pk2.x = pack_bf16(o4.x * inv, o4.y * inv);
-      pk2.y = pack_bf16(o4.z * inv, o4.w * inv);
-      *reinterpret_cast<uint2*>(a.out + b * a.o_b + (int64_t)mr * a.o_n + h * a.o_h + c4 * 4) = pk2;
-      if (a.lse && c4 == 0) a.lse[((int64_t)b * a.H + h) * N + mr] = (M + log2f(lsum)) * kLn2;
-    } else {
-      const int64_t base = ((((int64_t)b * a.H + h) * a.Sp + sup) * N + mr);
-      *reinterpret_cast<float4*>(a.ws_o + base * kD + c4 * 4) = o4;
-      if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
-    }
-  }
-  if (merge_timeout && tid == 0) atomicOr(&g_attn_error, 1u);
-  // stay until every peer has received what this block sent (its staged rows are the source)
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
 // =======================================================================================
-// Warp-specialised version of the tcgen05 kernel (the default).
-//
-// Same arithmetic, same shared-memory operand layout and same split merge as the kernel
-// above, but the three kinds of work run in their own warps and talk through mbarriers only;
-// there is no block-wide barrier inside the loop:
+// The kernel is warp-specialised: three kinds of work run in their own warps and talk through
+// mbarriers only; there is no block-wide barrier inside the loop:
 //   warp 4, one thread: TMA producer.  K and V tiles (and Q once) arrive as 64 x 64 boxes of
 //           a 4-D tensor map with 128-byte swizzle, which is exactly the operand layout; rows
 //           past the tensor's extent are zero-filled by the copy engine.  A slot is refilled
@@ -919,7 +175,8 @@ tree_attention_tc_kernel(AttnArgs a) {
 //   warps 0..3: softmax.  Wait for S(t), read it from TMEM, scale / mask / online softmax, fold
 //           P V(t-1) into the register accumulators, store P(t), signal the MMA warp.
 // Every wait is bounded; a wait that gives up raises a block-wide abort word that every other
-// wait polls, so all roles leave their loops and the block still frees its TMEM.
+// wait polls, so all roles leave their loops and the block still frees its TMEM; the host
+// reads the failure through rest_device_error_flags.
 // =======================================================================================
 constexpr int kWsThreads = 192;
 constexpr int kWsBarBytes = 192;
@@ -1497,27 +754,13 @@ bool encode_box_map(CUtensorMap* map, const void* base, int64_t rows, int64_t he
 
 struct SplitPlan { int S, C, Sp; };
 
-// Key splits per (context, head): enough blocks to fill the GPU once (never a partial second
-// wave), at most one split per tile, rounded down to a whole number of clusters.
-// REST_ATTENTION_IMPL selects an older kernel for comparison runs: "cp_async" = the tcgen05
-// kernel fed by cp.async, "mma_sync" = the mma.sync kernel.  Unset or anything else: the
-// warp-specialised tcgen05 + TMA kernel.
-int attention_impl() {
-  static const int v = [] {
-    const char* e = getenv("REST_ATTENTION_IMPL");
-    if (e && strcmp(e, "mma_sync") == 0) return 2;
-    if (e && strcmp(e, "cp_async") == 0) return 1;
-    return 0;
-  }();
-  return v;
-}
-bool use_tcgen05() { return attention_impl() != 2; }
-
+// Key splits per (context, head, row block): enough blocks to fill the GPU once (never a
+// partial second wave), at most one split per tile, rounded down to a whole number of clusters.
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
-  // the tcgen05 kernel gives every 64-row block of the draft rows its own thread blocks
-  const int64_t units = (int64_t)B * H * (use_tcgen05() ? (N + 63) / 64 : 1);
-  const int blocks_per_sm = (use_tcgen05() || N <= 64) ? 2 : 1;
+  // every 64-row block of the draft rows has its own thread blocks; two blocks fit an SM
+  const int64_t units = (int64_t)B * H * ((N + 63) / 64);
+  const int blocks_per_sm = 2;
   int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
   if (S > ntiles) S = ntiles;
   SplitPlan p;
@@ -1528,10 +771,6 @@ SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   if (p.S > 512) p.S = 512;
   p.Sp = p.S / p.C;
   return p;
-}
-
-size_t attn_smem_bytes(int N) {
-  return (size_t)N * kRowBytes + 2 * (size_t)kStages * kTileBytes + (size_t)N * 16;
 }
 
 }  // namespace
@@ -1592,22 +831,13 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
     a.ws_ml = a.ws_o + (size_t)B * H * a.Sp * N * kD;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int impl = attention_impl();
-  const bool tc = impl != 2;
-  a.NBLK = tc ? (N + 63) / 64 : 1;
-  const size_t smem = impl == 0 ? (size_t)ws_smem_bytes() : impl == 1 ? (size_t)tc_smem_bytes(1) : attn_smem_bytes(N);
-  if (impl == 0)
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 4, smem));
-  else if (impl == 1)
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_tc_kernel<1>),
-                                            3, smem));
-  else
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_kernel),
-                                            2, smem));
+  a.NBLK = (N + 63) / 64;
+  const size_t smem = (size_t)ws_smem_bytes();
+  REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 2, smem));
   if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(B * H * a.NBLK * a.S), 1, 1);
-  cfg.blockDim = dim3((unsigned)(impl == 0 ? kWsThreads : impl == 1 ? kTcThreads : (N / 16) * 32), 1, 1);
+  cfg.blockDim = dim3((unsigned)kWsThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -1615,26 +845,20 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   attr[0].val.clusterDim.x = (unsigned)a.C;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  // the warp-specialised kernel waits (griddepcontrol.wait) before its first global access, so it
-  // may be launched while the kernel before it in the stream is still draining
+  // the kernel waits (griddepcontrol.wait) before its first global access, so it may be
+  // launched while the kernel before it in the stream is still draining
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = impl == 0 ? 2 : 1;
-  if (impl == 0) {
-    // tensor maps: Q (d, N rows, H, B); K and V (d, max_kv rows, H_kv, B)
-    CUtensorMap tm_q, tm_k, tm_v;
-    int v_slot[3];
-    if (!encode_box_map(&tm_q, d_q, N, H, B, a.q_n, a.q_h, a.q_b, a.q_slot) ||
-        !encode_box_map(&tm_k, d_k, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, a.kv_slot) ||
-        !encode_box_map(&tm_v, d_v, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, v_slot))
-      return rest::note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, a, tm_q, tm_k, tm_v));
-  } else if (impl == 1) {
-    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<1>, a));
-  } else {
-    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_kernel, a));
-  }
+  cfg.numAttrs = 2;
+  // tensor maps: Q (d, N rows, H, B); K and V (d, max_kv rows, H_kv, B)
+  CUtensorMap tm_q, tm_k, tm_v;
+  int v_slot[3];
+  if (!encode_box_map(&tm_q, d_q, N, H, B, a.q_n, a.q_h, a.q_b, a.q_slot) ||
+      !encode_box_map(&tm_k, d_k, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, a.kv_slot) ||
+      !encode_box_map(&tm_v, d_v, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, v_slot))
+    return rest::note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+  REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, a, tm_q, tm_k, tm_v));
   rest::count_launch();
   if (a.Sp > 1) {
     const int64_t units = (int64_t)B * H * N;
