@@ -35,7 +35,7 @@ METRIC = "draft trees/s through retrieve+trie+mask, tree attention (all layers) 
 # dram__bytes_read.sum + dram__bytes_write.sum of one tree_attention_ws_kernel launch at the
 # single_stream attention shape, from the ncu capture summarised under profiles/ (the kernel has
 # not changed since); other shapes have no capture and report null.
-NCU_TRAFFIC_BYTES = {("single_stream", "tree_attention_ws_kernel"): 35_186_688}
+NCU_TRAFFIC_BYTES = {("single_stream", "tree_attention_ws_kernel"): 35_187_200}
 UNIT = "trees/s"
 N_CTX_POOL = 64          # distinct contexts rotated through the steps
 
@@ -386,20 +386,44 @@ def main():
         sum(t.numel() * 4 for t in h_acc) + sum(o.numel() * 2 for o in h_out)
     ctx_t, ver_t = torch.from_numpy(ctx_np), torch.from_numpy(ver_np)
 
+    # Two copy streams run beside the compute stream inside the graph: all inputs go in on one
+    # (layer l's attention waits only for its own queries), each layer's output goes out on the
+    # other as soon as that layer is done.
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
     def e2e_calls(_):
-        s_ctx.copy_(h_ctx, non_blocking=True)
-        s_ver.copy_(h_ver, non_blocking=True)
+        main = torch.cuda.current_stream()
+        s_in.wait_stream(main)
+        s_out.wait_stream(main)
+        q_ready = []
+        with torch.cuda.stream(s_in):
+            s_ctx.copy_(h_ctx, non_blocking=True)
+            s_ver.copy_(h_ver, non_blocking=True)
+            in_ready = torch.cuda.Event()
+            in_ready.record(s_in)
+            for layer in range(layers):
+                qs[layer].copy_(h_q[layer], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(s_in)
+                q_ready.append(ev)
+        main.wait_event(in_ready)
         rest.rest_draft(ds, s_ctx, d_ctx_len, out=tree, **dkw)
         for layer in range(layers):
-            qs[layer].copy_(h_q[layer], non_blocking=True)
+            main.wait_event(q_ready[layer])
             rest.rest_tree_attention(qs[layer], ks[layer], vs[layer], d_kv_len, tree.mask, scale,
                                      max_kv=L + N, out=outs[layer], workspace=ws)
-            h_out[layer].copy_(outs[layer], non_blocking=True)
+            done = torch.cuda.Event()
+            done.record(main)
+            s_out.wait_event(done)
+            with torch.cuda.stream(s_out):
+                h_out[layer].copy_(outs[layer], non_blocking=True)
         rest.rest_accept(tree.tokens, tree.parents, tree.n_nodes, s_ver, w.m, out=acc)
         for k, t in h_tree.items():
             t.copy_(getattr(tree, k), non_blocking=True)
         for hacc, dacc in zip(h_acc, acc):
             hacc.copy_(dacc, non_blocking=True)
+        main.wait_stream(s_in)
+        main.wait_stream(s_out)
 
     e2e_graph, _ = capture(e2e_calls, 0)
 
