@@ -666,6 +666,372 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// =======================================================================================
+// Wide variant for N > 64 draft rows: one thread block covers all (up to 128) rows.
+//
+// The tensor core needs the same time for an M = 64 and an M = 128 instruction, so two 64-row
+// blocks per head spend twice the tensor time per K/V byte and the tensor pipe, not HBM,
+// bounds N = 128.  Here S = Q K^T and O = P V are M = 128 instructions: accumulator row i lives
+// in TMEM lane i, softmax warp w owns lanes 32w .. 32w+31 and every thread owns one whole row
+// (no shuffles).  O stays in TMEM and accumulates across tiles; the running maximum used for the
+// exponentials is only raised when a tile's maximum exceeds it by more than 2^8, and only then
+// is the O row rescaled in TMEM (rare after the first tiles), so the per-tile work is
+// load S, mask, exp2, pack P.  Probabilities are at most 2^8, harmless in bf16 / fp32.
+// Splits write un-normalised partials to the caller's workspace; the combine kernel merges.
+// =======================================================================================
+constexpr int kWideQBytes = 128 * kRowBytes;            // 32 KB: 128 rows x 128 dims
+constexpr int kWidePBytes = 128 * 128;                  // 16 KB: 128 rows x 64 keys
+constexpr int kWideBarOffset = kWideQBytes + 2 * kTcStages * kTileBytes + kWidePBytes;   // 112 KB
+__host__ __device__ constexpr int wide_smem_bytes() { return kWideBarOffset + kWsBarBytes; }
+constexpr float kRescaleStep = 8.f;                     // log2 units
+
+// 32 TMEM lanes (one per thread) x 32 consecutive columns
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kWsThreads, 2)
+tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
+                           const __grid_constant__ CUtensorMap tm_k,
+                           const __grid_constant__ CUtensorMap tm_v) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const int N = a.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool is_softmax = warp < 4;
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t sQ = sbase;
+  const uint32_t sK = sQ + kWideQBytes;
+  const uint32_t sV = sK + kTcStages * kTileBytes;
+  const uint32_t sP = sV + kTcStages * kTileBytes;
+  const uint32_t bars = sbase + kWideBarOffset;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kWideBarOffset + kBarTmemSlot);
+  volatile uint32_t* abort_word = reinterpret_cast<volatile uint32_t*>(smem + kWideBarOffset + kBarAbort);
+
+  int bid = blockIdx.x;
+  const int split = bid % a.S; bid /= a.S;
+  const int h = bid % a.H;
+  const int b = bid / a.H;
+  const int hk = h / a.group;
+
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  if ((sbase & 1023u) != 0) {   // the swizzled operand layout needs a 1024-byte aligned base
+    if (tid == 0) atomicOr(&g_attn_error, 2u);
+    return;                     // uniform over the grid: every block sees the same offset
+  }
+
+  if (tid == 0) {
+    mbar_init(bars + kBarKFull, 1); mbar_init(bars + kBarKFull + 8, 1);
+    mbar_init(bars + kBarVFull, 1); mbar_init(bars + kBarVFull + 8, 1);
+    mbar_init(bars + kBarSFull, 1); mbar_init(bars + kBarSFull + 8, 1);
+    mbar_init(bars + kBarOFull, 1);
+    mbar_init(bars + kBarKFree, 1); mbar_init(bars + kBarKFree + 8, 1);
+    mbar_init(bars + kBarVFree, 1); mbar_init(bars + kBarVFree + 8, 1);
+    mbar_init(bars + kBarPFull, 4);            // one arrival per softmax warp
+    mbar_init(bars + kBarQFull, 1);
+    *abort_word = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // everything above is independent of the inputs; from here on global memory is read
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int L = a.kv_len[b];
+  const int total = L + N;
+  const int ntiles = (total + kBN - 1) / kBN;
+  const int t0 = tc_tile_begin(split, ntiles, a.S);
+  const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
+  const int nt = t1 - t0;
+
+  // softmax thread = draft row 32 warp + lane; its tree-mask row as two 64-bit halves
+  const int row = (warp & 3) * 32 + lane;
+  unsigned long long mlo = 0ull, mhi = 0ull;
+  if (is_softmax && row < N) {
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row) * a.Wm + i];
+    mlo = (unsigned long long)w[0] | ((unsigned long long)w[1] << 32);
+    mhi = (unsigned long long)w[2] | ((unsigned long long)w[3] << 32);
+  }
+  float m_used = -INFINITY, l_run = 0.f;
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_warp = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+
+  if (warp == 4) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(bars + kBarQFull, (uint32_t)kWideQBytes);
+      // two 64-dim halves, each [128 rows x 128 B]; rows past N are zero-filled
+      tma_load_box(sQ, &tm_q, 0, 0, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 64 * 128, &tm_q, 0, 64, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 128 * 128, &tm_q, 64, 0, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 192 * 128, &tm_q, 64, 64, h, b, a.q_slot, bars + kBarQFull);
+      int issued_k = 0, issued_v = 0;
+      for (int it = 0; it < nt; ++it) {
+        const int slot = it & 1, key0 = (t0 + it) * kBN;
+        const uint32_t free_parity = (uint32_t)(((it >> 1) + 1) & 1);
+        if (it >= 2 && !mbar_wait_abortable(bars + kBarKFree + slot * 8, free_parity, abort_word)) break;
+        mbar_expect_tx(bars + kBarKFull + slot * 8, (uint32_t)kTileBytes);
+        tma_load_box(sK + slot * kTileBytes, &tm_k, 0, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
+        tma_load_box(sK + slot * kTileBytes + 64 * 128, &tm_k, 64, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
+        ++issued_k;
+        if (it >= 2 && !mbar_wait_abortable(bars + kBarVFree + slot * 8, free_parity, abort_word)) break;
+        mbar_expect_tx(bars + kBarVFull + slot * 8, (uint32_t)kTileBytes);
+        tma_load_box(sV + slot * kTileBytes, &tm_v, 0, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
+        tma_load_box(sV + slot * kTileBytes + 64 * 128, &tm_v, 64, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
+        ++issued_v;
+      }
+      if (*abort_word != 0u) {
+        // giving up: let the copies already in flight land before this block goes away
+        mbar_wait(bars + kBarQFull, 0u);
+        for (int it = max(0, issued_k - 2); it < issued_k; ++it)
+          mbar_wait(bars + kBarKFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
+        for (int it = max(0, issued_v - 2); it < issued_v; ++it)
+          mbar_wait(bars + kBarVFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma_idesc(128, kBN, 0);
+      constexpr uint32_t idesc_o = umma_idesc(128, kD, 1);
+      const uint64_t dq0 = umma_desc(sQ, 16, 1024);
+      const uint64_t dk0 = umma_desc(sK, 16, 1024);
+      const uint64_t dp0 = umma_desc(sP, 16, 1024);
+      const uint64_t dv0 = umma_desc(sV, kBN * 128, 1024);
+      bool ok = mbar_wait_abortable(bars + kBarQFull, 0u, abort_word);
+      // S[it & 1] = Q K(it)^T; that buffer's previous reader signalled P(it - 2) after reading it
+      auto issue_qk = [&](int it) -> bool {
+        const int slot = it & 1;
+        if (!mbar_wait_abortable(bars + kBarKFull + slot * 8, (uint32_t)((it >> 1) & 1), abort_word)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t qoff = (uint32_t)((ks >> 2) * (128 * 128) + (ks & 3) * 32);
+          const uint32_t koff = (uint32_t)((ks >> 2) * (64 * 128) + (ks & 3) * 32);
+          umma_f16(tmem_base + kColS + slot * 64, dq0 + (qoff >> 4),
+                   dk0 + ((slot * kTileBytes + koff) >> 4), idesc_s, ks > 0);
+        }
+        umma_commit(bars + kBarSFull + slot * 8);
+        umma_commit(bars + kBarKFree + slot * 8);
+        return true;
+      };
+      if (ok && nt > 0) ok = issue_qk(0);
+      if (ok && nt > 1) ok = issue_qk(1);
+      for (int it = 0; ok && it < nt; ++it) {
+        const int slot = it & 1;
+        // P(it) is in shared memory, and O has been rescaled if this tile raised the maximum
+        if (!mbar_wait_abortable(bars + kBarPFull, (uint32_t)(it & 1), abort_word)) break;
+        if (!mbar_wait_abortable(bars + kBarVFull + slot * 8, (uint32_t)((it >> 1) & 1), abort_word)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          umma_f16(tmem_base + kColO, dp0 + ((kk * 32) >> 4),
+                   dv0 + ((slot * kTileBytes + kk * 2048) >> 4), idesc_o, (it > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bars + kBarOFull);
+        umma_commit(bars + kBarVFree + slot * 8);
+        if (it + 2 < nt) ok = issue_qk(it + 2);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax warps
+    // a wait's outcome is made warp-uniform, so the warp-wide TMEM instructions stay converged
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xFFFFFFFFu, mbar_wait_abortable(bar, parity, abort_word) ? 1 : 0) != 0;
+    };
+    bool ok = true;
+    for (int it = 0; it < nt; ++it) {
+      const int key0 = (t0 + it) * kBN;
+      if (!wait_all(bars + kBarSFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t s0[32], s1[32];
+      tmem_ld_32x32(tmem_warp + kColS + (it & 1) * 64, s0);
+      tmem_ld_32x32(tmem_warp + kColS + (it & 1) * 64 + 32, s1);
+      tmem_wait_ld();
+      float mx = -INFINITY;
+      if (key0 + kBN <= L) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float v0 = __uint_as_float(s0[j]) * a.scale_log2, v1 = __uint_as_float(s1[j]) * a.scale_log2;
+          s0[j] = __float_as_uint(v0); s1[j] = __float_as_uint(v1);
+          mx = fmaxf(mx, fmaxf(v0, v1));
+        }
+      } else {
+        // "key j of this tile is visible to this row": prefix keys, then the row's tree bits
+        // moved to where key L sits in this tile
+        const int off = L - key0;                // position of key L in this tile (may be < 0)
+        const unsigned long long pre = off >= 64 ? ~0ull : (off <= 0 ? 0ull : ((1ull << off) - 1ull));
+        unsigned long long tb;
+        if (off >= 64) tb = 0ull;
+        else if (off >= 0) tb = mlo << off;
+        else if (off > -64) tb = (mlo >> (-off)) | (mhi << (64 + off));
+        else if (off > -128) tb = mhi >> (-off - 64);
+        else tb = 0ull;
+        const unsigned long long vis = pre | tb;
+        const uint32_t vlo = (uint32_t)vis, vhi = (uint32_t)(vis >> 32);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float v0 = ((vlo >> j) & 1u) ? __uint_as_float(s0[j]) * a.scale_log2 : -INFINITY;
+          const float v1 = ((vhi >> j) & 1u) ? __uint_as_float(s1[j]) * a.scale_log2 : -INFINITY;
+          s0[j] = __float_as_uint(v0); s1[j] = __float_as_uint(v1);
+          mx = fmaxf(mx, fmaxf(v0, v1));
+        }
+      }
+      // raise the reference maximum only when this tile exceeds it by more than the step
+      bool o_done = it == 0;                      // "P V(it - 1) has completed" is known
+      if (__any_sync(0xFFFFFFFFu, mx > m_used + kRescaleStep)) {
+        const float m_new = fmaxf(m_used, mx);
+        const float alpha = (m_new == -INFINITY) ? 1.f : ex2(m_used - m_new);   // m_used = -inf gives 0
+        if (it > 0) {
+          if (!wait_all(bars + kBarOFull, (uint32_t)((it - 1) & 1))) { ok = false; break; }
+          tc_fence_after();
+          o_done = true;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t orr[32];
+            tmem_ld_32x32(tmem_warp + kColO + c * 32, orr);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) orr[j] = __float_as_uint(__uint_as_float(orr[j]) * alpha);
+            tmem_st_32x32(tmem_warp + kColO + c * 32, orr);
+          }
+          tmem_wait_st();
+        }
+        l_run *= alpha;
+        m_used = m_new;
+      }
+      const float ms = (m_used == -INFINITY) ? 0.f : m_used;
+      uint32_t pk[32];
+      float ps = 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float e0 = ex2(__uint_as_float(s0[2 * j]) - ms), e1 = ex2(__uint_as_float(s0[2 * j + 1]) - ms);
+        const float e2 = ex2(__uint_as_float(s1[2 * j]) - ms), e3 = ex2(__uint_as_float(s1[2 * j + 1]) - ms);
+        pk[j] = pack_bf16(e0, e1);
+        pk[16 + j] = pack_bf16(e2, e3);
+        // the sum takes the rounded probabilities, the ones P V uses: with a lazily raised
+        // maximum the largest probability is not exactly 1, and rounding it in the numerator
+        // only would show up in peaked rows
+        ps += (__uint_as_float(pk[j] << 16) + __uint_as_float(pk[j] & 0xFFFF0000u)) +
+              (__uint_as_float(pk[16 + j] << 16) + __uint_as_float(pk[16 + j] & 0xFFFF0000u));
+      }
+      l_run += ps;
+      // the single P buffer is free once P V(it - 1) has completed
+      if (!o_done && !wait_all(bars + kBarOFull, (uint32_t)((it - 1) & 1))) { ok = false; break; }
+      if (key0 + kBN > total) {
+        // Ragged last tile: rows of V past the last real key hold whatever the cache holds
+        // there.  Their probabilities are zero, but 0 x NaN is NaN: clear them.
+        if (!wait_all(bars + kBarVFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1))) { ok = false; break; }
+        const int first = total - key0;            // 0 < first < 64
+        for (int c = tid; c < (kBN - first) * 16; c += 128) {
+          const int vr = first + (c >> 4), chunk = c & 15;
+          const uint32_t dst = sV + (it & 1) * kTileBytes + (chunk >> 3) * (64 * 128) + (vr >> 3) * 1024 +
+                               (vr & 7) * 128 + (((chunk & 7) ^ (vr & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0u) : "memory");
+        }
+      }
+      {
+        // P row (64 bf16 = 8 chunks of 16 B) -> shared memory, K-major 128-byte-swizzled
+        const uint32_t prow = sP + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(prow + ((c ^ (row & 7)) << 4)), "r"(pk[4 * c]), "r"(pk[4 * c + 1]),
+                         "r"(pk[4 * c + 2]), "r"(pk[4 * c + 3])
+                       : "memory");
+      }
+      fence_async_smem();                          // P (and cleared V rows) -> visible to the tensor core
+      tc_fence_before();                           // this warp's TMEM accesses are done
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + kBarPFull);
+    }
+    // epilogue: O row out of TMEM
+    if (ok && nt > 0 && wait_all(bars + kBarOFull, (uint32_t)((nt - 1) & 1))) {
+      tc_fence_after();
+      const bool live = row < N;
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + row;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t orr[32];
+        __syncwarp();
+        tmem_ld_32x32(tmem_warp + kColO + c * 32, orr);
+        tmem_wait_ld();
+        if (live && a.S == 1) {
+          __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)row * a.o_n + h * a.o_h + c * 32;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 pv;
+            pv.x = pack_bf16(__uint_as_float(orr[8 * q4]) * inv, __uint_as_float(orr[8 * q4 + 1]) * inv);
+            pv.y = pack_bf16(__uint_as_float(orr[8 * q4 + 2]) * inv, __uint_as_float(orr[8 * q4 + 3]) * inv);
+            pv.z = pack_bf16(__uint_as_float(orr[8 * q4 + 4]) * inv, __uint_as_float(orr[8 * q4 + 5]) * inv);
+            pv.w = pack_bf16(__uint_as_float(orr[8 * q4 + 6]) * inv, __uint_as_float(orr[8 * q4 + 7]) * inv);
+            *reinterpret_cast<uint4*>(op + q4 * 8) = pv;
+          }
+        } else if (live) {
+          float* wp = a.ws_o + part * kD + c * 32;
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            *reinterpret_cast<uint4*>(wp + q4 * 4) =
+                make_uint4(orr[4 * q4], orr[4 * q4 + 1], orr[4 * q4 + 2], orr[4 * q4 + 3]);
+        }
+      }
+      if (live) {
+        if (a.S == 1) {
+          if (a.lse) a.lse[((int64_t)b * a.H + h) * N + row] = (m_used + log2f(l_run)) * kLn2;
+        } else {
+          a.ws_ml[part * 2] = m_used;
+          a.ws_ml[part * 2 + 1] = l_run;
+        }
+      }
+    } else if (ok && nt == 0 && a.S > 1 && row < N) {
+      // a split beyond this context's last tile: an empty partial the combine kernel skips
+      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + row;
+      a.ws_ml[part * 2] = -INFINITY;
+      a.ws_ml[part * 2 + 1] = 0.f;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_word != 0u && tid == 0) atomicOr(&g_attn_error, 1u);
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols)
+                 : "memory");
+  }
+}
+
 // Merges the per-split partials: one warp per (context, head, row), 4 output dims per lane.
 __global__ void __launch_bounds__(128)
 tree_attention_combine_kernel(AttnArgs a) {
@@ -756,8 +1122,19 @@ struct SplitPlan { int S, C, Sp; };
 
 // Key splits per (context, head, row block): enough blocks to fill the GPU once (never a
 // partial second wave), at most one split per tile, rounded down to a whole number of clusters.
+// N > 64 runs the wide kernel: one block per (context, head, split), no clusters, every split's
+// partial goes through the workspace.
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
+  if (N > 64) {
+    int64_t S = ((int64_t)kNumSMs * 2) / ((int64_t)B * H);
+    if (S > ntiles) S = ntiles;
+    if (S > 512) S = 512;
+    if (S < 1) S = 1;
+    SplitPlan p;
+    p.S = (int)S; p.C = 1; p.Sp = (int)S;
+    return p;
+  }
   // every 64-row block of the draft rows has its own thread blocks; two blocks fit an SM
   const int64_t units = (int64_t)B * H * ((N + 63) / 64);
   const int blocks_per_sm = 2;
@@ -831,9 +1208,13 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
     a.ws_ml = a.ws_o + (size_t)B * H * a.Sp * N * kD;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  a.NBLK = (N + 63) / 64;
-  const size_t smem = (size_t)ws_smem_bytes();
-  REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 2, smem));
+  const bool wide = N > 64;
+  a.NBLK = wide ? 1 : (N + 63) / 64;
+  const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
+  if (wide)
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_wide_kernel), 3, smem));
+  else
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 2, smem));
   if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(B * H * a.NBLK * a.S), 1, 1);
@@ -858,7 +1239,10 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
       !encode_box_map(&tm_k, d_k, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, a.kv_slot) ||
       !encode_box_map(&tm_v, d_v, max_kv, H_kv, B, a.kv_l, a.kv_h, a.kv_b, v_slot))
     return rest::note_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-  REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, a, tm_q, tm_k, tm_v));
+  if (wide)
+    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_wide_kernel, a, tm_q, tm_k, tm_v));
+  else
+    REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, a, tm_q, tm_k, tm_v));
   rest::count_launch();
   if (a.Sp > 1) {
     const int64_t units = (int64_t)B * H * N;
