@@ -53,6 +53,12 @@ def run_case(seed, B, H, N, L, Lcap=None, H_kv=None, kv_len=None, n_nodes=None, 
     (2, 3, 48, 200),         # N not a multiple of 32
     (1, 1, 64, 4096 + 17),   # many splits for one head
     (20, 16, 64, 513),       # enough units for a single split: direct output path
+    (40, 8, 128, 700),       # N = 128, one split per (context, head): direct output path
+    (2, 3, 96, 300),         # 64 < N < 128: rows past N are padding of the 128-row block
+    (1, 2, 80, 64),          # N = 80, prefix of exactly one tile
+    (1, 1, 128, 0),          # N = 128, no prefix: only tree keys
+    (1, 1, 128, 8192 + 5),   # N = 128, one head cut into many splits
+    (1, 3, 112, 130),
 ])
 def test_matches_fp64_oracle(B, H, N, L):
     run_case(7, B, H, N, L)
@@ -63,6 +69,37 @@ def test_ragged_batch_grouped_heads_padding_nodes_and_strides():
     # trees with unused slots, KV buffer longer than needed
     run_case(11, 4, 8, 64, 700, Lcap=900, H_kv=2, kv_len=[700, 1, 333, 64], n_nodes=41)
     run_case(12, 2, 6, 32, 90, H_kv=3, kv_len=[90, 31], n_nodes=1, scale=0.2)
+
+
+def test_wide_rows_ragged_batch_and_grouped_heads():
+    # N > 64 with contexts far shorter than the longest one: some key splits get no tile at all
+    run_case(13, 4, 8, 128, 900, Lcap=1100, H_kv=2, kv_len=[900, 1, 333, 64], n_nodes=77, max_depth=16)
+    run_case(14, 3, 6, 96, 200, H_kv=3, kv_len=[200, 31, 0], n_nodes=1, scale=0.2)
+
+
+@pytest.mark.parametrize("B,H,N,L", [(1, 2, 128, 1500), (30, 10, 128, 1500), (2, 2, 64, 1500)])
+def test_scores_whose_maximum_keeps_growing(B, H, N, L):
+    # Keys grow with their position, so the running maximum of every row rises again and again,
+    # tile after tile, by far more than any lazy-rescale threshold; every fifth tile jumps.
+    # Rows become so peaked that an output is nearly a single V row, with magnitudes up to 4-5,
+    # where rounding the output to bf16 alone costs up to 2^-8 |x| (0.0156 at 4): the absolute
+    # bound is therefore 1e-2 + 2^-8 |reference| here; the row-wise bound is unchanged.
+    D = 128
+    q, k, v = datagen.make_qkv(31, B, H, N, D, L + N)
+    pos = torch.arange(L + N, dtype=torch.float32)
+    factor = 1.0 + 7.0 * pos / (L + N)
+    factor[(pos.long() // 64) % 5 == 3] *= 2.5
+    k = (k.float() * factor[None, None, :, None]).to(torch.bfloat16)
+    masks = np.stack([datagen.make_random_tree(3100 + b, N, 12)[2] for b in range(B)])
+    kv_len = np.full(B, L, np.int32)
+    scale = 1.0 / math.sqrt(D)
+    ref = oracle.tree_attention(bits(q), bits(k), bits(v), kv_len, masks, scale)
+    out = rest.rest_tree_attention(q.cuda(), k.cuda(), v.cuda(), to_dev(kv_len), to_dev(masks), scale)
+    torch.cuda.synchronize()
+    err = np.abs(out.float().cpu().numpy().astype(np.float64) - ref)
+    assert (err <= MAX_ABS + np.abs(ref) / 256.0).all(), float((err - np.abs(ref) / 256.0).max())
+    _, max_rel = attention_errors(out, ref)
+    assert max_rel <= MAX_REL, max_rel
 
 
 def test_invariants_on_the_gpu_output():
