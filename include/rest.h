@@ -150,6 +150,7 @@ rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params
  *   d_mask    uint32[B,N,ceil(N/32)] as written by rest_draft
  *   d_lse     optional float[B,H,N]: log of the softmax denominator (natural log, of scaled scores)
  *   d_ws      scratch of rest_tree_attention_workspace_bytes() bytes
+ *   scale     softmax scale, finite and > 0 (else REST_INVALID_ARG)
  *   Limits: D = 128; N in {16, 32, 48, ..., 128}; H % H_kv == 0.
  */
 size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,

@@ -880,14 +880,13 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       tmem_ld_32x32(tmem_warp + kColS + (it & 1) * 64, s0);
       tmem_ld_32x32(tmem_warp + kColS + (it & 1) * 64 + 32, s1);
       tmem_wait_ld();
+      // maximum of the raw scores (the scale is positive, so it commutes with max); the scale
+      // is applied inside the exponent's multiply-add below
       float mx = -INFINITY;
       if (key0 + kBN <= L) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float v0 = __uint_as_float(s0[j]) * a.scale_log2, v1 = __uint_as_float(s1[j]) * a.scale_log2;
-          s0[j] = __float_as_uint(v0); s1[j] = __float_as_uint(v1);
-          mx = fmaxf(mx, fmaxf(v0, v1));
-        }
+        for (int j = 0; j < 32; ++j)
+          mx = fmaxf(mx, fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j])));
       } else {
         // "key j of this tile is visible to this row": prefix keys, then the row's tree bits
         // moved to where key L sits in this tile
@@ -903,12 +902,12 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
         const uint32_t vlo = (uint32_t)vis, vhi = (uint32_t)(vis >> 32);
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          const float v0 = ((vlo >> j) & 1u) ? __uint_as_float(s0[j]) * a.scale_log2 : -INFINITY;
-          const float v1 = ((vhi >> j) & 1u) ? __uint_as_float(s1[j]) * a.scale_log2 : -INFINITY;
-          s0[j] = __float_as_uint(v0); s1[j] = __float_as_uint(v1);
-          mx = fmaxf(mx, fmaxf(v0, v1));
+          if (!((vlo >> j) & 1u)) s0[j] = 0xFF800000u;   // -inf
+          if (!((vhi >> j) & 1u)) s1[j] = 0xFF800000u;
+          mx = fmaxf(mx, fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j])));
         }
       }
+      mx *= a.scale_log2;
       // raise the reference maximum only when this tile exceeds it by more than the step
       bool o_done = it == 0;                      // "P V(it - 1) has completed" is known
       if (__any_sync(0xFFFFFFFFu, mx > m_used + kRescaleStep)) {
@@ -937,8 +936,10 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       float ps = 0.f;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float e0 = ex2(__uint_as_float(s0[2 * j]) - ms), e1 = ex2(__uint_as_float(s0[2 * j + 1]) - ms);
-        const float e2 = ex2(__uint_as_float(s1[2 * j]) - ms), e3 = ex2(__uint_as_float(s1[2 * j + 1]) - ms);
+        const float e0 = ex2(fmaf(__uint_as_float(s0[2 * j]), a.scale_log2, -ms));
+        const float e1 = ex2(fmaf(__uint_as_float(s0[2 * j + 1]), a.scale_log2, -ms));
+        const float e2 = ex2(fmaf(__uint_as_float(s1[2 * j]), a.scale_log2, -ms));
+        const float e3 = ex2(fmaf(__uint_as_float(s1[2 * j + 1]), a.scale_log2, -ms));
         pk[j] = pack_bf16(e0, e1);
         pk[16 + j] = pack_bf16(e2, e3);
         // the sum takes the rounded probabilities, the ones P V uses: with a lazily raised
@@ -1178,6 +1179,7 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   if (B < 0 || H < 1 || H_kv < 1 || N < 1 || max_kv < 1 || !strides) return REST_INVALID_ARG;
   if (B == 0) return REST_OK;
   if (!d_q || !d_k || !d_v || !d_kv_len || !d_mask || !d_out) return REST_INVALID_ARG;
+  if (!(scale > 0.f) || !(scale < INFINITY)) return REST_INVALID_ARG;
   if (D != kD || N > REST_MAX_N || (N % 16) != 0 || (H % H_kv) != 0) return REST_UNSUPPORTED;
   for (int i = 0; i < 9; ++i)
     if (strides[i] < 0 || (strides[i] % 8) != 0) return REST_INVALID_ARG;
