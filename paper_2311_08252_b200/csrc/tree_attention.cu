@@ -711,6 +711,29 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
       : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// three-input maximum, and packed two-float multiply-add / add (one issue slot for two lanes)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ void fma2(float& x0, float& x1, float a0, float a1, float b, float c) {
+  asm("{ .reg .b64 ra, rb, rc, rd;\n\t"
+      "mov.b64 ra, {%2, %3};\n\t"
+      "mov.b64 rb, {%4, %4};\n\t"
+      "mov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+      "mov.b64 {%0, %1}, rd; }"
+      : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add2(float& acc0, float& acc1, float a0, float a1) {
+  asm("{ .reg .b64 ra, rb, rd;\n\t"
+      "mov.b64 ra, {%0, %1};\n\t"
+      "mov.b64 rb, {%2, %3};\n\t"
+      "add.rn.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd; }"
+      : "+f"(acc0), "+f"(acc1) : "f"(a0), "f"(a1));
+}
 
 __global__ void __launch_bounds__(kWsThreads, 2)
 tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
@@ -882,11 +905,11 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       tmem_wait_ld();
       // maximum of the raw scores (the scale is positive, so it commutes with max); the scale
       // is applied inside the exponent's multiply-add below
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // independent chains
       if (key0 + kBN <= L) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)
-          mx = fmaxf(mx, fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j])));
+          mx4[j & 3] = max3(mx4[j & 3], __uint_as_float(s0[j]), __uint_as_float(s1[j]));
       } else {
         // "key j of this tile is visible to this row": prefix keys, then the row's tree bits
         // moved to where key L sits in this tile
@@ -904,10 +927,10 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
         for (int j = 0; j < 32; ++j) {
           if (!((vlo >> j) & 1u)) s0[j] = 0xFF800000u;   // -inf
           if (!((vhi >> j) & 1u)) s1[j] = 0xFF800000u;
-          mx = fmaxf(mx, fmaxf(__uint_as_float(s0[j]), __uint_as_float(s1[j])));
+          mx4[j & 3] = max3(mx4[j & 3], __uint_as_float(s0[j]), __uint_as_float(s1[j]));
         }
       }
-      mx *= a.scale_log2;
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
       // raise the reference maximum only when this tile exceeds it by more than the step
       bool o_done = it == 0;                      // "P V(it - 1) has completed" is known
       if (__any_sync(0xFFFFFFFFu, mx > m_used + kRescaleStep)) {
@@ -933,22 +956,22 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       }
       const float ms = (m_used == -INFINITY) ? 0.f : m_used;
       uint32_t pk[32];
-      float ps = 0.f;
+      float ps[4] = {0.f, 0.f, 0.f, 0.f};
+      const float neg_ms = -ms;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const float e0 = ex2(fmaf(__uint_as_float(s0[2 * j]), a.scale_log2, -ms));
-        const float e1 = ex2(fmaf(__uint_as_float(s0[2 * j + 1]), a.scale_log2, -ms));
-        const float e2 = ex2(fmaf(__uint_as_float(s1[2 * j]), a.scale_log2, -ms));
-        const float e3 = ex2(fmaf(__uint_as_float(s1[2 * j + 1]), a.scale_log2, -ms));
-        pk[j] = pack_bf16(e0, e1);
-        pk[16 + j] = pack_bf16(e2, e3);
+        float x0, x1, x2, x3;
+        fma2(x0, x1, __uint_as_float(s0[2 * j]), __uint_as_float(s0[2 * j + 1]), a.scale_log2, neg_ms);
+        fma2(x2, x3, __uint_as_float(s1[2 * j]), __uint_as_float(s1[2 * j + 1]), a.scale_log2, neg_ms);
+        pk[j] = pack_bf16(ex2(x0), ex2(x1));
+        pk[16 + j] = pack_bf16(ex2(x2), ex2(x3));
         // the sum takes the rounded probabilities, the ones P V uses: with a lazily raised
         // maximum the largest probability is not exactly 1, and rounding it in the numerator
         // only would show up in peaked rows
-        ps += (__uint_as_float(pk[j] << 16) + __uint_as_float(pk[j] & 0xFFFF0000u)) +
-              (__uint_as_float(pk[16 + j] << 16) + __uint_as_float(pk[16 + j] & 0xFFFF0000u));
+        add2(ps[0], ps[1], __uint_as_float(pk[j] << 16), __uint_as_float(pk[j] & 0xFFFF0000u));
+        add2(ps[2], ps[3], __uint_as_float(pk[16 + j] << 16), __uint_as_float(pk[16 + j] & 0xFFFF0000u));
       }
-      l_run += ps;
+      l_run += (ps[0] + ps[1]) + (ps[2] + ps[3]);
       // the single P buffer is free once P V(it - 1) has completed
       if (!o_done && !wait_all(bars + kBarOFull, (uint32_t)((it - 1) & 1))) { ok = false; break; }
       if (key0 + kBN > total) {
