@@ -151,6 +151,16 @@ def draft_bytes(n_tokens, sa_bytes, n_min, n_max, Kp, m, N):
     return search + Kp * (sa_bytes + 4 * m) + N * (16 + N // 8)
 
 
+def draft_chain_reads(n_tokens, mean_candidates):
+    """Dependent global reads on the critical path of one draft: every 32-ary search round is a
+    suffix-array read followed by the token read it points to; lower bound over the whole array,
+    one galloping round plus the upper bound over the matched range, one gather round, and the
+    final token read of the emitted nodes."""
+    r_lower = math.ceil(math.log(max(n_tokens, 2)) / math.log(33))
+    r_upper = 1 + math.ceil(math.log(max(mean_candidates, 2)) / math.log(33))
+    return 2 * (r_lower + r_upper + 1) + 1
+
+
 def oracle_step_sample(w, T, sa, ctxs, q, k, v, kv_len, n_ctx, scale):
     """Times the CPU oracle on a bounded sample of one step: n_ctx drafts and accepts, and one
     attention layer (all heads).  Returns per-step seconds extrapolated to all layers."""
@@ -446,6 +456,8 @@ def main():
         return
 
     peak, peak_kind = measured_peaks()
+    read_ns = rest.dependent_read_latency_ns(device=dev)
+    chain = draft_chain_reads(w.n_tokens, kp_sum / (pool * B))
     a_bytes = attention_bytes(B, H, H, N, D, L)
     d_bytes = draft_bytes(w.n_tokens, w.sa_bytes, w.n_min, w.n_max, kp_sum / (pool * B), w.m, N) * B
     line = {
@@ -468,7 +480,10 @@ def main():
         "roofline_draft": {"kernel": "rest_draft_kernel", "bound": "hbm (latency-bound at B=1)",
                            "achieved": d_bytes / t_draft / 1e9, "peak": peak, "unit": "GB/s",
                            "frac": d_bytes / t_draft / 1e9 / peak,
-                           "algorithmic_bytes_per_launch": d_bytes},
+                           "algorithmic_bytes_per_launch": d_bytes,
+                           "dependent_read_ns": read_ns, "dependent_reads_on_critical_path": chain,
+                           "latency_floor_us": chain * read_ns / 1e3,
+                           "frac_of_latency_floor": chain * read_ns / 1e3 / (t_draft * 1e6)},
         "e2e": {"value": world * B / t_e2e, "unit": UNIT, "ms_per_step": t_e2e * 1e3,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),

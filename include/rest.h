@@ -238,6 +238,19 @@ rest_status rest_kv_commit(void* d_k, void* d_v, const int64_t* kv_strides, cons
                            int32_t* d_new_kv_len, void* stream);
 
 /*
+ * rest_probe_dependent_reads - measurement aid (the paper has no counterpart).
+ *
+ * One device thread follows `steps` dependent loads idx = d_next[idx] from `start` and writes
+ * d_out[0] = elapsed nanoseconds (device global timer), d_out[1] = the final index.  With a
+ * random cyclic table much larger than L2 this is the latency of one dependent DRAM read; the
+ * searches of Algorithm 1 are chains of such reads, so it bounds a single draft from below.
+ *   d_next  uint32[n] device table (entries >= n are treated as 0), n <= 2^32 - 1
+ *   d_out   uint64[2] device
+ */
+rest_status rest_probe_dependent_reads(const uint32_t* d_next, uint64_t n, uint32_t start,
+                                       uint32_t steps, uint64_t* d_out, void* stream);
+
+/*
  * Device-side trouble that no per-call status can carry.  Every wait inside the kernels is
  * bounded; a kernel that gives up sets a bit here instead of spinning, and its output is then
  * undefined.  Reads and clears the flags of the current device (synchronises the device).

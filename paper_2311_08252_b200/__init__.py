@@ -29,7 +29,7 @@ EXPORTS = (
     "rest_draft_workspace_bytes", "rest_draft",
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
     "rest_tree_attention_static_scratch",
-    "rest_device_error_flags", "rest_kv_commit",
+    "rest_device_error_flags", "rest_kv_commit", "rest_probe_dependent_reads",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -84,6 +84,8 @@ def lib():
     L.rest_accept.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     L.rest_kv_commit.restype = i32
     L.rest_kv_commit.argtypes = [vp, vp, ctypes.POINTER(i64), vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+    L.rest_probe_dependent_reads.restype = i32
+    L.rest_probe_dependent_reads.argtypes = [vp, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, vp, vp]
     L.rest_device_error_flags.restype = i32
     L.rest_device_error_flags.argtypes = [ctypes.POINTER(u32)]
     L.rest_status_string.restype = ctypes.c_char_p
@@ -323,3 +325,30 @@ def rest_kv_commit(k, v, kv_len, accept_nodes, accept_len, N, new_kv_len=None, s
                           _stream(stream))
     _check(rc, "rest_kv_commit")
     return new_kv_len
+
+
+def dependent_read_latency_ns(table_bytes: int = 1 << 30, steps: int = 4096, device=None, seed: int = 1) -> float:
+    """Nanoseconds per dependent DRAM read on this GPU: builds a random single-cycle table of
+    table_bytes (much larger than L2) with torch, then one device thread chases it
+    (rest_probe_dependent_reads).  A measurement aid for the draft path's latency floor."""
+    import torch
+    L = lib()
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    n = table_bytes // 4
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    perm = torch.randperm(n, generator=g, device=device)
+    nxt = torch.empty(n, dtype=torch.int32, device=device)
+    nxt[perm] = torch.roll(perm, -1).to(torch.int32)       # values < 2^31 for n <= 2^31
+    del perm
+    out = torch.zeros(2, dtype=torch.int64, device=device)
+    best = None
+    for rep in range(3):                                   # different stretches of the cycle
+        start = int(nxt[rep * 7919 % n].item())
+        torch.cuda.synchronize(device)
+        _check(L.rest_probe_dependent_reads(nxt.data_ptr(), n, start, steps, out.data_ptr(), _stream(None)),
+               "rest_probe_dependent_reads")
+        torch.cuda.synchronize(device)
+        ns = float(out[0].item()) / steps
+        best = ns if best is None else min(best, ns)
+    return best

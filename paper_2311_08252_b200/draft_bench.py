@@ -7,7 +7,9 @@ The datastore is the workload's recipe at --n-tokens tokens (host-built suffix a
 under the temp directory like bench.py does).  Contexts follow the workload's context recipe.
 Prints one JSON line per (workload, batch): microseconds per call, trees/s, the algorithmic
 bytes of the call (bisection probes for every suffix length + the candidate rows actually
-gathered + outputs) and the fraction of the measured HBM copy bandwidth they amount to.
+gathered + outputs), the fraction of the measured HBM copy bandwidth they amount to, and the
+latency floor of one call: the measured latency of a dependent DRAM read times the number of
+dependent reads on a draft's critical path (no call can finish faster, whatever the batch).
 """
 from __future__ import annotations
 
@@ -38,6 +40,7 @@ def main():
     args = ap.parse_args()
     peak, peak_kind = bench.measured_peaks()
     dev = torch.device("cuda:0")
+    read_ns = rest.dependent_read_latency_ns(device=dev)
     for name in args.workloads:
         w = datagen.WORKLOADS[name].scaled(n_tokens=min(args.n_tokens, datagen.WORKLOADS[name].n_tokens))
         T, sa, _ = bench.load_datastore(w)
@@ -70,7 +73,12 @@ def main():
                 "mean_candidates": kp_mean, "mean_nodes": float(out.n_nodes.float().mean().item()),
                 "us_per_call": us, "trees_per_s": B / us * 1e6, "algorithmic_bytes": alg,
                 "achieved_gbs": alg / us / 1e3, "peak_gbs": peak, "peak_kind": peak_kind,
-                "frac": alg / us / 1e3 / peak}), flush=True)
+                "frac": alg / us / 1e3 / peak,
+                "dependent_read_ns": read_ns,
+                "dependent_reads_on_critical_path": bench.draft_chain_reads(w.n_tokens, kp_mean),
+                "latency_floor_us": bench.draft_chain_reads(w.n_tokens, kp_mean) * read_ns / 1e3,
+                "frac_of_latency_floor": bench.draft_chain_reads(w.n_tokens, kp_mean) * read_ns / 1e3 / us}),
+                flush=True)
         ds.close()
         del ds
         torch.cuda.empty_cache()
