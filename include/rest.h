@@ -76,7 +76,7 @@ typedef struct {
  * Datastore (Sec. 3.2 "Datastore construction" and "Retrieving from the datastore": a token
  * stream whose every position is a (context, continuation) pair, indexed by a suffix array).
  *
- *   d_tokens   int32[n_tokens], values in [0, vocab), vocab < 2^31; 16-byte aligned
+ *   d_tokens   int32[n_tokens], values in [0, vocab), vocab < 2^31
  *   d_sa       int32[n_tokens] (sa_bytes = 4, n_tokens < 2^31) or int64[n_tokens] (sa_bytes = 8):
  *              start positions of all suffixes in lexicographic order of their tokens (compared
  *              as unsigned integers, a suffix that is a proper prefix of another sorts first).

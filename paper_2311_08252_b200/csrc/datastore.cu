@@ -88,8 +88,6 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
   if (!d_tokens || !d_sa || n_tokens == 0 || vocab == 0 || vocab >= 0x80000000u)
     return REST_INVALID_ARG;
   if (sa_bytes != 4 && sa_bytes != 8) return REST_INVALID_ARG;
-  // the draft kernel reads token rows as aligned 16-byte words
-  if (reinterpret_cast<uintptr_t>(d_tokens) & 15) return REST_INVALID_ARG;
   if (sa_bytes == 4 && n_tokens > 0x7FFFFFFFull) return REST_INVALID_ARG;
   if (n_tokens > (1ull << 40)) return REST_UNSUPPORTED;
   if (flags & REST_DS_VALIDATE) {

@@ -50,38 +50,6 @@ struct DraftArgs {
   int kcap;     // K rounded up to a multiple of 32
 };
 
-// tk[k] = T[p + k] for k < cnt (cnt <= MAXT, p + cnt <= n_tokens), read as aligned 16-byte
-// words: a row of 16 tokens costs at most five load instructions instead of sixteen (every lane
-// reads somewhere else, so each load instruction is 32 separate transactions whatever its width).
-// Entries at and beyond cnt are unspecified.  T is 16-byte aligned; the word that would reach
-// past the end of the stream is read token by token.
-template <int MAXT>
-__device__ __forceinline__ void load_tokens(const int32_t* __restrict__ T, int64_t n_tokens,
-                                            int64_t p, int cnt, int (&tk)[MAXT]) {
-  constexpr int NCH = (MAXT + 3) / 4 + 1;
-  const int off = (int)(p & 3);
-  const int64_t base = p - off;
-  int w[NCH * 4];
-#pragma unroll
-  for (int c = 0; c < NCH; ++c) {
-    const int64_t cb = base + 4 * c;
-    int4 v = make_int4(0, 0, 0, 0);
-    if (4 * c < off + cnt) {
-      if (cb + 4 <= n_tokens) {
-        v = __ldg(reinterpret_cast<const int4*>(T + cb));
-      } else {
-        if (cb < n_tokens) v.x = __ldg(T + cb);
-        if (cb + 1 < n_tokens) v.y = __ldg(T + cb + 1);
-        if (cb + 2 < n_tokens) v.z = __ldg(T + cb + 2);
-      }
-    }
-    w[4 * c] = v.x; w[4 * c + 1] = v.y; w[4 * c + 2] = v.z; w[4 * c + 3] = v.w;
-  }
-#pragma unroll
-  for (int k = 0; k < MAXT; ++k)
-    tk[k] = off == 0 ? w[k] : off == 1 ? w[k + 1] : off == 2 ? w[k + 2] : w[k + 3];
-}
-
 // Three-way comparison of the first n tokens of the suffix stored in slot `slot` with q.
 // -1 / 0 / +1; a suffix that ends early is smaller.  An out-of-range suffix-array entry
 // compares as smaller and raises `bad`.
@@ -92,8 +60,8 @@ __device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* _
   int64_t p = (int64_t)__ldg(sa + slot);
   if (p < 0 || p >= n_tokens) { bad = true; return -1; }
   int tk[16];
-  const int64_t rem = n_tokens - p;
-  load_tokens<16>(T, n_tokens, p, (int)(rem < n ? rem : n), tk);
+#pragma unroll
+  for (int k = 0; k < 16; ++k) tk[k] = (k < n && p + k < n_tokens) ? __ldg(T + p + k) : 0;
   int r = 0;
 #pragma unroll
   for (int k = 15; k >= 0; --k) {
@@ -346,9 +314,8 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       int64_t base = p + n_win;
       int64_t rem = n_tokens - base;
       len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
-      load_tokens<kMaxM>(T, n_tokens, base, len, row);
 #pragma unroll
-      for (int d = 0; d < kMaxM; ++d) row[d] = (d < len) ? row[d] : 0;
+      for (int d = 0; d < kMaxM; ++d) row[d] = (d < len) ? __ldg(T + base + d) : 0;
     } else {
 #pragma unroll
       for (int d = 0; d < kMaxM; ++d) row[d] = 0;
@@ -362,9 +329,8 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       int64_t base = p + n_win;
       int64_t rem = n_tokens - base;
       plen = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
-      load_tokens<kMaxM>(T, n_tokens, base, plen, prev);
 #pragma unroll
-      for (int d = 0; d < kMaxM; ++d) prev[d] = (d < plen) ? prev[d] : 0;
+      for (int d = 0; d < kMaxM; ++d) prev[d] = (d < plen) ? __ldg(T + base + d) : 0;
     }
     int lcp = 0;
     if (valid && j > 0) {
