@@ -54,7 +54,7 @@ enum { REST_DS_VALIDATE = 1u };
 enum {
   REST_MAX_SUFFIX = 16,   /* n_max */
   REST_MAX_M = 16,        /* continuation length */
-  REST_MAX_N = 128,       /* draft tokens per tree */
+  REST_MAX_N = 256,       /* draft tokens per tree */
   REST_MAX_K = 32768,     /* candidates per context */
   REST_HEAD_DIM = 128
 };
@@ -65,7 +65,7 @@ typedef struct rest_datastore rest_datastore;   /* opaque host object holding de
  *   n_max, n_min  longest / shortest context suffix tried by Algorithm 1 (1 <= n_min <= n_max <= 16)
  *   K             cap on the number of continuation candidates used per context (1..32768)
  *   m             continuation length (1..16)
- *   N             maximum number of draft tokens, the paper's c (1..128)
+ *   N             maximum number of draft tokens, the paper's c (1..256)
  *   sample_mode   which K of cnt > K matches are used: REST_SAMPLE_STRIDED takes suffix-array
  *                 slot lo + floor(j*cnt/K), REST_SAMPLE_FIRST_K takes lo + j, j = 0..K-1      */
 typedef struct {
@@ -151,7 +151,7 @@ rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params
  *   d_lse     optional float[B,H,N]: log of the softmax denominator (natural log, of scaled scores)
  *   d_ws      scratch of rest_tree_attention_workspace_bytes() bytes
  *   scale     softmax scale, finite and > 0 (else REST_INVALID_ARG)
- *   Limits: D = 128; N in {16, 32, 48, ..., 128}; H % H_kv == 0.
+ *   Limits: D = 128; N in {16, 32, 48, ..., 256}; H % H_kv == 0.
  */
 size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
                                            int32_t max_kv);

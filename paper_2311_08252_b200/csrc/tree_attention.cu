@@ -63,7 +63,7 @@ struct AttnArgs {
   int64_t q_b, q_n, q_h, kv_b, kv_h, kv_l, o_b, o_n, o_h;
   int B, H, group, N, Wm;
   int S;            // key splits per (context, head) = C * Sp
-  int NBLK;         // 64-row query blocks per (context, head): each gets its own thread blocks
+  int NBLK;         // 128-row query blocks per (context, head) in the wide kernel (else 1)
   int q_slot[3], kv_slot[3];   // tensor-map coordinate index (1..3) of rows, head, batch
   int C;            // blocks per cluster
   int Sp;           // clusters per (context, head); > 1 needs the merge kernel
@@ -667,7 +667,8 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
 }
 
 // =======================================================================================
-// Wide variant for N > 64 draft rows: one thread block covers all (up to 128) rows.
+// Wide variant for N > 64 draft rows: one thread block covers 128 rows (N <= 256: one or two
+// row blocks per head, adjacent in the grid so that they stream the same K/V tiles together).
 //
 // The tensor core needs the same time for an M = 64 and an M = 128 instruction, so two 64-row
 // blocks per head spend twice the tensor time per K/V byte and the tensor pipe, not HBM,
@@ -735,6 +736,16 @@ __device__ __forceinline__ void add2(float& acc0, float& acc1, float a0, float a
       : "+f"(acc0), "+f"(acc1) : "f"(a0), "f"(a1));
 }
 
+// bits [shift, shift + 64) of a 256-bit row mask, zero outside [0, 256)
+__device__ __forceinline__ unsigned long long mask_window(const unsigned long long (&m)[4], int shift) {
+  if (shift <= -64 || shift >= 256) return 0ull;
+  if (shift < 0) return m[0] << (-shift);
+  const int wi = shift >> 6, r = shift & 63;
+  const unsigned long long lo = wi == 0 ? m[0] : wi == 1 ? m[1] : wi == 2 ? m[2] : m[3];
+  const unsigned long long hi = wi == 0 ? m[1] : wi == 1 ? m[2] : wi == 2 ? m[3] : 0ull;
+  return r ? (lo >> r) | (hi << (64 - r)) : lo;
+}
+
 __global__ void __launch_bounds__(kWsThreads, 2)
 tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
                            const __grid_constant__ CUtensorMap tm_k,
@@ -742,7 +753,6 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   extern __shared__ __align__(1024) unsigned char smem[];
   const int N = a.N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const bool is_softmax = warp < 4;
   const uint32_t sbase = smem_u32(smem);
   const uint32_t sQ = sbase;
   const uint32_t sK = sQ + kWideQBytes;
@@ -754,9 +764,11 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
 
   int bid = blockIdx.x;
   const int split = bid % a.S; bid /= a.S;
+  const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 128-row block of the N draft rows
   const int h = bid % a.H;
   const int b = bid / a.H;
   const int hk = h / a.group;
+  const int row0 = rblk * 128;                       // first draft row of this thread block
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -793,17 +805,9 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   const int t1 = tc_tile_begin(split + 1, ntiles, a.S);
   const int nt = t1 - t0;
 
-  // softmax thread = draft row 32 warp + lane; its tree-mask row as two 64-bit halves
-  const int row = (warp & 3) * 32 + lane;
-  unsigned long long mlo = 0ull, mhi = 0ull;
-  if (is_softmax && row < N) {
-    uint32_t w[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-      if (i < a.Wm) w[i] = a.mask[((int64_t)b * N + row) * a.Wm + i];
-    mlo = (unsigned long long)w[0] | ((unsigned long long)w[1] << 32);
-    mhi = (unsigned long long)w[2] | ((unsigned long long)w[3] << 32);
-  }
+  // softmax thread = draft row row0 + 32 warp + lane
+  const int row = (warp & 3) * 32 + lane;            // row inside this block
+  const int grow = row0 + row;                       // draft row
   float m_used = -INFINITY, l_run = 0.f;
 
   tc_fence_before();
@@ -817,10 +821,10 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
     if (lane == 0) {
       mbar_expect_tx(bars + kBarQFull, (uint32_t)kWideQBytes);
       // two 64-dim halves, each [128 rows x 128 B]; rows past N are zero-filled
-      tma_load_box(sQ, &tm_q, 0, 0, h, b, a.q_slot, bars + kBarQFull);
-      tma_load_box(sQ + 64 * 128, &tm_q, 0, 64, h, b, a.q_slot, bars + kBarQFull);
-      tma_load_box(sQ + 128 * 128, &tm_q, 64, 0, h, b, a.q_slot, bars + kBarQFull);
-      tma_load_box(sQ + 192 * 128, &tm_q, 64, 64, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ, &tm_q, 0, row0, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 64 * 128, &tm_q, 0, row0 + 64, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 128 * 128, &tm_q, 64, row0, h, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 192 * 128, &tm_q, 64, row0 + 64, h, b, a.q_slot, bars + kBarQFull);
       int issued_k = 0, issued_v = 0;
       for (int it = 0; it < nt; ++it) {
         const int slot = it & 1, key0 = (t0 + it) * kBN;
@@ -915,13 +919,19 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
         // moved to where key L sits in this tile
         const int off = L - key0;                // position of key L in this tile (may be < 0)
         const unsigned long long pre = off >= 64 ? ~0ull : (off <= 0 ? 0ull : ((1ull << off) - 1ull));
-        unsigned long long tb;
-        if (off >= 64) tb = 0ull;
-        else if (off >= 0) tb = mlo << off;
-        else if (off > -64) tb = (mlo >> (-off)) | (mhi << (64 + off));
-        else if (off > -128) tb = mhi >> (-off - 64);
-        else tb = 0ull;
-        const unsigned long long vis = pre | tb;
+        // the row's tree mask (up to 256 bits) is only needed here, in the last few tiles of a
+        // context: read it from global memory (cached) rather than hold it in registers
+        unsigned long long mrow[4] = {0ull, 0ull, 0ull, 0ull};
+        if (grow < N) {
+          const uint32_t* mp = a.mask + ((int64_t)b * N + grow) * a.Wm;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t w0 = 2 * i < a.Wm ? __ldg(mp + 2 * i) : 0u;
+            const uint32_t w1 = 2 * i + 1 < a.Wm ? __ldg(mp + 2 * i + 1) : 0u;
+            mrow[i] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);
+          }
+        }
+        const unsigned long long vis = pre | mask_window(mrow, -off);
         const uint32_t vlo = (uint32_t)vis, vhi = (uint32_t)(vis >> 32);
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
@@ -1004,9 +1014,9 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
     // epilogue: O row out of TMEM
     if (ok && nt > 0 && wait_all(bars + kBarOFull, (uint32_t)((nt - 1) & 1))) {
       tc_fence_after();
-      const bool live = row < N;
+      const bool live = grow < N;
       const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + row;
+      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + grow;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t orr[32];
@@ -1014,7 +1024,7 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
         tmem_ld_32x32(tmem_warp + kColO + c * 32, orr);
         tmem_wait_ld();
         if (live && a.S == 1) {
-          __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)row * a.o_n + h * a.o_h + c * 32;
+          __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)grow * a.o_n + h * a.o_h + c * 32;
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             uint4 pv;
@@ -1034,15 +1044,15 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       }
       if (live) {
         if (a.S == 1) {
-          if (a.lse) a.lse[((int64_t)b * a.H + h) * N + row] = (m_used + log2f(l_run)) * kLn2;
+          if (a.lse) a.lse[((int64_t)b * a.H + h) * N + grow] = (m_used + log2f(l_run)) * kLn2;
         } else {
           a.ws_ml[part * 2] = m_used;
           a.ws_ml[part * 2 + 1] = l_run;
         }
       }
-    } else if (ok && nt == 0 && a.S > 1 && row < N) {
+    } else if (ok && nt == 0 && a.S > 1 && grow < N) {
       // a split beyond this context's last tile: an empty partial the combine kernel skips
-      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + row;
+      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + grow;
       a.ws_ml[part * 2] = -INFINITY;
       a.ws_ml[part * 2 + 1] = 0.f;
     }
@@ -1151,7 +1161,7 @@ struct SplitPlan { int S, C, Sp; };
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
   if (N > 64) {
-    int64_t S = ((int64_t)kNumSMs * 2) / ((int64_t)B * H);
+    int64_t S = ((int64_t)kNumSMs * 2) / ((int64_t)B * H * ((N + 127) / 128));
     if (S > ntiles) S = ntiles;
     if (S > 512) S = 512;
     if (S < 1) S = 1;
@@ -1234,7 +1244,7 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool wide = N > 64;
-  a.NBLK = wide ? 1 : (N + 63) / 64;
+  a.NBLK = wide ? (N + 127) / 128 : 1;
   const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
   if (wide)
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_wide_kernel), 3, smem));

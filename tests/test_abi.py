@@ -57,7 +57,7 @@ def test_host_argument_checks_return_status_codes():
     assert L.rest_draft(h, ctypes.byref(bad), *args) == 2
     bad = rest._Params(16, 2, 5000, 17, 64, 0)
     assert L.rest_draft(h, ctypes.byref(bad), *args) == 2
-    bad = rest._Params(16, 2, 5000, 10, 129, 0)
+    bad = rest._Params(16, 2, 5000, 10, 257, 0)
     assert L.rest_draft(h, ctypes.byref(bad), *args) == 2
     bad = rest._Params(16, 0, 5000, 10, 64, 0)
     assert L.rest_draft(h, ctypes.byref(bad), *args) == 1
@@ -70,6 +70,9 @@ def test_host_argument_checks_return_status_codes():
     assert att(64, 64, 4, 4) == 2
     assert att(40, 128, 4, 4) == 2
     assert att(64, 128, 4, 3) == 2
+    assert att(272, 128, 4, 4) == 2
+    assert L.rest_tree_attention(256, 256, 256, strides, 256, 256, 1, 4, 4, 64, 128, 512, 0.0, 256,
+                                 None, None, 0, None) == 1       # the softmax scale must be positive
     assert L.rest_tree_attention(256, 256, 256, strides, 256, 256, 1, 2, 2, 64, 128, 8256, 1.0, 256,
                                  None, None, 0, None) == 1       # needs a workspace, none given
     odd = (ctypes.c_int64 * 9)(*([124] * 9))

@@ -18,7 +18,7 @@ def gpu_accept(tokens, parents, n_nodes, ver, max_depth):
     return [o.cpu().numpy() for o in out]
 
 
-@pytest.mark.parametrize("name,N", [("tiny", 64), ("stress", 128)])
+@pytest.mark.parametrize("name,N", [("tiny", 64), ("stress", 128), ("stress", 256)])
 def test_accept_matches_oracle_on_drafted_trees(name, N):
     w = datagen.WORKLOADS[name].scaled(n_tokens=500_000)
     T = datagen.make_tokens(w)

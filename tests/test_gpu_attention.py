@@ -59,6 +59,11 @@ def run_case(seed, B, H, N, L, Lcap=None, H_kv=None, kv_len=None, n_nodes=None, 
     (1, 1, 128, 0),          # N = 128, no prefix: only tree keys
     (1, 1, 128, 8192 + 5),   # N = 128, one head cut into many splits
     (1, 3, 112, 130),
+    (2, 3, 256, 500),        # N = 256: two 128-row blocks per head
+    (1, 2, 192, 100),        # second row block half empty
+    (1, 1, 144, 0),          # N = 144, no prefix
+    (1, 1, 256, 4096 + 9),   # N = 256, many splits
+    (24, 8, 256, 700),       # N = 256, one split: direct output path
 ])
 def test_matches_fp64_oracle(B, H, N, L):
     run_case(7, B, H, N, L)
@@ -75,6 +80,7 @@ def test_wide_rows_ragged_batch_and_grouped_heads():
     # N > 64 with contexts far shorter than the longest one: some key splits get no tile at all
     run_case(13, 4, 8, 128, 900, Lcap=1100, H_kv=2, kv_len=[900, 1, 333, 64], n_nodes=77, max_depth=16)
     run_case(14, 3, 6, 96, 200, H_kv=3, kv_len=[200, 31, 0], n_nodes=1, scale=0.2)
+    run_case(15, 3, 4, 256, 600, Lcap=900, H_kv=2, kv_len=[600, 2, 129], n_nodes=201, max_depth=16)
 
 
 @pytest.mark.parametrize("B,H,N,L", [(1, 2, 128, 1500), (30, 10, 128, 1500), (2, 2, 64, 1500)])

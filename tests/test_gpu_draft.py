@@ -31,6 +31,8 @@ def test_worked_example():
     (6, 8, 4096, 5000, 10, 64, 4),
     (7, 2, 40000, 20000, 16, 128, 4),   # stress shape: K = 20000, m = 16
     (8, 3, 70000, 32768, 1, 1, 4),      # extremes: K max, m = 1, N = 1
+    (9, 3, 30000, 20000, 16, 256, 4),   # N = 256: the largest tree
+    (10, 4, 9000, 5000, 12, 200, 8),    # N = 200, not a multiple of 32
 ])
 def test_small_alphabets_match_oracle(seed, vocab, n_tok, K, m, N, sa_bytes):
     rng = np.random.default_rng(seed)
@@ -66,6 +68,21 @@ def test_workload_recipes_match_oracle(name, n_tok, B):
     got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, **kw)
     assert_draft_equal(got, ref, name)
     assert (ref["n_nodes"] > 0).sum() > B // 2
+
+
+def test_largest_trees_on_the_stress_recipe():
+    w = datagen.WORKLOADS["stress"].scaled(n_tokens=2_000_000)
+    T = datagen.make_tokens(w)
+    sa = datagen.build_suffix_array(T, w.vocab)
+    B = 96
+    ctx = datagen.make_contexts(w, T, B=B, Lc=64)
+    ctx_len = np.full(B, 64, np.int32)
+    for N in (256, 176):
+        kw = dict(K=w.K, m=w.m, N=N)
+        ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+        assert_draft_equal(got, ref, f"N={N}")
+        assert ref["n_nodes"].max() > 128
 
 
 def test_other_suffix_limits_and_repeatability():

@@ -69,3 +69,25 @@ def test_draft_full_single_stream_datastore():
     got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, K=w.K, m=w.m, N=w.N)
     assert_draft_equal(got, ref, "single_stream, 100 M tokens")
     assert (ref["n_nodes"] > 0).mean() > 0.5
+
+
+@pytest.mark.parametrize("name,n_tokens", [("stress", 500_000_000), ("batched", 1_000_000_000),
+                                           ("large", 1_000_000_000)])
+def test_draft_largest_datastores(name, n_tokens):
+    """The 500 M-token stress datastore, the 1 B-token batched one, and the large recipe with its
+    int64 suffix array at 1 B tokens (the 4 B-token array cannot be built in this host's memory).
+    Building these suffix arrays on the host takes minutes, so the test only runs when
+    REST_FULL_DATASTORES=1."""
+    import os
+    if os.environ.get("REST_FULL_DATASTORES") != "1":
+        pytest.skip("set REST_FULL_DATASTORES=1 to build the 0.5-1 B-token suffix arrays")
+    w = datagen.WORKLOADS[name].scaled(n_tokens=n_tokens)
+    T = datagen.make_tokens(w)
+    sa = datagen.build_suffix_array(T, w.vocab, sa_bytes=w.sa_bytes)
+    B, Lc = w.B, 64
+    ctx = datagen.make_contexts(w, T, B=B, Lc=Lc)
+    ctx_len = np.full(B, Lc, np.int32)
+    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, K=w.K, m=w.m, N=w.N)
+    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, K=w.K, m=w.m, N=w.N)
+    assert_draft_equal(got, ref, f"{name}, {n_tokens} tokens")
+    assert (ref["n_nodes"] > 0).mean() > 0.5
