@@ -151,6 +151,16 @@ def draft_bytes(n_tokens, sa_bytes, n_min, n_max, Kp, m, N):
     return search + Kp * (sa_bytes + 4 * m) + N * (16 + N // 8)
 
 
+def draft_sector_bytes(n_tokens, sa_bytes, n_min, n_max, Kp, m, N):
+    """The same accesses counted in whole 32-byte DRAM sectors: a suffix-array entry costs one
+    sector, a row of k tokens at an arbitrary 4-byte offset touches ceil((4k + 28) / 32) of
+    them.  DRAM counters of the draft kernel sit near this figure, not near the useful bytes."""
+    lg = math.ceil(math.log2(max(n_tokens, 2)))
+    row = lambda k: 32 * math.ceil((4 * k + 28) / 32)
+    search = sum(2 * lg * (32 + row(n)) for n in range(n_min, n_max + 1))
+    return search + Kp * (32 + row(m)) + 32 * math.ceil(N * (16 + N // 8) / 32)
+
+
 def draft_chain_reads(n_tokens, mean_candidates):
     """Dependent global reads on the critical path of one draft: every 32-ary search round is a
     suffix-array read followed by the token read it points to; lower bound over the whole array,
@@ -481,6 +491,8 @@ def main():
                            "achieved": d_bytes / t_draft / 1e9, "peak": peak, "unit": "GB/s",
                            "frac": d_bytes / t_draft / 1e9 / peak,
                            "algorithmic_bytes_per_launch": d_bytes,
+                           "sector_granular_bytes_per_launch": draft_sector_bytes(
+                               w.n_tokens, w.sa_bytes, w.n_min, w.n_max, kp_sum / (pool * B), w.m, N) * B,
                            "dependent_read_ns": read_ns, "dependent_reads_on_critical_path": chain,
                            "latency_floor_us": chain * read_ns / 1e3,
                            "frac_of_latency_floor": chain * read_ns / 1e3 / (t_draft * 1e6)},
