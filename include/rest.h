@@ -238,6 +238,25 @@ rest_status rest_kv_commit(void* d_k, void* d_v, const int64_t* kv_strides, cons
                            int32_t* d_new_kv_len, void* stream);
 
 /*
+ * rest_suffix_array_build - the datastore's suffix array, built on the device (Sec. 3.2
+ * "Datastore construction"; "Retrieving from the datastore" matches through a suffix array).
+ * Set-up work: call it once, then rest_datastore_create on the result.
+ *
+ *   Order: suffixes compare on their first 32 tokens (unsigned, a suffix that ends early is
+ *   smaller); suffixes equal on those are ordered by position.  rest_draft reads at most
+ *   n_max + m <= 32 tokens of a suffix, so its results are those of the full order.
+ *
+ *   d_tokens  int32[n_tokens] device, values in [0, 2^31 - 1)
+ *   sa_bytes  4 or 8: d_sa is int32[n_tokens] or int64[n_tokens] (device, written)
+ *   d_ws      device scratch of rest_suffix_array_workspace_bytes(n_tokens) bytes (about
+ *             32 bytes per token + 64 MiB), 256-byte aligned
+ *   Limits: n_tokens <= 2^31 - 1 (REST_UNSUPPORTED beyond).  Asynchronous on `stream`.
+ */
+size_t rest_suffix_array_workspace_bytes(uint64_t n_tokens);
+rest_status rest_suffix_array_build(const int32_t* d_tokens, uint64_t n_tokens, int32_t sa_bytes,
+                                    void* d_sa, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
  * rest_probe_dependent_reads - measurement aid (the paper has no counterpart).
  *
  * One device thread follows `steps` dependent loads idx = d_next[idx] from `start` and writes

@@ -1,0 +1,73 @@
+"""rest_suffix_array_build against the oracle's comparison sort (where the 32-token order is the
+full order), against the order's definition checked entry by entry, and through rest_draft."""
+import numpy as np
+import pytest
+import torch
+
+import datagen
+import oracle
+import paper_2311_08252_b200 as rest
+from gpu_util import assert_draft_equal, gpu_draft, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_sa(T, sa_bytes=4):
+    sa = rest.rest_suffix_array_build(to_dev(np.asarray(T, np.int32)), sa_bytes=sa_bytes)
+    torch.cuda.synchronize()
+    return sa.cpu().numpy()
+
+
+def bounded_order_reference(T, W=32):
+    """The order's definition, by brute force: sort positions by (first W tokens, padded with -1
+    past the end, then position)."""
+    n = len(T)
+    keys = [(tuple(int(x) for x in T[p:p + W]) , p) for p in range(n)]
+    # a suffix that ends early is smaller: tuple comparison already puts a proper prefix first
+    return np.array([p for _, p in sorted(keys)], np.int64)
+
+
+@pytest.mark.parametrize("seed,vocab,n", [(1, 32000, 5000), (2, 50, 20000), (3, 2**31 - 2, 3000)])
+def test_equals_the_full_suffix_order_when_no_two_suffixes_share_32_tokens(seed, vocab, n):
+    rng = np.random.default_rng(seed)
+    T = rng.integers(0, vocab, n).astype(np.int32)
+    T[-1] = vocab - 1
+    want = oracle.suffix_array(T)
+    assert np.array_equal(gpu_sa(T), want)
+    assert np.array_equal(gpu_sa(T, 8), want.astype(np.int64))
+
+
+@pytest.mark.parametrize("name", ["binary", "constant", "period3", "two_runs", "single", "pair"])
+def test_repetitive_streams_follow_the_bounded_order(name):
+    rng = np.random.default_rng(5)
+    T = {"binary": rng.integers(0, 2, 3000), "constant": np.full(500, 7),
+         "period3": np.tile([4, 1, 9], 400), "two_runs": np.r_[np.full(300, 3), np.full(300, 2)],
+         "single": np.array([11]), "pair": np.array([5, 5])}[name].astype(np.int32)
+    got = gpu_sa(T)
+    assert np.array_equal(got, bounded_order_reference(T))
+    assert got.dtype == np.int32
+
+
+@pytest.mark.parametrize("name", ["single_stream", "stress", "large"])
+def test_workload_recipes_and_drafts_on_the_device_built_array(name):
+    w = datagen.WORKLOADS[name].scaled(n_tokens=1_500_000)
+    T = datagen.make_tokens(w)
+    sa = gpu_sa(T, w.sa_bytes)
+    assert datagen.verify_suffix_array(T, sa, W=32) == 0          # permutation, ordered, ties by position
+    B = 64
+    ctx = datagen.make_contexts(w, T, B=B, Lc=64)
+    ctx_len = np.full(B, 64, np.int32)
+    kw = dict(K=w.K, m=w.m, N=w.N)
+    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, **kw)
+    assert_draft_equal(got, ref, name)
+    assert (ref["n_nodes"] > 0).mean() > 0.5
+
+
+def test_argument_checks():
+    L = rest.lib()
+    assert L.rest_suffix_array_workspace_bytes(0) == 0
+    assert L.rest_suffix_array_workspace_bytes(1 << 31) == 0
+    assert L.rest_suffix_array_build(256, 10, 5, 256, 256, 1 << 30, None) == 1
+    assert L.rest_suffix_array_build(256, 10, 4, 256, 256, 16, None) == 3
+    assert L.rest_suffix_array_build(256, 1 << 31, 4, 256, 256, 1 << 30, None) == 2
