@@ -262,21 +262,12 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     # ---- inputs (setup, untimed) -------------------------------------------------------
-    if world > 1:
-        if rank == 0:
-            T, sa, _ = load_datastore(w)
-            d_T, d_sa = torch.from_numpy(T).to(dev), torch.from_numpy(sa).to(dev)
-        else:
-            d_T = torch.empty(w.n_tokens, dtype=torch.int32, device=dev)
-            d_sa = torch.empty(w.n_tokens, dtype=torch.int32 if w.sa_bytes == 4 else torch.int64,
-                               device=dev)
-        dist.broadcast(d_T, 0)
-        dist.broadcast(d_sa, 0)
-        T = d_T.cpu().numpy() if rank != 0 else T
-        sa = None if rank != 0 else sa
-    else:
-        T, sa, _ = load_datastore(w)
-        d_T, d_sa = torch.from_numpy(T).to(dev), torch.from_numpy(sa).to(dev)
+    # every rank generates the same seeded token stream and builds its own copy of the suffix
+    # array on its GPU (the datastore is replicated; nothing is exchanged)
+    T = datagen.make_tokens(w)
+    d_T = torch.from_numpy(T).to(dev)
+    d_sa = rest.rest_suffix_array_build(d_T, w.sa_bytes)
+    sa = None
     ds = rest.Datastore(d_T, d_sa, w.vocab, validate=True)
 
     B, N, H, D, L, layers = w.B, w.N, w.H, w.D, w.L, w.layers

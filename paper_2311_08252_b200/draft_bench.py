@@ -3,8 +3,8 @@
     python -m paper_2311_08252_b200.draft_bench [--workloads single_stream stress]
                                                 [--n-tokens 100000000] [--batches 1 256 4096]
 
-The datastore is the workload's recipe at --n-tokens tokens (host-built suffix array, cached
-under the temp directory like bench.py does).  Contexts follow the workload's context recipe.
+The datastore is the workload's recipe at --n-tokens tokens; its suffix array is built on the
+device (rest_suffix_array_build).  Contexts follow the workload's context recipe.
 Prints one JSON line per (workload, batch): microseconds per call, trees/s, the algorithmic
 bytes of the call (bisection probes for every suffix length + the candidate rows actually
 gathered + outputs), the fraction of the measured HBM copy bandwidth they amount to, and the
@@ -43,8 +43,10 @@ def main():
     read_ns = rest.dependent_read_latency_ns(device=dev)
     for name in args.workloads:
         w = datagen.WORKLOADS[name].scaled(n_tokens=min(args.n_tokens, datagen.WORKLOADS[name].n_tokens))
-        T, sa, _ = bench.load_datastore(w)
-        ds = rest.Datastore(torch.from_numpy(T).to(dev), torch.from_numpy(sa).to(dev), w.vocab)
+        T = datagen.make_tokens(w)
+        d_T = torch.from_numpy(T).to(dev)
+        d_sa = rest.rest_suffix_array_build(d_T, w.sa_bytes)
+        ds = rest.Datastore(d_T, d_sa, w.vocab)
         Lc = min(w.Lc, 64)                       # only the last n_max tokens are ever read
         for B in args.batches:
             nsets = 4                            # rotate context sets so probes differ call to call
