@@ -1175,9 +1175,10 @@ SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
   if (S > ntiles) S = ntiles;
   SplitPlan p;
+  // up to 8 splits: one cluster of exactly that many blocks (any size, not only powers of two);
+  // beyond: whole clusters of 8, merged by the combine kernel
   if (S >= kMaxCluster) { p.C = kMaxCluster; p.S = (int)(S / kMaxCluster) * kMaxCluster; }
-  else if (S >= 4) { p.C = 4; p.S = 4; }
-  else if (S >= 2) { p.C = 2; p.S = 2; }
+  else if (S >= 2) { p.C = (int)S; p.S = (int)S; }
   else { p.C = 1; p.S = 1; }
   if (p.S > 512) p.S = 512;
   p.Sp = p.S / p.C;

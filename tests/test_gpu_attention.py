@@ -53,6 +53,10 @@ def run_case(seed, B, H, N, L, Lcap=None, H_kv=None, kv_len=None, n_nodes=None, 
     (2, 3, 48, 200),         # N not a multiple of 32
     (1, 1, 64, 4096 + 17),   # many splits for one head
     (20, 16, 64, 513),       # enough units for a single split: direct output path
+    (7, 14, 64, 700),        # 3 splits: a cluster of three
+    (1, 59, 64, 700),        # 5 splits
+    (7, 7, 64, 1000),        # 6 splits
+    (6, 7, 48, 900),         # 7 splits, N = 48: owners get uneven row counts
     (40, 8, 128, 700),       # N = 128, one split per (context, head): direct output path
     (2, 3, 96, 300),         # 64 < N < 128: rows past N are padding of the 128-row block
     (1, 2, 80, 64),          # N = 80, prefix of exactly one tile
