@@ -59,19 +59,18 @@ __device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* _
                                      bool& bad) {
   int64_t p = (int64_t)__ldg(sa + slot);
   if (p < 0 || p >= n_tokens) { bad = true; return -1; }
+  const int64_t rem = n_tokens - p;
+  const int avail = rem < (int64_t)n ? (int)rem : n;     // tokens of the suffix that exist
+  const int32_t* __restrict__ row = T + p;
   int tk[16];
 #pragma unroll
-  for (int k = 0; k < 16; ++k) tk[k] = (k < n && p + k < n_tokens) ? __ldg(T + p + k) : 0;
-  int r = 0;
+  for (int k = 0; k < 16; ++k) tk[k] = (k < avail) ? __ldg(row + k) : 0;
+  int r = avail < n ? -1 : 0;                            // equal so far, but it ends early: smaller
 #pragma unroll
   for (int k = 15; k >= 0; --k) {
-    if (k < n) {
-      if (p + k >= n_tokens) {
-        r = -1;
-      } else {
-        uint32_t a = (uint32_t)tk[k], b = (uint32_t)q[k];
-        if (a != b) r = a < b ? -1 : 1;
-      }
+    if (k < avail) {
+      uint32_t a = (uint32_t)tk[k], b = (uint32_t)q[k];
+      if (a != b) r = a < b ? -1 : 1;
     }
   }
   return r;
@@ -86,7 +85,11 @@ __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __r
                                    int n, int lane, bool& eq, bool& bad) {
   while (hi - lo > 32) {
     int64_t size = hi - lo;
-    int64_t pos = lo + ((int64_t)(lane + 1) * size) / 33;
+    // 32 probes that cut the interval into 33 parts: floor((lane + 1) * size * floor(2^64 / 33)
+    // / 2^64) is at most (lane + 1) * size / 33, increasing in the lane, and below size; which
+    // slots are probed does not change the answer, only how fast the interval shrinks
+    int64_t pos = lo + (int64_t)__umul64hi((unsigned long long)(lane + 1) * (unsigned long long)size,
+                                           0x07C1F07C1F07C1F0ull);
     int c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
     bool t = STRICT ? (c > 0) : (c >= 0);
     unsigned b = __ballot_sync(kFull, t);
