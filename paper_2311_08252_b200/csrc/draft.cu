@@ -79,10 +79,13 @@ __device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* _
 // First slot in [lo, hi) whose comparison is >= 0 (STRICT = false) or > 0 (STRICT = true);
 // hi when there is none.  Warp-cooperative; all lanes return the same value.  `eq` reports
 // whether the returned slot compared equal (in: whether slot `hi` is known to compare equal).
+// `next_gt` (STRICT = false only): the first slot that compares greater, when the last round's
+// probes happen to show it (the run of equal slots ends inside the last 32 probed slots, or runs
+// up to a slot already known to be greater); -1 when it is not known.
 template <typename SaT, bool STRICT>
 __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
                                    int64_t n_tokens, int64_t lo, int64_t hi, const int (&q)[16],
-                                   int n, int lane, bool& eq, bool& bad) {
+                                   int n, int lane, bool& eq, bool& bad, int64_t* next_gt = nullptr) {
   while (hi - lo > 32) {
     int64_t size = hi - lo;
     // 32 probes that cut the interval into 33 parts: floor((lane + 1) * size * floor(2^64 / 33)
@@ -110,6 +113,11 @@ __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __r
   if (pos < hi) c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
   bool t = (pos < hi) && (STRICT ? (c > 0) : (c >= 0));
   unsigned b = __ballot_sync(kFull, t);
+  if (!STRICT && next_gt) {
+    // slot hi compares greater unless `eq` says it is equal (hi = end of the array counts as greater)
+    const unsigned gt = __ballot_sync(kFull, (pos < hi) && c > 0);
+    *next_gt = gt ? lo + (__ffs(gt) - 1) : (eq ? (int64_t)-1 : hi);
+  }
   if (b != 0) {
     int f = __ffs(b) - 1;
     int cf = __shfl_sync(kFull, c, f);
@@ -267,9 +275,12 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
 #pragma unroll
       for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
       bool bad = false, eq = false;
-      int64_t lb = warp_first_true<SaT, false>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad);
+      int64_t next_gt = -1;
+      int64_t lb = warp_first_true<SaT, false>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
       int64_t ub = lb;
-      if (eq && lb < n_tokens) {
+      if (eq && lb < n_tokens && next_gt >= 0) {
+        ub = next_gt;        // the last round of the lower bound already showed where the run ends
+      } else if (eq && lb < n_tokens) {
         // gallop: lane l probes lb + 2^l
         int64_t pos = lb + ((int64_t)1 << lane);
         bool t = true;
