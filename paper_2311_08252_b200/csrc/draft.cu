@@ -151,49 +151,30 @@ __device__ __forceinline__ int prev_set(const uint32_t* __restrict__ row, int j)
   return (w << 5) + 31 - __clz(bits | 1u);
 }
 
-// Executed by the whole block (it contains block barriers).  hist[0..nbins) holds counts;
-// total >= need >= 1.  Finds the largest bin b with sum(hist[k], k > b) < need; writes b and that
-// sum.  Every thread sums a few bins, top bins first; a block-wide prefix sum finds the thread
-// whose bins cross `need`, and that thread pins the bin down.  wsum: kWarps words of scratch.
-__device__ void block_threshold_desc(const uint32_t* hist, int nbins, uint32_t need, int tid,
-                                     uint32_t* wsum, int* out_bin, uint32_t* out_above) {
-  const int lane = tid & 31, warp = tid >> 5;
-  const int per = (nbins + kThreads - 1) / kThreads;
-  const int top = nbins - 1 - tid * per;
+// Executed by one warp.  hist[0..nbins) holds counts; total >= need >= 1.  Finds the largest
+// bin b with sum(hist[k], k > b) < need; returns b and that sum.
+__device__ void warp_threshold_desc(const uint32_t* hist, int nbins, uint32_t need, int lane,
+                                    int* out_bin, uint32_t* out_above) {
+  int per = (nbins + 31) / 32;
+  int top = nbins - 1 - lane * per;
+  int bot = max(0, top - per + 1);
   uint32_t s = 0;
-  for (int k = 0; k < per; ++k)
-    if (top - k >= 0) s += hist[top - k];
+  for (int b = top; b >= bot && b >= 0; --b) s += hist[b];
   uint32_t incl = s;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     uint32_t v = __shfl_up_sync(kFull, incl, o);
     if (lane >= o) incl += v;
   }
-  if (lane == 31) wsum[warp] = incl;
-  __syncthreads();
-  uint32_t base = 0;
-  for (int w = 0; w < warp; ++w) base += wsum[w];
-  const uint32_t excl = base + incl - s;
-  if (excl < need && need <= excl + s) {
+  uint32_t excl = incl - s;
+  if (excl < need && need <= incl) {
     uint32_t acc = excl;
-    for (int k = 0; k < per; ++k) {
-      const uint32_t h = hist[top - k];      // top - k >= 0: bins below 0 would not add to s
-      if (acc + h >= need) { *out_bin = top - k; *out_above = acc; break; }
+    for (int b = top; b >= bot; --b) {
+      uint32_t h = hist[b];
+      if (acc + h >= need) { *out_bin = b; *out_above = acc; break; }
       acc += h;
     }
   }
-  __syncthreads();
-}
-
-// atomicAdd(counter, 1) for every calling lane with one atomic per group of lanes that are
-// executing this together; returns each lane's own slot.
-__device__ __forceinline__ uint32_t warp_aggregated_inc(uint32_t* counter, int lane) {
-  const unsigned act = __activemask();
-  const int leader = __ffs(act) - 1;
-  uint32_t base = 0;
-  if (lane == leader) base = atomicAdd(counter, (uint32_t)__popc(act));
-  base = __shfl_sync(act, base, leader);
-  return base + (uint32_t)__popc(act & ((1u << lane) - 1u));
 }
 
 struct Smem {
@@ -268,6 +249,8 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   }
 
   // ---- phase 1: search --------------------------------------------------------------
+  // 1a: lower bound of every suffix length, one warp each.  ub = -1 marks "matches, end of the
+  // run not known yet".
   {
     const int n = a.n_min + warp;
     if (n <= nq) {
@@ -277,36 +260,47 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       bool bad = false, eq = false;
       int64_t next_gt = -1;
       int64_t lb = warp_first_true<SaT, false>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
-      int64_t ub = lb;
-      if (eq && lb < n_tokens && next_gt >= 0) {
-        ub = next_gt;        // the last round of the lower bound already showed where the run ends
-      } else if (eq && lb < n_tokens) {
-        // gallop: lane l probes lb + 2^l
-        int64_t pos = lb + ((int64_t)1 << lane);
-        bool t = true;
-        if (pos < n_tokens) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
-        unsigned bal = __ballot_sync(kFull, t);
-        int64_t lo2, hi2 = n_tokens;
-        bool eq2 = false;
-        if (bal == 0) {
-          lo2 = lb + ((int64_t)1 << 31) + 1;
-        } else {
-          int f = __ffs(bal) - 1;
-          int64_t pf = lb + ((int64_t)1 << f);
-          hi2 = pf < n_tokens ? pf : n_tokens;
-          lo2 = f > 0 ? lb + ((int64_t)1 << (f - 1)) + 1 : lb + 1;
-        }
-        if (lo2 > hi2) lo2 = hi2;
-        ub = warp_first_true<SaT, true>(T, sa, n_tokens, lo2, hi2, q, n, lane, eq2, bad);
-      }
       if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
-      if (lane == 0) { s.lb[n] = lb; s.ub[n] = ub; }
+      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_tokens) ? next_gt : lb; }
     }
   }
   __syncthreads();
   int n_win = 0;
   for (int n = nq; n >= a.n_min; --n)
-    if (s.ub[n] > s.lb[n]) { n_win = n; break; }
+    if (s.ub[n] != s.lb[n]) { n_win = n; break; }
+  // 1b: only the winning length needs its upper bound, and only if the last round of its lower
+  // bound did not already show where the run ends (shorter lengths match far more slots and
+  // would need the most rounds: they are never looked at again)
+  if (n_win != 0 && s.ub[n_win] < 0) {       // block-uniform
+    if (warp == n_win - a.n_min) {
+      const int n = n_win;
+      int q[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
+      bool bad = false;
+      const int64_t lb = s.lb[n];
+      // gallop: lane l probes lb + 2^l
+      int64_t pos = lb + ((int64_t)1 << lane);
+      bool t = true;
+      if (pos < n_tokens) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
+      unsigned bal = __ballot_sync(kFull, t);
+      int64_t lo2, hi2 = n_tokens;
+      bool eq2 = false;
+      if (bal == 0) {
+        lo2 = lb + ((int64_t)1 << 31) + 1;
+      } else {
+        int f = __ffs(bal) - 1;
+        int64_t pf = lb + ((int64_t)1 << f);
+        hi2 = pf < n_tokens ? pf : n_tokens;
+        lo2 = f > 0 ? lb + ((int64_t)1 << (f - 1)) + 1 : lb + 1;
+      }
+      if (lo2 > hi2) lo2 = hi2;
+      const int64_t ub = warp_first_true<SaT, true>(T, sa, n_tokens, lo2, hi2, q, n, lane, eq2, bad);
+      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+      if (lane == 0) s.ub[n] = ub;
+    }
+    __syncthreads();
+  }
   if (s.err != 0 || n_win == 0) {
     if (tid == 0) {
       a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
@@ -440,15 +434,13 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
     const int lcp = ll & 0xFF, len = ll >> 8;
     // Weights along a row never grow with depth: walk down from the first depth at which the
     // row starts a node until the weight drops to 1; every deeper node of the row weighs 1.
-    uint32_t nheavy = 0, nbin0 = 0;
+    uint32_t nheavy = 0;
     int d1 = len + 1;                      // first depth of weight 1 (len + 1: none)
     if (valid) {
       for (int d = lcp + 1; d <= len; ++d) {
         const int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
         if (c < 2) { d1 = d; break; }
-        // bin of the key (c << 5 | 16 - d) >> 10 = c >> 5.  Nearly every node weighs less than
-        // 32 and lands in bin 0: those are counted in a register and added once per warp
-        if ((c >> 5) == 0) ++nbin0; else atomicAdd(&s.hist_hi[c >> 5], 1u);
+        atomicAdd(&s.hist_hi[((c << 5) | (16 - d)) >> 10], 1u);
         ++nheavy;
       }
     }
@@ -459,12 +451,8 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       if (lane == 0 && (st | en)) atomicAdd(&s.e1diff[d], __popc(st) - __popc(en));
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      nheavy += __shfl_xor_sync(kFull, nheavy, o);
-      nbin0 += __shfl_xor_sync(kFull, nbin0, o);
-    }
+    for (int o = 16; o > 0; o >>= 1) nheavy += __shfl_xor_sync(kFull, nheavy, o);
     if (lane == 0 && nheavy) atomicAdd(&s.heavy_total, nheavy);
-    if (lane == 0 && nbin0) atomicAdd(&s.hist_hi[0], nbin0);
   }
   __syncthreads();
 
@@ -479,7 +467,8 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   uint32_t r_tie;      // plus the first r_tie nodes (by row) with key == tstar
   const uint32_t heavy_total = s.heavy_total;
   if (heavy_total >= (uint32_t)N) {
-    block_threshold_desc(s.hist_hi, kHistHi, (uint32_t)N, tid, s.warp_cnt, &s.bin_hi, &s.above_hi);
+    if (warp == 0) warp_threshold_desc(s.hist_hi, kHistHi, (uint32_t)N, lane, &s.bin_hi, &s.above_hi);
+    __syncthreads();
     const int bin_hi = s.bin_hi;
     for (int it = 0; it < niter; ++it) {
       const int jbase = it * kThreads + warp * 32;
@@ -492,15 +481,13 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
         int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
         if (c < 2) break;   // weights do not grow with depth
         uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
-        if ((int)(key >> 10) == bin_hi) {
-          // few distinct keys (small weights at ten depths): lanes with the same key add once
-          const unsigned same = __match_any_sync(__activemask(), key);
-          if (lane == __ffs(same) - 1) atomicAdd(&s.hist_lo[key & 1023u], (uint32_t)__popc(same));
-        }
+        if ((int)(key >> 10) == bin_hi) atomicAdd(&s.hist_lo[key & 1023u], 1u);
       }
     }
     __syncthreads();
-    block_threshold_desc(s.hist_lo, kHistLo, (uint32_t)N - s.above_hi, tid, s.warp_cnt, &s.bin_lo, &s.above_lo);
+    if (warp == 0)
+      warp_threshold_desc(s.hist_lo, kHistLo, (uint32_t)N - s.above_hi, lane, &s.bin_lo, &s.above_lo);
+    __syncthreads();
     tstar = ((uint32_t)bin_hi << 10) | (uint32_t)s.bin_lo;
     r_tie = (uint32_t)N - s.above_hi - s.above_lo;
   } else {
@@ -529,7 +516,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
         int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
         uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
         if (key > tstar) {
-          uint32_t slot = warp_aggregated_inc(&s.nsel, lane);
+          uint32_t slot = atomicAdd(&s.nsel, 1u);
           if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)j; s.selcnt[slot] = c; }
         } else {
           tie = key == tstar;
@@ -549,7 +536,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       }
       uint32_t rank = before + __popc(bal & ((1u << lane) - 1u));
       if (tie && rank < r_tie) {
-        uint32_t slot = warp_aggregated_inc(&s.nsel, lane);
+        uint32_t slot = atomicAdd(&s.nsel, 1u);
         if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d_tie << 16) | (uint32_t)j; s.selcnt[slot] = c_tie; }
       }
       tie_base += total;
