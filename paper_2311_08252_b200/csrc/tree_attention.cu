@@ -64,6 +64,7 @@ struct AttnArgs {
   int B, H, group, N, Wm;
   int S;            // key splits per (context, head) = C * Sp
   int NBLK;         // 128-row query blocks per (context, head) in the wide kernel (else 1)
+  int pack;         // query heads per block in the wide kernel: 2 when N = 64 and heads share KV
   int q_slot[3], kv_slot[3];   // tensor-map coordinate index (1..3) of rows, head, batch
   int C;            // blocks per cluster
   int Sp;           // clusters per (context, head); > 1 needs the merge kernel
@@ -765,9 +766,12 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   int bid = blockIdx.x;
   const int split = bid % a.S; bid /= a.S;
   const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 128-row block of the N draft rows
-  const int h = bid % a.H;
-  const int b = bid / a.H;
-  const int hk = h / a.group;
+  // pack = 2 (N = 64, grouped KV heads): the block's 128 rows are the 64 draft rows of two query
+  // heads that share one KV head, so that K/V stream is read once for both
+  const int heads_per_block = a.pack;
+  const int h0 = (bid % (a.H / heads_per_block)) * heads_per_block;
+  const int b = bid / (a.H / heads_per_block);
+  const int hk = h0 / a.group;
   const int row0 = rblk * 128;                       // first draft row of this thread block
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -807,7 +811,8 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
 
   // softmax thread = draft row row0 + 32 warp + lane
   const int row = (warp & 3) * 32 + lane;            // row inside this block
-  const int grow = row0 + row;                       // draft row
+  const int grow = heads_per_block == 2 ? (row & 63) : row0 + row;   // draft row
+  const int h = heads_per_block == 2 ? h0 + (row >> 6) : h0;         // its query head
   float m_used = -INFINITY, l_run = 0.f;
 
   tc_fence_before();
@@ -821,10 +826,12 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
     if (lane == 0) {
       mbar_expect_tx(bars + kBarQFull, (uint32_t)kWideQBytes);
       // two 64-dim halves, each [128 rows x 128 B]; rows past N are zero-filled
-      tma_load_box(sQ, &tm_q, 0, row0, h, b, a.q_slot, bars + kBarQFull);
-      tma_load_box(sQ + 64 * 128, &tm_q, 0, row0 + 64, h, b, a.q_slot, bars + kBarQFull);
-      tma_load_box(sQ + 128 * 128, &tm_q, 64, row0, h, b, a.q_slot, bars + kBarQFull);
-      tma_load_box(sQ + 192 * 128, &tm_q, 64, row0 + 64, h, b, a.q_slot, bars + kBarQFull);
+      // second 64 rows: the next 64 draft rows of the same head, or the second head's rows
+      const int r1 = heads_per_block == 2 ? 0 : row0 + 64, h1 = heads_per_block == 2 ? h0 + 1 : h0;
+      tma_load_box(sQ, &tm_q, 0, row0, h0, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 64 * 128, &tm_q, 0, r1, h1, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 128 * 128, &tm_q, 64, row0, h0, b, a.q_slot, bars + kBarQFull);
+      tma_load_box(sQ + 192 * 128, &tm_q, 64, r1, h1, b, a.q_slot, bars + kBarQFull);
       int issued_k = 0, issued_v = 0;
       for (int it = 0; it < nt; ++it) {
         const int slot = it & 1, key0 = (t0 + it) * kBN;
@@ -1244,8 +1251,11 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
     a.ws_ml = a.ws_o + (size_t)B * H * a.Sp * N * kD;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool wide = N > 64;
-  a.NBLK = wide ? (N + 127) / 128 : 1;
+  // Grouped KV heads with N = 64 and a batch that fills the GPU without key splits: two query
+  // heads of a group share one 128-row block of the wide kernel (their K/V is streamed once)
+  a.pack = (N == 64 && (a.group % 2) == 0 && (int64_t)B * H / 2 >= 2 * kNumSMs) ? 2 : 1;
+  const bool wide = N > 64 || a.pack == 2;
+  a.NBLK = N > 64 ? (N + 127) / 128 : 1;
   const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
   if (wide)
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_wide_kernel), 3, smem));
@@ -1253,7 +1263,7 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 2, smem));
   if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(B * H * a.NBLK * a.S), 1, 1);
+  cfg.gridDim = dim3((unsigned)(B * (H / a.pack) * a.NBLK * a.S), 1, 1);
   cfg.blockDim = dim3((unsigned)kWsThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;

@@ -80,6 +80,15 @@ def test_ragged_batch_grouped_heads_padding_nodes_and_strides():
     run_case(12, 2, 6, 32, 90, H_kv=3, kv_len=[90, 31], n_nodes=1, scale=0.2)
 
 
+def test_grouped_heads_large_batch_two_query_heads_per_block():
+    # N = 64, heads in groups, batch large enough that no key split is needed: pairs of query
+    # heads of a group are computed by one block
+    rng = np.random.default_rng(3)
+    run_case(16, 40, 16, 64, 513, H_kv=4, kv_len=rng.integers(0, 514, 40), n_nodes=50)
+    run_case(17, 20, 32, 64, 300, H_kv=16, kv_len=rng.integers(1, 301, 20))
+    run_case(18, 75, 8, 64, 130, H_kv=1, Lcap=300)
+
+
 def test_wide_rows_ragged_batch_and_grouped_heads():
     # N > 64 with contexts far shorter than the longest one: some key splits get no tile at all
     run_case(13, 4, 8, 128, 900, Lcap=1100, H_kv=2, kv_len=[900, 1, 333, 64], n_nodes=77, max_depth=16)
