@@ -814,6 +814,7 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   const int grow = heads_per_block == 2 ? (row & 63) : row0 + row;   // draft row
   const int h = heads_per_block == 2 ? h0 + (row >> 6) : h0;         // its query head
   float m_used = -INFINITY, l_run = 0.f;
+  bool have_o = false;                 // this warp may read a finished O out of TMEM
 
   tc_fence_before();
   __syncthreads();
@@ -1018,19 +1019,23 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + kBarPFull);
     }
-    // epilogue: O row out of TMEM
-    if (ok && nt > 0 && wait_all(bars + kBarOFull, (uint32_t)((nt - 1) & 1))) {
-      tc_fence_after();
-      const bool live = grow < N;
+    have_o = ok && nt > 0 && wait_all(bars + kBarOFull, (uint32_t)((nt - 1) & 1));
+    if (have_o) tc_fence_after();
+  }
+
+  const bool softmax_warp = warp < 4;
+  const bool live = grow < N;
+  if (a.C == 1) {
+    // ---- no cluster: straight to the output, or (several clusters of one block never happen)
+    if (softmax_warp && have_o) {
       const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + grow;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t orr[32];
         __syncwarp();
         tmem_ld_32x32(tmem_warp + kColO + c * 32, orr);
         tmem_wait_ld();
-        if (live && a.S == 1) {
+        if (live) {
           __nv_bfloat16* op = a.out + b * a.o_b + (int64_t)grow * a.o_n + h * a.o_h + c * 32;
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
@@ -1041,27 +1046,98 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
             pv.w = pack_bf16(__uint_as_float(orr[8 * q4 + 6]) * inv, __uint_as_float(orr[8 * q4 + 7]) * inv);
             *reinterpret_cast<uint4*>(op + q4 * 8) = pv;
           }
-        } else if (live) {
-          float* wp = a.ws_o + part * kD + c * 32;
+        }
+      }
+      if (live && a.lse) a.lse[((int64_t)b * a.H + h) * N + grow] = (m_used + log2f(l_run)) * kLn2;
+    }
+  } else {
+    // ---- merge across the cluster.  Rows [r*R, r*R + R) of this 128-row block belong to block
+    // r.  After a first cluster barrier (every block's operand tiles are dead) each softmax
+    // thread stores its row - 128 floats of O out of TMEM, then max and sum - straight into the
+    // owner's shared memory (posted remote stores, slot = sender's rank); after a second barrier
+    // each owner reduces its C slots locally.  Both barriers are passed by every thread of every
+    // block whatever happened before, so a block that gave up cannot leave its mates waiting.
+    const int C = a.C;
+    const int rank = split % C;
+    const int Nl = min(128, N - row0);
+    const int R = (Nl + C - 1) / C;
+    float* sRecv = reinterpret_cast<float*>(smem);                     // [C][R][kOStride]
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (softmax_warp) {
+      const int owner = live ? row / R : 0;
+      const uint32_t dst_local = smem_u32(sRecv + ((size_t)rank * R + (row - owner * R)) * kOStride);
+      uint32_t dst;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(dst) : "r"(dst_local), "r"(owner));
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t orr[32];
+        __syncwarp();
+        if (have_o) {                       // warp-uniform
+          tmem_ld_32x32(tmem_warp + kColO + c * 32, orr);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) orr[j] = 0u;
+        }
+        if (live) {
 #pragma unroll
           for (int q4 = 0; q4 < 8; ++q4)
-            *reinterpret_cast<uint4*>(wp + q4 * 4) =
-                make_uint4(orr[4 * q4], orr[4 * q4 + 1], orr[4 * q4 + 2], orr[4 * q4 + 3]);
+            asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};"
+                         ::"r"(dst + (uint32_t)((c * 32 + q4 * 4) * 4)), "r"(orr[4 * q4]), "r"(orr[4 * q4 + 1]),
+                           "r"(orr[4 * q4 + 2]), "r"(orr[4 * q4 + 3])
+                         : "memory");
         }
       }
       if (live) {
-        if (a.S == 1) {
-          if (a.lse) a.lse[((int64_t)b * a.H + h) * N + grow] = (m_used + log2f(l_run)) * kLn2;
-        } else {
-          a.ws_ml[part * 2] = m_used;
-          a.ws_ml[part * 2 + 1] = l_run;
+        const float mm = have_o ? m_used : -INFINITY, ll = have_o ? l_run : 0.f;
+        asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(dst + (uint32_t)(kD * 4)), "f"(mm), "f"(ll)
+                     : "memory");
+      }
+    }
+    tc_fence_before();
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const int sup = split / C;
+    const int my_rows = max(0, min(R, Nl - rank * R));
+    for (int idx = tid; idx < my_rows * 32; idx += kWsThreads) {
+      const int lr = idx >> 5, mr = row0 + rank * R + lr, c4 = idx & 31;   // mr: draft row
+      float2 ml[kMaxCluster];
+      float4 ov[kMaxCluster];
+#pragma unroll
+      for (int p = 0; p < kMaxCluster; ++p) {
+        if (p < C) {
+          const float* rr = sRecv + (size_t)(p * R + lr) * kOStride;
+          ml[p] = *reinterpret_cast<const float2*>(rr + kD);
+          ov[p] = *reinterpret_cast<const float4*>(rr + c4 * 4);
         }
       }
-    } else if (ok && nt == 0 && a.S > 1 && grow < N) {
-      // a split beyond this context's last tile: an empty partial the combine kernel skips
-      const int64_t part = (((int64_t)b * a.H + h) * a.Sp + split) * N + grow;
-      a.ws_ml[part * 2] = -INFINITY;
-      a.ws_ml[part * 2 + 1] = 0.f;
+      float M = -INFINITY;
+#pragma unroll
+      for (int p = 0; p < kMaxCluster; ++p)
+        if (p < C) M = fmaxf(M, ml[p].x);
+      float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      float lsum = 0.f;
+#pragma unroll
+      for (int p = 0; p < kMaxCluster; ++p) {
+        if (p < C) {
+          const float w = (ml[p].x == -INFINITY) ? 0.f : ex2(ml[p].x - M);
+          lsum += ml[p].y * w;
+          o4.x += ov[p].x * w; o4.y += ov[p].y * w; o4.z += ov[p].z * w; o4.w += ov[p].w * w;
+        }
+      }
+      if (a.Sp == 1) {
+        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+        uint2 pk2;
+        pk2.x = pack_bf16(o4.x * inv, o4.y * inv);
+        pk2.y = pack_bf16(o4.z * inv, o4.w * inv);
+        *reinterpret_cast<uint2*>(a.out + b * a.o_b + (int64_t)mr * a.o_n + h0 * a.o_h + c4 * 4) = pk2;
+        if (a.lse && c4 == 0) a.lse[((int64_t)b * a.H + h0) * N + mr] = (M + log2f(lsum)) * kLn2;
+      } else {
+        const int64_t base = ((((int64_t)b * a.H + h0) * a.Sp + sup) * N + mr);
+        *reinterpret_cast<float4*>(a.ws_o + base * kD + c4 * 4) = o4;
+        if (c4 == 0) { a.ws_ml[base * 2] = M; a.ws_ml[base * 2 + 1] = lsum; }
+      }
     }
   }
   tc_fence_before();
@@ -1163,8 +1239,8 @@ struct SplitPlan { int S, C, Sp; };
 
 // Key splits per (context, head, row block): enough blocks to fill the GPU once (never a
 // partial second wave), at most one split per tile, rounded down to a whole number of clusters.
-// N > 64 runs the wide kernel: one block per (context, head, split), no clusters, every split's
-// partial goes through the workspace.
+// N > 64 runs the wide kernel, one block per (context, head, 128-row block, split), with the
+// same cluster rule.
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
   if (N > 64) {
@@ -1173,7 +1249,9 @@ SplitPlan plan_splits(int B, int H, int N, int max_kv) {
     if (S > 512) S = 512;
     if (S < 1) S = 1;
     SplitPlan p;
-    p.S = (int)S; p.C = 1; p.Sp = (int)S;
+    if (S >= kMaxCluster) { p.C = kMaxCluster; p.S = (int)(S / kMaxCluster) * kMaxCluster; }
+    else { p.C = (int)S; p.S = (int)S; }
+    p.Sp = p.S / p.C;
     return p;
   }
   // every 64-row block of the draft rows has its own thread blocks; two blocks fit an SM
