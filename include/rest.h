@@ -177,11 +177,9 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  *     d_ws / ws_bytes.  The call itself performs no device or host allocation.
  *   - Returns REST_WORKSPACE_TOO_SMALL, launching nothing, when
  *     rest_tree_attention_workspace_bytes(B, H, N, D, max_kv) exceeds REST_STATIC_SCRATCH_BYTES.
- *     For N <= 64 scratch is only needed when one (context, head) pair is cut into more than
- *     8 key ranges, i.e. for very few pairs with long caches: B*H = 2, N = 64, max_kv = 4160
- *     needs 0.51 MiB and fits; B*H = 2, N = 64, max_kv = 8256 needs 1.02 MiB and is refused.
- *     For N > 64 every key range's partial goes through the scratch (B*H*S*N*520 bytes for S
- *     ranges): small batches with long caches are refused, large batches (S = 1) need none.
+ *     Scratch is only needed when one (context, head) pair is cut into more than 8 key ranges,
+ *     i.e. for very few pairs with long caches: B*H = 2, N = 64, max_kv = 4160 needs 0.51 MiB
+ *     and fits; B*H = 2, N = 64, max_kv = 8256 needs 1.02 MiB and is refused.
  *   - The first call on each device looks up the array's device address (one runtime query,
  *     with that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.
