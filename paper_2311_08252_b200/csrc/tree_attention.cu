@@ -29,6 +29,7 @@
 // mbarrier; the owner reduces locally and writes bf16 output.  Only when more than 8 splits
 // are needed do the cluster-merged partials go to the caller's workspace for a second, small
 // merge kernel.
+#include <atomic>
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -1235,38 +1236,68 @@ bool encode_box_map(CUtensorMap* map, const void* base, int64_t rows, int64_t he
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// How many clusters of c blocks of a kernel can be resident on the current device at once.
+// The scheduler places a cluster inside one GPC, so this is not 2 * SMs / c: 37 clusters of 8
+// do not fit although 296 blocks would, and the 37th cluster would run as a second wave.  Asked
+// from the runtime once per device, kernel and size; without a device (size queries on a machine
+// that has none) the plain quotient stands in.
+int cluster_capacity(bool wide, int c) {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cache[kMaxDev][2][kMaxCluster + 1];
+  const int nominal = (2 * kNumSMs) / c;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { (void)cudaGetLastError(); return nominal; }
+  const int have = cache[dev][wide ? 1 : 0][c].load(std::memory_order_relaxed);
+  if (have > 0) return have;
+  const void* fn = wide ? reinterpret_cast<const void*>(tree_attention_wide_kernel)
+                        : reinterpret_cast<const void*>(tree_attention_ws_kernel);
+  const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
+  int n = 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(c * 64), 1, 1);
+  cfg.blockDim = dim3((unsigned)kWsThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)c;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (rest::ensure_dynamic_smem(fn, wide ? 3 : 2, smem) != cudaSuccess ||
+      cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return nominal;
+  }
+  cache[dev][wide ? 1 : 0][c].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 struct SplitPlan { int S, C, Sp; };
 
-// Key splits per (context, head, row block): enough blocks to fill the GPU once (never a
-// partial second wave), at most one split per tile, rounded down to a whole number of clusters.
-// N > 64 runs the wide kernel, one block per (context, head, 128-row block, split), with the
-// same cluster rule.
+// Key splits per unit (context, head, row block).  The splits of a unit form clusters of C
+// blocks (merged on chip); Sp clusters per unit (merged by the combine kernel when Sp > 1).
+// The plan is the largest cluster size whose clusters all fit on the GPU at once - a partial
+// second wave would double the time - then as many clusters per unit as still fit, and never
+// more splits than tiles.
 SplitPlan plan_splits(int B, int H, int N, int max_kv) {
   const int ntiles = (max_kv + kBN - 1) / kBN;
-  if (N > 64) {
-    int64_t S = ((int64_t)kNumSMs * 2) / ((int64_t)B * H * ((N + 127) / 128));
-    if (S > ntiles) S = ntiles;
-    if (S > 512) S = 512;
-    if (S < 1) S = 1;
-    SplitPlan p;
-    if (S >= kMaxCluster) { p.C = kMaxCluster; p.S = (int)(S / kMaxCluster) * kMaxCluster; }
-    else { p.C = (int)S; p.S = (int)S; }
-    p.Sp = p.S / p.C;
-    return p;
-  }
-  // every 64-row block of the draft rows has its own thread blocks; two blocks fit an SM
-  const int64_t units = (int64_t)B * H * ((N + 63) / 64);
-  const int blocks_per_sm = 2;
-  int64_t S = ((int64_t)kNumSMs * blocks_per_sm) / units;
-  if (S > ntiles) S = ntiles;
+  const bool wide = N > 64;
+  const int64_t units = (int64_t)B * H * (wide ? (N + 127) / 128 : 1);
   SplitPlan p;
-  // up to 8 splits: one cluster of exactly that many blocks (any size, not only powers of two);
-  // beyond: whole clusters of 8, merged by the combine kernel
-  if (S >= kMaxCluster) { p.C = kMaxCluster; p.S = (int)(S / kMaxCluster) * kMaxCluster; }
-  else if (S >= 2) { p.C = (int)S; p.S = (int)S; }
-  else { p.C = 1; p.S = 1; }
-  if (p.S > 512) p.S = 512;
-  p.Sp = p.S / p.C;
+  p.C = 1; p.S = 1; p.Sp = 1;
+  for (int c = kMaxCluster; c >= 2; --c) {
+    if (c > ntiles) continue;
+    const int64_t cap = cluster_capacity(wide, c);
+    if (units > cap) continue;
+    int64_t sp = cap / units;
+    if (sp > ntiles / c) sp = ntiles / c;
+    if (sp > 64) sp = 64;
+    if (sp < 1) sp = 1;
+    p.C = c; p.Sp = (int)sp; p.S = c * (int)sp;
+    break;
+  }
   return p;
 }
 
