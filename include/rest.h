@@ -178,8 +178,10 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  *   - Returns REST_WORKSPACE_TOO_SMALL, launching nothing, when
  *     rest_tree_attention_workspace_bytes(B, H, N, D, max_kv) exceeds REST_STATIC_SCRATCH_BYTES.
  *     Scratch is only needed when one (context, head) pair is cut into more than 8 key ranges,
- *     i.e. for very few pairs with long caches: B*H = 2, N = 64, max_kv = 4160 needs 0.51 MiB
- *     and fits; B*H = 2, N = 64, max_kv = 8256 needs 1.02 MiB and is refused.
+ *     i.e. for very few pairs with long caches, and then holds one partial of N x 130 floats per
+ *     cluster of 8 ranges; no more clusters are used than the GPU can run at once (about 30).
+ *     With N <= 64 every shape fits; B*H = 1, N = 256, max_kv = 16640 needs about 2 MiB and
+ *     is refused.
  *   - The first call on each device looks up the array's device address (one runtime query,
  *     with that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.
