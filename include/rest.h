@@ -162,6 +162,16 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
                                 float* d_lse, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
+ * rest_tree_attention_plan - how rest_tree_attention would cut the key range for this shape on
+ * the current device (a planning aid; the paper has no counterpart).  out[0] = key ranges per
+ * (context, head), out[1] = blocks per cluster (ranges merged on chip), out[2] = clusters per
+ * (context, head) (merged through the workspace when > 1), out[3] = clusters of that size the
+ * device can run at once.  Host pointers.
+ */
+rest_status rest_tree_attention_plan(int32_t B, int32_t H, int32_t N, int32_t D, int32_t max_kv,
+                                     int32_t* out);
+
+/*
  * rest_tree_attention_static_scratch - rest_tree_attention for callers that cannot allocate.
  *
  * (The paper has no counterpart; this is a packaging variant of the call above.)
@@ -170,7 +180,7 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  * a serving process that handed every free byte of device memory to its own KV-cache pool at
  * start-up, or a decode loop whose rules forbid allocation calls because cudaMalloc/cudaFree
  * may stall the whole device.  For them the split-KV partials live in a fixed array of
- * REST_STATIC_SCRATCH_BYTES (1 MiB) inside the library image.  Every GPU that loads the
+ * REST_STATIC_SCRATCH_BYTES (768 KiB) inside the library image.  Every GPU that loads the
  * library holds that array until the process exits, whether or not this call is used.
  *
  *   - Arguments, layouts, results and limits are those of rest_tree_attention, without
@@ -180,8 +190,8 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  *     Scratch is only needed when one (context, head) pair is cut into more than 8 key ranges,
  *     i.e. for very few pairs with long caches, and then holds one partial of N x 130 floats per
  *     cluster of 8 ranges; no more clusters are used than the GPU can run at once (about 30).
- *     With N <= 64 every shape fits; B*H = 1, N = 256, max_kv = 16640 needs about 2 MiB and
- *     is refused.
+ *     B*H = 2, N = 64, max_kv = 4160 needs 0.51 MiB and fits; B*H = 1, N = 64, max_kv = 16448
+ *     needs about 0.9 MiB and is refused.
  *   - The first call on each device looks up the array's device address (one runtime query,
  *     with that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.
@@ -189,7 +199,7 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
  *     start at zero.  But two calls whose kernels may overlap on the GPU (different streams)
  *     race on the array: serialise them.
  */
-enum { REST_STATIC_SCRATCH_BYTES = 1024 * 1024 };
+enum { REST_STATIC_SCRATCH_BYTES = 768 * 1024 };
 rest_status rest_tree_attention_static_scratch(
     const void* d_q, const void* d_k, const void* d_v, const int64_t* strides,
     const int32_t* d_kv_len, const uint32_t* d_mask, int32_t B, int32_t H, int32_t H_kv, int32_t N,

@@ -30,7 +30,7 @@ EXPORTS = (
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
     "rest_tree_attention_static_scratch",
     "rest_device_error_flags", "rest_kv_commit", "rest_probe_dependent_reads",
-    "rest_suffix_array_workspace_bytes", "rest_suffix_array_build",
+    "rest_suffix_array_workspace_bytes", "rest_suffix_array_build", "rest_tree_attention_plan",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -89,6 +89,8 @@ def lib():
     L.rest_suffix_array_workspace_bytes.argtypes = [u64]
     L.rest_suffix_array_build.restype = i32
     L.rest_suffix_array_build.argtypes = [vp, u64, i32, vp, vp, sz, vp]
+    L.rest_tree_attention_plan.restype = i32
+    L.rest_tree_attention_plan.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
     L.rest_probe_dependent_reads.restype = i32
     L.rest_probe_dependent_reads.argtypes = [vp, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_uint32, vp, vp]
     L.rest_device_error_flags.restype = i32
@@ -270,7 +272,7 @@ def rest_tree_attention(q, k, v, kv_len, mask, scale, max_kv=None, out=None, lse
 def rest_tree_attention_static_scratch(q, k, v, kv_len, mask, scale, out, max_kv=None, lse=None,
                                        stream=None):
     """rest_tree_attention without a workspace argument, for callers that must not allocate:
-    the split partials go to a fixed 1 MiB array inside the library.  `out` (bf16 [B,N,H,D])
+    the split partials go to a fixed 768 KiB array inside the library.  `out` (bf16 [B,N,H,D])
     is supplied by the caller, so this wrapper allocates nothing on the device either.
     Raises RestError (workspace too small) when the shape needs more than the fixed array.
     Calls share that array: do not let two of them overlap on the GPU."""
@@ -376,3 +378,11 @@ def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None):
     # set-up call: wait here, so that the scratch can be released whatever stream was used
     torch.cuda.synchronize(tokens.device)
     return sa
+
+
+def tree_attention_plan(B, H, N, D, max_kv) -> dict:
+    """Key ranges per (context, head), blocks per cluster, clusters per (context, head), and how
+    many clusters of that size the current device runs at once."""
+    out = (ctypes.c_int32 * 4)()
+    _check(lib().rest_tree_attention_plan(B, H, N, D, max_kv, out), "rest_tree_attention_plan")
+    return {"splits": out[0], "cluster": out[1], "clusters_per_unit": out[2], "capacity": out[3]}

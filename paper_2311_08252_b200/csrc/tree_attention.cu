@@ -1312,6 +1312,16 @@ extern "C" rest_status rest_device_error_flags(uint32_t* h_flags) {
   return REST_OK;
 }
 
+extern "C" rest_status rest_tree_attention_plan(int32_t B, int32_t H, int32_t N, int32_t D,
+                                                int32_t max_kv, int32_t* out) {
+  if (!out || B <= 0 || H <= 0 || N <= 0 || max_kv <= 0) return REST_INVALID_ARG;
+  if (D != kD || N > REST_MAX_N) return REST_UNSUPPORTED;
+  const SplitPlan p = plan_splits(B, H, N, max_kv);
+  out[0] = p.S; out[1] = p.C; out[2] = p.Sp;
+  out[3] = cluster_capacity(N > 64, p.C);
+  return REST_OK;
+}
+
 extern "C" size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
                                                       int32_t max_kv) {
   if (B <= 0 || H <= 0 || N <= 0 || D != kD || max_kv <= 0) return 0;
