@@ -191,7 +191,7 @@ rest_status rest_tree_attention_plan(int32_t B, int32_t H, int32_t N, int32_t D,
  *     i.e. for very few pairs with long caches, and then holds one partial of N x 130 floats per
  *     cluster of 8 ranges; no more clusters are used than the GPU can run at once (about 30).
  *     B*H = 2, N = 64, max_kv = 4160 needs 0.51 MiB and fits; B*H = 1, N = 64, max_kv = 16448
- *     needs about 0.9 MiB and is refused.
+ *     needs about 1 MiB and is refused.
  *   - The first call on each device looks up the array's device address (one runtime query,
  *     with that device current).  Make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.

@@ -1239,9 +1239,12 @@ bool encode_box_map(CUtensorMap* map, const void* base, int64_t rows, int64_t he
 
 // How many clusters of c blocks of a kernel can be resident on the current device at once.
 // The scheduler places a cluster inside one GPC, so this is not 2 * SMs / c: 37 clusters of 8
-// do not fit although 296 blocks would, and the 37th cluster would run as a second wave.  Asked
-// from the runtime once per device, kernel and size; without a device (size queries on a machine
-// that has none) the plain quotient stands in.
+// do not fit although 296 blocks would, and the 37th cluster would run as a second wave.
+// cudaOccupancyMaxActiveClusters knows the GPC layout but counts one block per SM for these
+// kernels, while two are resident in practice; a cluster of c blocks at two per SM covers
+// ceil(c / 2) SMs, so the number asked for is that of clusters of ceil(c / 2) blocks (all SMs
+// for c <= 2).  Asked once per device, kernel and size; without a device (size queries on a
+// machine that has none) the plain quotient stands in.
 int cluster_capacity(bool wide, int c) {
   constexpr int kMaxDev = 64;
   static std::atomic<int> cache[kMaxDev][2][kMaxCluster + 1];
@@ -1250,25 +1253,33 @@ int cluster_capacity(bool wide, int c) {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { (void)cudaGetLastError(); return nominal; }
   const int have = cache[dev][wide ? 1 : 0][c].load(std::memory_order_relaxed);
   if (have > 0) return have;
-  const void* fn = wide ? reinterpret_cast<const void*>(tree_attention_wide_kernel)
-                        : reinterpret_cast<const void*>(tree_attention_ws_kernel);
-  const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
+  const int half = (c + 1) / 2;
   int n = 0;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(c * 64), 1, 1);
-  cfg.blockDim = dim3((unsigned)kWsThreads, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = (unsigned)c;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (rest::ensure_dynamic_smem(fn, wide ? 3 : 2, smem) != cudaSuccess ||
-      cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess || n <= 0) {
-    (void)cudaGetLastError();
-    return nominal;
+  if (half == 1) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      return nominal;
+    }
+  } else {
+    const void* fn = wide ? reinterpret_cast<const void*>(tree_attention_wide_kernel)
+                          : reinterpret_cast<const void*>(tree_attention_ws_kernel);
+    const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(half * 64), 1, 1);
+    cfg.blockDim = dim3((unsigned)kWsThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)half;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (rest::ensure_dynamic_smem(fn, wide ? 3 : 2, smem) != cudaSuccess ||
+        cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      return nominal;
+    }
   }
   cache[dev][wide ? 1 : 0][c].store(n, std::memory_order_relaxed);
   return n;
