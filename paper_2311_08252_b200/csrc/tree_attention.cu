@@ -65,6 +65,7 @@ struct AttnArgs {
   int B, H, group, N, Wm;
   int S;            // key splits per (context, head) = C * Sp
   int NBLK;         // 128-row query blocks per (context, head) in the wide kernel (else 1)
+  int unit0;        // first unit (context, head, row block) of this launch
   int pack;         // query heads per block in the wide kernel: 2 when N = 64 and heads share KV
   int q_slot[3], kv_slot[3];   // tensor-map coordinate index (1..3) of rows, head, batch
   int C;            // blocks per cluster
@@ -250,7 +251,7 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   volatile uint32_t* abort_word = reinterpret_cast<volatile uint32_t*>(smem + tc_bar_offset(1) + kBarAbort);
 
   int bid = blockIdx.x;
-  const int split = bid % a.S; bid /= a.S;
+  const int split = bid % a.S; bid = bid / a.S + a.unit0;
   const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 64-row block of the N draft rows
   const int h = bid % a.H;
   const int b = bid / a.H;
@@ -765,7 +766,7 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
   volatile uint32_t* abort_word = reinterpret_cast<volatile uint32_t*>(smem + kWideBarOffset + kBarAbort);
 
   int bid = blockIdx.x;
-  const int split = bid % a.S; bid /= a.S;
+  const int split = bid % a.S; bid = bid / a.S + a.unit0;
   const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 128-row block of the N draft rows
   // pack = 2 (N = 64, grouped KV heads): the block's 128 rows are the 64 draft rows of two query
   // heads that share one KV head, so that K/V stream is read once for both
@@ -1392,8 +1393,26 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   else
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 2, smem));
   if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
+  // Units that need no key split but do not fill a whole number of waves: the units of the last,
+  // partial wave go into a second launch with their key range cut over one cluster each, so that
+  // the wave ends after a fraction of a full block's time instead of a whole one.  Worth it when
+  // a block has enough tiles for the saving to exceed the merge and the launch.
+  const int64_t units = (int64_t)B * (H / a.pack) * a.NBLK;
+  const int64_t slots = 2 * (int64_t)cluster_capacity(wide, 1);
+  const int ntiles_max = (max_kv + kBN - 1) / kBN;
+  int64_t tail_units = 0;
+  int tail_c = 1;
+  if (a.S == 1 && a.pack == 1 && units > slots && ntiles_max >= 16) {
+    const int64_t r = units % slots;
+    if (r > 0) {
+      for (int c = kMaxCluster; c >= 2; --c) {
+        if (r <= cluster_capacity(wide, c)) { tail_units = r; tail_c = c; break; }
+      }
+    }
+  }
+  a.unit0 = 0;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(B * (H / a.pack) * a.NBLK * a.S), 1, 1);
+  cfg.gridDim = dim3((unsigned)((units - tail_units) * a.S), 1, 1);
   cfg.blockDim = dim3((unsigned)kWsThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
@@ -1420,9 +1439,21 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   else
     REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, a, tm_q, tm_k, tm_v));
   rest::count_launch();
+  if (tail_units > 0) {
+    AttnArgs t = a;
+    t.unit0 = (int)(units - tail_units);
+    t.S = tail_c; t.C = tail_c; t.Sp = 1;
+    cfg.gridDim = dim3((unsigned)(tail_units * tail_c), 1, 1);
+    attr[0].val.clusterDim.x = (unsigned)tail_c;
+    if (wide)
+      REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_wide_kernel, t, tm_q, tm_k, tm_v));
+    else
+      REST_CUDA_TRY(cudaLaunchKernelEx(&cfg, tree_attention_ws_kernel, t, tm_q, tm_k, tm_v));
+    rest::count_launch();
+  }
   if (a.Sp > 1) {
-    const int64_t units = (int64_t)B * H * N;
-    tree_attention_combine_kernel<<<(unsigned)((units + 3) / 4), 128, 0, st>>>(a);
+    const int64_t rows = (int64_t)B * H * N;
+    tree_attention_combine_kernel<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(a);
     rest::count_launch();
     REST_CUDA_TRY(cudaGetLastError());
   }

@@ -89,6 +89,15 @@ def test_grouped_heads_large_batch_two_query_heads_per_block():
     run_case(18, 75, 8, 64, 130, H_kv=1, Lcap=300)
 
 
+def test_partial_last_wave_goes_into_a_second_launch_with_key_splits():
+    # slightly more (context, head) units than fit at once, caches of 16+ tiles: the units of
+    # the partial last wave run as a second launch whose key range is cut over a cluster
+    rng = np.random.default_rng(4)
+    run_case(19, 10, 32, 64, 1100, kv_len=rng.integers(0, 1101, 10))
+    run_case(20, 5, 62, 128, 1300, kv_len=rng.integers(900, 1301, 5), max_depth=16)
+    run_case(21, 38, 8, 32, 1024)
+
+
 def test_wide_rows_ragged_batch_and_grouped_heads():
     # N > 64 with contexts far shorter than the longest one: some key splits get no tile at all
     run_case(13, 4, 8, 128, 900, Lcap=1100, H_kv=2, kv_len=[900, 1, 333, 64], n_nodes=77, max_depth=16)
