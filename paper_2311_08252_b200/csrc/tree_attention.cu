@@ -230,19 +230,6 @@ __device__ __forceinline__ void tma_load_box(uint32_t dst, const CUtensorMap* ma
       : "memory");
 }
 
-// the same box, only brought into L2 (no shared memory, no barrier): the later load of the box
-// then takes an L2 round trip instead of an HBM one
-__device__ __forceinline__ void tma_prefetch_box(const CUtensorMap* map, int c0, int row, int head, int batch,
-                                                 const int (&slot)[3]) {
-  const int c1 = slot[0] == 1 ? row : slot[1] == 1 ? head : batch;
-  const int c2 = slot[0] == 2 ? row : slot[1] == 2 ? head : batch;
-  const int c3 = slot[0] == 3 ? row : slot[1] == 3 ? head : batch;
-  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global [%0, {%1, %2, %3, %4}];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-               : "memory");
-}
-constexpr int kPrefetchAhead = 8;     // tiles requested into L2 ahead of the shared-memory ring
-
 __global__ void __launch_bounds__(kWsThreads, 2)
 tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
                          const __grid_constant__ CUtensorMap tm_k,
@@ -350,22 +337,10 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       mbar_expect_tx(bars + kBarQFull, (uint32_t)kQBlockBytes);
       tma_load_box(sQ, &tm_q, 0, row0, h, b, a.q_slot, bars + kBarQFull);
       tma_load_box(sQ + 64 * 128, &tm_q, 64, row0, h, b, a.q_slot, bars + kBarQFull);
-      // The ring holds two tiles, so a block's own loads cover one HBM round trip per two
-      // tiles; tiles further ahead are requested into L2 right away, and their ring loads then
-      // complete in an L2 round trip.
-      auto prefetch_tile = [&](int it) {
-        const int key0 = (t0 + it) * kBN;
-        tma_prefetch_box(&tm_k, 0, key0, hk, b, a.kv_slot);
-        tma_prefetch_box(&tm_k, 64, key0, hk, b, a.kv_slot);
-        tma_prefetch_box(&tm_v, 0, key0, hk, b, a.kv_slot);
-        tma_prefetch_box(&tm_v, 64, key0, hk, b, a.kv_slot);
-      };
-      for (int it = 2; it < nt && it < kPrefetchAhead; ++it) prefetch_tile(it);
       int issued_k = 0, issued_v = 0;
       for (int it = 0; it < nt; ++it) {
         const int slot = it & 1, key0 = (t0 + it) * kBN;
         const uint32_t free_parity = (uint32_t)(((it >> 1) + 1) & 1);
-        if (it + kPrefetchAhead < nt) prefetch_tile(it + kPrefetchAhead);
         if (it >= 2 && !mbar_wait_abortable(bars + kBarKFree + slot * 8, free_parity, abort_word)) break;
         mbar_expect_tx(bars + kBarKFull + slot * 8, (uint32_t)kTileBytes);
         tma_load_box(sK + slot * kTileBytes, &tm_k, 0, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
@@ -860,22 +835,10 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       tma_load_box(sQ + 64 * 128, &tm_q, 0, r1, h1, b, a.q_slot, bars + kBarQFull);
       tma_load_box(sQ + 128 * 128, &tm_q, 64, row0, h0, b, a.q_slot, bars + kBarQFull);
       tma_load_box(sQ + 192 * 128, &tm_q, 64, r1, h1, b, a.q_slot, bars + kBarQFull);
-      // The ring holds two tiles, so a block's own loads cover one HBM round trip per two
-      // tiles; tiles further ahead are requested into L2 right away, and their ring loads then
-      // complete in an L2 round trip.
-      auto prefetch_tile = [&](int it) {
-        const int key0 = (t0 + it) * kBN;
-        tma_prefetch_box(&tm_k, 0, key0, hk, b, a.kv_slot);
-        tma_prefetch_box(&tm_k, 64, key0, hk, b, a.kv_slot);
-        tma_prefetch_box(&tm_v, 0, key0, hk, b, a.kv_slot);
-        tma_prefetch_box(&tm_v, 64, key0, hk, b, a.kv_slot);
-      };
-      for (int it = 2; it < nt && it < kPrefetchAhead; ++it) prefetch_tile(it);
       int issued_k = 0, issued_v = 0;
       for (int it = 0; it < nt; ++it) {
         const int slot = it & 1, key0 = (t0 + it) * kBN;
         const uint32_t free_parity = (uint32_t)(((it >> 1) + 1) & 1);
-        if (it + kPrefetchAhead < nt) prefetch_tile(it + kPrefetchAhead);
         if (it >= 2 && !mbar_wait_abortable(bars + kBarKFree + slot * 8, free_parity, abort_word)) break;
         mbar_expect_tx(bars + kBarKFull + slot * 8, (uint32_t)kTileBytes);
         tma_load_box(sK + slot * kTileBytes, &tm_k, 0, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
