@@ -385,8 +385,13 @@ def main():
     # graph replay copies them in, runs the step and copies the results out, then the host waits.
     h_ctx = torch.empty((B, w.Lc), dtype=torch.int32).pin_memory()
     h_ver = torch.empty((B, N + 1), dtype=torch.int32).pin_memory()
-    h_q = [q.cpu().pin_memory() for q in qs]
-    h_out = [torch.empty((B, N, H, D), dtype=torch.bfloat16).pin_memory() for _ in range(layers)]
+    # queries and outputs of all layers in one buffer each, copied in groups of layers: fewer
+    # cross-stream dependencies in the graph than one copy per layer
+    group = 4
+    q_all = torch.stack(qs)                                   # [layers, B, N, H, D] on the device
+    out_all = torch.empty((layers, B, N, H, D), dtype=torch.bfloat16, device=dev)
+    h_q = q_all.cpu().pin_memory()
+    h_out = torch.empty((layers, B, N, H, D), dtype=torch.bfloat16).pin_memory()
     h_tree = {k: torch.empty_like(getattr(tree, k), device="cpu").pin_memory()
               for k in ("tokens", "parents", "depth", "pos_ids", "mask", "n_nodes", "match_n")}
     h_acc = [torch.empty_like(a, device="cpu").pin_memory() for a in acc]
@@ -394,12 +399,12 @@ def main():
     s_ver = torch.empty((B, N + 1), dtype=torch.int32, device=dev)
     h2d = s_ctx.numel() * 4 + s_ver.numel() * 4 + sum(q.numel() * 2 for q in qs)
     d2h = sum(t.numel() * t.element_size() for t in h_tree.values()) + \
-        sum(t.numel() * 4 for t in h_acc) + sum(o.numel() * 2 for o in h_out)
+        sum(t.numel() * 4 for t in h_acc) + h_out.numel() * 2
     ctx_t, ver_t = torch.from_numpy(ctx_np), torch.from_numpy(ver_np)
 
     # Two copy streams run beside the compute stream inside the graph: all inputs go in on one
-    # (layer l's attention waits only for its own queries), each layer's output goes out on the
-    # other as soon as that layer is done.
+    # (a layer's attention waits only for its own group of queries), each group of layers'
+    # outputs goes out on the other as soon as the group is done.
     s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
 
     def e2e_calls(_):
@@ -412,22 +417,25 @@ def main():
             s_ver.copy_(h_ver, non_blocking=True)
             in_ready = torch.cuda.Event()
             in_ready.record(s_in)
-            for layer in range(layers):
-                qs[layer].copy_(h_q[layer], non_blocking=True)
+            for l0 in range(0, layers, group):
+                q_all[l0:l0 + group].copy_(h_q[l0:l0 + group], non_blocking=True)
                 ev = torch.cuda.Event()
                 ev.record(s_in)
                 q_ready.append(ev)
         main.wait_event(in_ready)
         rest.rest_draft(ds, s_ctx, d_ctx_len, out=tree, **dkw)
         for layer in range(layers):
-            main.wait_event(q_ready[layer])
-            rest.rest_tree_attention(qs[layer], ks[layer], vs[layer], d_kv_len, tree.mask, scale,
-                                     max_kv=L + N, out=outs[layer], workspace=ws)
-            done = torch.cuda.Event()
-            done.record(main)
-            s_out.wait_event(done)
-            with torch.cuda.stream(s_out):
-                h_out[layer].copy_(outs[layer], non_blocking=True)
+            if layer % group == 0:
+                main.wait_event(q_ready[layer // group])
+            rest.rest_tree_attention(q_all[layer], ks[layer], vs[layer], d_kv_len, tree.mask, scale,
+                                     max_kv=L + N, out=out_all[layer], workspace=ws)
+            if layer % group == group - 1 or layer == layers - 1:
+                l0 = layer - layer % group
+                done = torch.cuda.Event()
+                done.record(main)
+                s_out.wait_event(done)
+                with torch.cuda.stream(s_out):
+                    h_out[l0:layer + 1].copy_(out_all[l0:layer + 1], non_blocking=True)
         rest.rest_accept(tree.tokens, tree.parents, tree.n_nodes, s_ver, w.m, out=acc)
         for k, t in h_tree.items():
             t.copy_(getattr(tree, k), non_blocking=True)
