@@ -148,7 +148,9 @@ rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params
  *   d_kv_len  int32[B], 0 <= L and L + N <= rows available
  *   max_kv    upper bound on L + N over the batch (sizes the split of the key range)
  *   d_mask    uint32[B,N,ceil(N/32)] as written by rest_draft
- *   d_lse     optional float[B,H,N]: log of the softmax denominator (natural log, of scaled scores)
+ *   d_lse     optional float[B,H,N]: log of the softmax denominator (natural log, of scaled
+ *             scores); with N > 64 the denominator sums the bf16-rounded probabilities that the
+ *             output is built from, so it carries bf16 precision (a few 1e-3 absolute)
  *   d_ws      scratch of rest_tree_attention_workspace_bytes() bytes
  *   scale     softmax scale, finite and > 0 (else REST_INVALID_ARG)
  *   Limits: D = 128; N in {16, 32, 48, ..., 256}; H % H_kv == 0.

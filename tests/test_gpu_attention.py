@@ -181,3 +181,46 @@ def test_attention_on_drafted_masks_full_head_count():
                                 ref_d["mask"], scale)
     max_abs, max_rel = attention_errors(out[:, :, hs], ref)
     assert max_abs <= MAX_ABS and max_rel <= MAX_REL, (max_abs, max_rel)
+
+
+def test_random_shapes_against_the_oracle():
+    """Seeded sweep over batch sizes (also just around whole waves of blocks), head groupings,
+    tree sizes, ragged prefixes and scales.  Outputs may reach magnitudes where rounding to bf16
+    alone costs 2^-8 |x|, so the absolute bound is 1e-2 + 2^-8 |reference|; the log-sum-exp bound
+    is 5e-3 (with more than 64 draft rows the denominator sums bf16-rounded probabilities)."""
+    rng = np.random.default_rng(20231108)
+    done = 0
+    while done < 60:
+        N = int(rng.choice([16, 32, 48, 64, 64, 64, 80, 128, 128, 192, 256]))
+        H_kv = int(rng.integers(1, 9))
+        H = H_kv * int(rng.choice([1, 1, 1, 2, 4]))
+        mode = int(rng.integers(0, 3))
+        if mode == 0:
+            B = int(rng.integers(1, 4))
+        elif mode == 1:
+            B = max(1, int(rng.choice([148, 296, 300, 320, 600])) // H + int(rng.integers(0, 2)))
+        else:
+            B = int(rng.integers(1, 40))
+        L = int(rng.choice([0, 1, 63, 64, 65, 200, 513, 1024, 1100, 2048]))
+        if B * H * (L + N) * N > 2e8:
+            continue
+        kv_len = rng.integers(0, L + 1, B).astype(np.int32)
+        if rng.random() < 0.5:
+            kv_len[:] = L
+        Lcap = L + N + int(rng.choice([0, 0, 7, 64]))
+        q, k, v = datagen.make_qkv(int(rng.integers(1, 1 << 30)), B, H, N, 128, Lcap, H_kv=H_kv)
+        masks = np.stack([datagen.make_random_tree(int(rng.integers(1, 1 << 30)), N, int(rng.integers(1, 17)),
+                                                   int(rng.integers(1, N + 1)))[2] for _ in range(B)])
+        scale = float(rng.choice([1 / math.sqrt(128), 0.05, 0.2]))
+        ref, ref_lse = oracle.tree_attention(bits(q), bits(k), bits(v), kv_len, masks, scale, H_kv=H_kv,
+                                             want_lse=True)
+        lse = torch.empty((B, H, N), dtype=torch.float32, device="cuda:0")
+        out = rest.rest_tree_attention(q.cuda(), k.cuda(), v.cuda(), to_dev(kv_len), to_dev(masks), scale,
+                                       lse=lse)
+        torch.cuda.synchronize()
+        what = dict(B=B, H=H, H_kv=H_kv, N=N, L=L, Lcap=Lcap, scale=scale)
+        err = np.abs(out.float().cpu().numpy().astype(np.float64) - ref)
+        assert (err <= MAX_ABS + np.abs(ref) / 256.0).all(), what
+        assert attention_errors(out, ref)[1] <= MAX_REL, what
+        assert np.abs(lse.cpu().numpy().astype(np.float64) - ref_lse).max() <= 5e-3, what
+        done += 1
