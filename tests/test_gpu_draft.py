@@ -132,3 +132,38 @@ def test_bad_context_tokens_and_corrupt_datastore():
     got, _ = gpu_draft(Z, bad, 1, np.zeros((1, 20), np.int32), [20], m=3, N=4)
     assert got["status"].tolist() == [2] and got["n_nodes"].tolist() == [0]
     assert (got["tokens"] == -1).all()
+
+
+def test_random_parameters_against_the_oracle():
+    """Seeded sweep: random / periodic / self-repeating streams of 1 to 200 k tokens over alphabets
+    of 2 to 32000 symbols, both suffix-array widths, every suffix-length window, K from 1 to the
+    maximum, m and N over their whole ranges, both sampling modes, ragged context lengths."""
+    rng = np.random.default_rng(20231108)
+    for case in range(400):
+        vocab = int(rng.choice([2, 3, 4, 8, 50, 32000]))
+        n_tok = int(rng.choice([1, 2, 5, 33, 100, 1000, 5000, 40000, 200000]))
+        kind = int(rng.integers(0, 3))
+        if kind == 0:
+            T = rng.integers(0, vocab, n_tok)
+        elif kind == 1:
+            T = np.tile(rng.integers(0, vocab, int(rng.integers(1, 7))), n_tok)[:n_tok]
+        else:
+            T = rng.integers(0, vocab, n_tok)
+            if n_tok > 50:
+                T[n_tok // 2:] = T[:n_tok - n_tok // 2]
+        T = T.astype(np.int32)
+        sa = datagen.build_suffix_array(T, vocab, W=32, sa_bytes=int(rng.choice([4, 8])))
+        B, Lc = int(rng.integers(1, 50)), int(rng.integers(1, 40))
+        ctx = rng.integers(0, vocab, (B, Lc)).astype(np.int32)
+        for b in range(0, B, 2):
+            if n_tok > Lc:
+                p = int(rng.integers(0, n_tok - Lc + 1))
+                ctx[b] = T[p:p + Lc]
+        ctx_len = rng.integers(0, Lc + 1, B).astype(np.int32)
+        n_max = int(rng.integers(1, 17))
+        kw = dict(K=int(rng.choice([1, 7, 100, 5000, 32768])), m=int(rng.integers(1, 17)),
+                  N=int(rng.choice([1, 16, 64, 100, 128, 256])), n_max=n_max,
+                  n_min=int(rng.integers(1, n_max + 1)), sample_mode=int(rng.integers(0, 2)))
+        ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
+        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, **kw)
+        assert_draft_equal(got, ref, f"case {case}: vocab {vocab}, {n_tok} tokens, {kw}")
