@@ -224,3 +224,19 @@ def test_random_shapes_against_the_oracle():
         assert attention_errors(out, ref)[1] <= MAX_REL, what
         assert np.abs(lse.cpu().numpy().astype(np.float64) - ref_lse).max() <= 5e-3, what
         done += 1
+
+
+def test_split_plans_fit_the_device():
+    for B, H, N, L in [(1, 32, 64, 2048), (1, 37, 64, 8192), (3, 32, 64, 4096), (1, 1, 64, 16384),
+                       (1, 32, 128, 2048), (1, 4, 256, 8192), (256, 32, 64, 4096), (1, 2, 64, 100)]:
+        p = rest.tree_attention_plan(B, H, N, 128, L + N)
+        ntiles = (L + N + 63) // 64
+        units = B * H * (1 if N <= 64 else (N + 127) // 128)
+        assert p["splits"] == p["cluster"] * p["clusters_per_unit"]
+        assert 1 <= p["cluster"] <= 8 and p["splits"] <= max(ntiles, 1)
+        if p["cluster"] > 1:
+            assert units * p["clusters_per_unit"] <= p["capacity"], (B, H, N, L, p)
+        ws = rest.tree_attention_workspace_bytes(B, H, N, 128, L + N)
+        assert (ws == 0) == (p["clusters_per_unit"] == 1)
+        if ws:
+            assert ws == B * H * p["clusters_per_unit"] * N * 130 * 4
