@@ -2,8 +2,11 @@
  * rest.h - C ABI of the GPU hot path of one REST decoding step
  * (Retrieval-Based Speculative Decoding, arXiv 2311.08252).
  *
- * Draft side:   rest_datastore_create, rest_draft          (Sec. 3.2, Algorithms 1 and 2)
+ * Set-up:       rest_suffix_array_build, rest_datastore_create  (Sec. 3.2, datastore construction)
+ * Draft side:   rest_draft                                 (Sec. 3.2, Algorithms 1 and 2)
  * Verify side:  rest_tree_attention, rest_accept           (Sec. 3.2, draft verification / acceptance)
+ * Between steps: rest_kv_commit                            (the accepted path joins the prefix)
+ * Aids:         rest_tree_attention_plan, rest_probe_dependent_reads, rest_device_error_flags
  *
  * Conventions
  *   - Every pointer named d_* is a DEVICE pointer owned by the caller.  The library borrows
