@@ -252,12 +252,11 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
 
   int bid = blockIdx.x;
   const int split = bid % a.S; bid = bid / a.S + a.unit0;
-  const int rblk = bid % a.NBLK; bid /= a.NBLK;     // which 64-row block of the N draft rows
   const int h = bid % a.H;
   const int b = bid / a.H;
   const int hk = h / a.group;
-  const int row0 = rblk * 64;                        // first draft row of this thread block
-  const int Nl = min(64, N - row0);                  // its number of real rows
+  constexpr int row0 = 0;                            // this kernel serves N <= 64: one row block
+  const int Nl = N;                                  // its number of real rows
 
   // Programmatic dependent launch: the next kernel in the stream may start its own set-up now;
   // this kernel touches no global memory until the one before it has fully completed.
