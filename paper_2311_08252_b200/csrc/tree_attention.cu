@@ -336,28 +336,30 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       mbar_expect_tx(bars + kBarQFull, (uint32_t)kQBlockBytes);
       tma_load_box(sQ, &tm_q, 0, row0, h, b, a.q_slot, bars + kBarQFull);
       tma_load_box(sQ + 64 * 128, &tm_q, 64, row0, h, b, a.q_slot, bars + kBarQFull);
-      int issued_k = 0, issued_v = 0;
+    }
+    // K tiles by lane 0, V tiles by lane 1: a K slot frees as soon as its Q K^T has run, a V slot
+    // only after the softmax and P V of its tile; one thread issuing both in turn would hold the
+    // next K tile back behind the wait for a V slot.
+    if (lane < 2) {
+      const bool is_v = lane == 1;
+      const uint32_t ring = is_v ? sV : sK;
+      const CUtensorMap* map = is_v ? &tm_v : &tm_k;
+      const uint32_t full = bars + (is_v ? kBarVFull : kBarKFull), free_ = bars + (is_v ? kBarVFree : kBarKFree);
+      int issued = 0;
       for (int it = 0; it < nt; ++it) {
         const int slot = it & 1, key0 = (t0 + it) * kBN;
         const uint32_t free_parity = (uint32_t)(((it >> 1) + 1) & 1);
-        if (it >= 2 && !mbar_wait_abortable(bars + kBarKFree + slot * 8, free_parity, abort_word)) break;
-        mbar_expect_tx(bars + kBarKFull + slot * 8, (uint32_t)kTileBytes);
-        tma_load_box(sK + slot * kTileBytes, &tm_k, 0, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
-        tma_load_box(sK + slot * kTileBytes + 64 * 128, &tm_k, 64, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
-        ++issued_k;
-        if (it >= 2 && !mbar_wait_abortable(bars + kBarVFree + slot * 8, free_parity, abort_word)) break;
-        mbar_expect_tx(bars + kBarVFull + slot * 8, (uint32_t)kTileBytes);
-        tma_load_box(sV + slot * kTileBytes, &tm_v, 0, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
-        tma_load_box(sV + slot * kTileBytes + 64 * 128, &tm_v, 64, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
-        ++issued_v;
+        if (it >= 2 && !mbar_wait_abortable(free_ + slot * 8, free_parity, abort_word)) break;
+        mbar_expect_tx(full + slot * 8, (uint32_t)kTileBytes);
+        tma_load_box(ring + slot * kTileBytes, map, 0, key0, hk, b, a.kv_slot, full + slot * 8);
+        tma_load_box(ring + slot * kTileBytes + 64 * 128, map, 64, key0, hk, b, a.kv_slot, full + slot * 8);
+        ++issued;
       }
       if (*abort_word != 0u) {
         // giving up: let the copies already in flight land before this block goes away
-        mbar_wait(bars + kBarQFull, 0u);
-        for (int it = max(0, issued_k - 2); it < issued_k; ++it)
-          mbar_wait(bars + kBarKFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
-        for (int it = max(0, issued_v - 2); it < issued_v; ++it)
-          mbar_wait(bars + kBarVFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
+        if (!is_v) mbar_wait(bars + kBarQFull, 0u);
+        for (int it = max(0, issued - 2); it < issued; ++it)
+          mbar_wait(full + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
       }
     }
   } else if (warp == 5) {
@@ -834,28 +836,30 @@ tree_attention_wide_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
       tma_load_box(sQ + 64 * 128, &tm_q, 0, r1, h1, b, a.q_slot, bars + kBarQFull);
       tma_load_box(sQ + 128 * 128, &tm_q, 64, row0, h0, b, a.q_slot, bars + kBarQFull);
       tma_load_box(sQ + 192 * 128, &tm_q, 64, r1, h1, b, a.q_slot, bars + kBarQFull);
-      int issued_k = 0, issued_v = 0;
+    }
+    // K tiles by lane 0, V tiles by lane 1: a K slot frees as soon as its Q K^T has run, a V slot
+    // only after the softmax and P V of its tile; one thread issuing both in turn would hold the
+    // next K tile back behind the wait for a V slot.
+    if (lane < 2) {
+      const bool is_v = lane == 1;
+      const uint32_t ring = is_v ? sV : sK;
+      const CUtensorMap* map = is_v ? &tm_v : &tm_k;
+      const uint32_t full = bars + (is_v ? kBarVFull : kBarKFull), free_ = bars + (is_v ? kBarVFree : kBarKFree);
+      int issued = 0;
       for (int it = 0; it < nt; ++it) {
         const int slot = it & 1, key0 = (t0 + it) * kBN;
         const uint32_t free_parity = (uint32_t)(((it >> 1) + 1) & 1);
-        if (it >= 2 && !mbar_wait_abortable(bars + kBarKFree + slot * 8, free_parity, abort_word)) break;
-        mbar_expect_tx(bars + kBarKFull + slot * 8, (uint32_t)kTileBytes);
-        tma_load_box(sK + slot * kTileBytes, &tm_k, 0, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
-        tma_load_box(sK + slot * kTileBytes + 64 * 128, &tm_k, 64, key0, hk, b, a.kv_slot, bars + kBarKFull + slot * 8);
-        ++issued_k;
-        if (it >= 2 && !mbar_wait_abortable(bars + kBarVFree + slot * 8, free_parity, abort_word)) break;
-        mbar_expect_tx(bars + kBarVFull + slot * 8, (uint32_t)kTileBytes);
-        tma_load_box(sV + slot * kTileBytes, &tm_v, 0, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
-        tma_load_box(sV + slot * kTileBytes + 64 * 128, &tm_v, 64, key0, hk, b, a.kv_slot, bars + kBarVFull + slot * 8);
-        ++issued_v;
+        if (it >= 2 && !mbar_wait_abortable(free_ + slot * 8, free_parity, abort_word)) break;
+        mbar_expect_tx(full + slot * 8, (uint32_t)kTileBytes);
+        tma_load_box(ring + slot * kTileBytes, map, 0, key0, hk, b, a.kv_slot, full + slot * 8);
+        tma_load_box(ring + slot * kTileBytes + 64 * 128, map, 64, key0, hk, b, a.kv_slot, full + slot * 8);
+        ++issued;
       }
       if (*abort_word != 0u) {
         // giving up: let the copies already in flight land before this block goes away
-        mbar_wait(bars + kBarQFull, 0u);
-        for (int it = max(0, issued_k - 2); it < issued_k; ++it)
-          mbar_wait(bars + kBarKFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
-        for (int it = max(0, issued_v - 2); it < issued_v; ++it)
-          mbar_wait(bars + kBarVFull + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
+        if (!is_v) mbar_wait(bars + kBarQFull, 0u);
+        for (int it = max(0, issued - 2); it < issued; ++it)
+          mbar_wait(full + (it & 1) * 8, (uint32_t)((it >> 1) & 1));
       }
     }
   } else if (warp == 5) {
