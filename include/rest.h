@@ -50,7 +50,15 @@ enum {
   REST_CTX_INTERNAL = 3
 };
 
-enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1 };
+enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1, REST_SAMPLE_MASK = 0xFF };
+/* How rest_draft searches the suffix array, OR-ed into sample_mode; the results are the same
+ * either way.  SINGLE: all suffix lengths at once, 32 probes per round, 512 threads per context
+ * (fewest dependent reads, the fastest single context).  BATCHED: 256 threads per context, six
+ * or seven searches instead of fifteen (the lengths that match are n_min ... n* without a gap)
+ * and eight probes per round once the probes leave L2: more dependent rounds, fewer random
+ * DRAM reads, twice the contexts in flight.  AUTO picks BATCHED when the call has at least
+ * 16 contexts per SM. */
+enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 0x100, REST_SEARCH_BATCHED = 0x200 };
 enum { REST_DS_VALIDATE = 1u };
 
 /* Limits of this implementation. */

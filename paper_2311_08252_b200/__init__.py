@@ -22,6 +22,9 @@ _SO = os.path.join(_HERE, "librest.so")
 REST_OK = 0
 REST_SAMPLE_STRIDED = 0
 REST_SAMPLE_FIRST_K = 1
+REST_SEARCH_AUTO = 0
+REST_SEARCH_SINGLE = 0x100
+REST_SEARCH_BATCHED = 0x200
 REST_DS_VALIDATE = 1
 
 EXPORTS = (
@@ -209,10 +212,11 @@ def alloc_draft_output(B: int, N: int, device) -> DraftOutput:
 
 
 def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=64,
-               sample_mode=REST_SAMPLE_STRIDED, out: DraftOutput | None = None, stream=None
-               ) -> DraftOutput:
+               sample_mode=REST_SAMPLE_STRIDED, out: DraftOutput | None = None, stream=None,
+               search=REST_SEARCH_AUTO) -> DraftOutput:
     """Draft trees for contexts ctx int32[B, Lc] (row b holds ctx_len[b] tokens).  The mask
-    tensor is int32 storage of the uint32 words."""
+    tensor is int32 storage of the uint32 words.  `search` (REST_SEARCH_*) picks the
+    single-context or the batched suffix-array search; the results do not depend on it."""
     L = lib()
     _dev_i32(ctx_len, "ctx_len")
     import torch
@@ -221,7 +225,7 @@ def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=6
     B = ctx.shape[0]
     if out is None:
         out = alloc_draft_output(B, N, ctx.device)
-    prm = _Params(n_max, n_min, K, m, N, sample_mode)
+    prm = _Params(n_max, n_min, K, m, N, sample_mode | search)
     rc = L.rest_draft(ds._h, ctypes.byref(prm), ctx.data_ptr(), ctx.stride(0), ctx_len.data_ptr(), B,
                       out.tokens.data_ptr(), out.parents.data_ptr(), out.depth.data_ptr(),
                       out.pos_ids.data_ptr(), out.mask.data_ptr(), out.n_nodes.data_ptr(),

@@ -31,6 +31,15 @@ constexpr int kMaxN = REST_MAX_N;
 constexpr int kHistHi = 1056;   // bins of key >> 10, key < 2^20 + 32
 constexpr int kHistLo = 1024;
 constexpr unsigned kFull = 0xFFFFFFFFu;
+// Batched path (calls with far more contexts than the GPU holds at once): threads per block,
+// lanes per probe round once the probes leave L2, the number of 32-wide rounds before that,
+// and whether the suffix lengths are searched in two steps.  Measured at 4096 contexts on a
+// 100 M-token datastore: 512 threads, every length, 32 lanes 565 us; 256 threads with 4 or 8
+// lanes 533 / 509 us; 256 threads, 8 lanes, two steps 474 us; 128 threads were slower again.
+constexpr int kTpThreads = 256;
+constexpr int kTpArity = 8;
+constexpr bool kTpStaged = true;
+constexpr int kWideRounds = 3;
 
 struct DraftArgs {
   const int32_t* T;
@@ -82,22 +91,36 @@ __device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* _
 // `next_gt` (STRICT = false only): the first slot that compares greater, when the last round's
 // probes happen to show it (the run of equal slots ends inside the last 32 probed slots, or runs
 // up to a slot already known to be greater); -1 when it is not known.
-template <typename SaT, bool STRICT>
+//
+// A = 32: every round all 32 lanes probe (fewest dependent rounds: the single-context path).
+// A < 32: only the first WIDE rounds are 32 wide (a search over the whole array: their probe
+// positions are the top of a fixed 33-ary tree, the same for every context, and stay in L2); the rounds
+// below them, whose probes go to DRAM, use A lanes (A probes cut the interval into A + 1
+// parts), which costs more dependent rounds but far fewer random DRAM reads per search.
+template <typename SaT, bool STRICT, int A = 32, int WIDE = kWideRounds>
 __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
                                    int64_t n_tokens, int64_t lo, int64_t hi, const int (&q)[16],
                                    int n, int lane, bool& eq, bool& bad, int64_t* next_gt = nullptr) {
-  while (hi - lo > 32) {
+  // floor(2^64 / (A + 1))
+  constexpr unsigned long long kInv = A == 32 ? 0x07C1F07C1F07C1F0ull : ~0ull / (unsigned long long)(A + 1);
+  int round = 0;
+  while (hi - lo > A) {
     int64_t size = hi - lo;
-    // 32 probes that cut the interval into 33 parts: floor((lane + 1) * size * floor(2^64 / 33)
-    // / 2^64) is at most (lane + 1) * size / 33, increasing in the lane, and below size; which
-    // slots are probed does not change the answer, only how fast the interval shrinks
+    const bool wide = A == 32 || (round < WIDE && size > 32);
+    ++round;
+    // P probes that cut the interval into P + 1 parts: floor((lane + 1) * size * floor(2^64 /
+    // (P + 1)) / 2^64) is at most (lane + 1) * size / (P + 1), non-decreasing in the lane, and
+    // below size; which slots are probed does not change the answer, only how fast the
+    // interval shrinks
+    const int last = wide ? 31 : A - 1;
     int64_t pos = lo + (int64_t)__umul64hi((unsigned long long)(lane + 1) * (unsigned long long)size,
-                                           0x07C1F07C1F07C1F0ull);
-    int c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
+                                           wide ? 0x07C1F07C1F07C1F0ull : kInv);
+    int c = 1;
+    if (lane <= last) c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
     bool t = STRICT ? (c > 0) : (c >= 0);
-    unsigned b = __ballot_sync(kFull, t);
+    unsigned b = __ballot_sync(kFull, t && lane <= last);
     if (b == 0) {
-      lo = __shfl_sync(kFull, pos, 31) + 1;
+      lo = __shfl_sync(kFull, pos, last) + 1;
     } else {
       int f = __ffs(b) - 1;
       int64_t pf = __shfl_sync(kFull, pos, f);
@@ -199,8 +222,15 @@ struct Smem {
   uint32_t hist_lo[kHistLo];
 };
 
-template <typename SaT>
-__global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
+// TP = false: the single-context path, tuned for the fewest dependent reads.  TP = true: the
+// batched path, for calls with more contexts than the GPU holds at once; the same results by
+// fewer random DRAM reads per context (see phase 1).
+template <typename SaT, bool TP>
+__global__ void __launch_bounds__(TP ? kTpThreads : kThreads, TP ? 1024 / kTpThreads : 2)
+rest_draft_kernel(DraftArgs a) {
+  constexpr int NT = TP ? kTpThreads : kThreads;   // threads of this block
+  constexpr int NW = NT / 32;
+  static_assert(NT % 32 == 0 && NT >= 64, "whole warps; at least kMaxM + 2 threads");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& s = *reinterpret_cast<Smem*>(smem_raw);
   uint16_t* lenlcp = reinterpret_cast<uint16_t*>(smem_raw + sizeof(Smem));          // [kcap]
@@ -219,11 +249,11 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   const int clen = a.ctx_len[b];
   const int32_t* ctx = a.ctx + (int64_t)b * a.ctx_stride;
 
-  // Unused-slot defaults; thread i owns slot i for the whole kernel.
-  if (tid < N) {
-    int64_t o = (int64_t)b * N + tid;
+  // Unused-slot defaults; thread i owns slots i, i + NT, ... for the whole kernel.
+  for (int i = tid; i < N; i += NT) {
+    int64_t o = (int64_t)b * N + i;
     a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
-    for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (tid >> 5)) ? (1u << (tid & 31)) : 0u;
+    for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (i >> 5)) ? (1u << (i & 31)) : 0u;
     if (a.node_count) a.node_count[o] = 0;
   }
   const int nq = min(a.n_max, max(clen, 0));   // context tokens that can take part
@@ -231,8 +261,8 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; }
   if (tid <= kMaxM) s.e1[tid] = 0;
   if (tid <= kMaxM + 1) s.e1diff[tid] = 0;
-  for (int i = tid; i < kHistHi; i += kThreads) s.hist_hi[i] = 0;
-  for (int i = tid; i < kHistLo; i += kThreads) s.hist_lo[i] = 0;
+  for (int i = tid; i < kHistHi; i += NT) s.hist_hi[i] = 0;
+  for (int i = tid; i < kHistLo; i += NT) s.hist_lo[i] = 0;
   __syncthreads();
   if (tid < nq) {
     int t = ctx[clen - nq + tid];
@@ -251,17 +281,39 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   // ---- phase 1: search --------------------------------------------------------------
   // 1a: lower bound of every suffix length, one warp each.  ub = -1 marks "matches, end of the
   // run not known yet".
-  {
-    const int n = a.n_min + warp;
-    if (n <= nq) {
-      int q[16];
+  constexpr int kArity = TP ? kTpArity : 32;
+  auto lower_bound_of = [&](int n) {     // executed by one whole warp
+    int q[16];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
-      bool bad = false, eq = false;
-      int64_t next_gt = -1;
-      int64_t lb = warp_first_true<SaT, false>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
-      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
-      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_tokens) ? next_gt : lb; }
+    for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
+    bool bad = false, eq = false;
+    int64_t next_gt = -1;
+    int64_t lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
+    if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+    if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_tokens) ? next_gt : lb; }
+  };
+  if constexpr (!TP || !kTpStaged) {
+    for (int n = a.n_min + warp; n <= nq; n += NW) lower_bound_of(n);   // one length per warp when NW = 16
+  } else {
+    // If the suffix of length n occurs in the datastore, so does the one of length n - 1 (the
+    // same occurrence, one token later): the lengths that match are n_min ... n* without a
+    // gap.  Two steps of three or four searches find n* among up to 16 lengths: every fourth length
+    // first, then the three lengths above the longest of those that matched.  Lengths never
+    // searched keep lb = ub = 0, "no match", which is what they are.
+    const int nlen = nq - a.n_min + 1;
+    if (warp < 4) {
+      const int i = 3 + 4 * warp;
+      if (i < nlen) lower_bound_of(a.n_min + i);
+    }
+    __syncthreads();
+    int first = 0;
+    for (int w = 3; w >= 0; --w) {
+      const int i = 3 + 4 * w;
+      if (i < nlen && s.ub[a.n_min + i] != s.lb[a.n_min + i]) { first = i + 1; break; }
+    }
+    if (warp < 3) {
+      const int i = first + warp;
+      if (i < nlen) lower_bound_of(a.n_min + i);
     }
   }
   __syncthreads();
@@ -272,30 +324,37 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   // bound did not already show where the run ends (shorter lengths match far more slots and
   // would need the most rounds: they are never looked at again)
   if (n_win != 0 && s.ub[n_win] < 0) {       // block-uniform
-    if (warp == n_win - a.n_min) {
+    if (warp == (n_win - a.n_min) % NW) {
       const int n = n_win;
       int q[16];
 #pragma unroll
       for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
       bool bad = false;
       const int64_t lb = s.lb[n];
-      // gallop: lane l probes lb + 2^l
-      int64_t pos = lb + ((int64_t)1 << lane);
-      bool t = true;
-      if (pos < n_tokens) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
-      unsigned bal = __ballot_sync(kFull, t);
+      // gallop: slot lb + 2^e for e = 0 ... 31, all at once or kArity exponents per round; f =
+      // the first exponent whose slot compares greater or lies past the end (-1: none)
+      int f = -1;
+      for (int g = 0; g < 32 / kArity; ++g) {
+        bool t = false;
+        if (lane < kArity) {
+          const int64_t pos = lb + ((int64_t)1 << (g * kArity + lane));
+          t = true;
+          if (pos < n_tokens) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
+        }
+        const unsigned bal = __ballot_sync(kFull, t);
+        if (bal != 0) { f = g * kArity + __ffs(bal) - 1; break; }
+      }
       int64_t lo2, hi2 = n_tokens;
       bool eq2 = false;
-      if (bal == 0) {
+      if (f < 0) {
         lo2 = lb + ((int64_t)1 << 31) + 1;
       } else {
-        int f = __ffs(bal) - 1;
         int64_t pf = lb + ((int64_t)1 << f);
         hi2 = pf < n_tokens ? pf : n_tokens;
         lo2 = f > 0 ? lb + ((int64_t)1 << (f - 1)) + 1 : lb + 1;
       }
       if (lo2 > hi2) lo2 = hi2;
-      const int64_t ub = warp_first_true<SaT, true>(T, sa, n_tokens, lo2, hi2, q, n, lane, eq2, bad);
+      const int64_t ub = warp_first_true<SaT, true, kArity, 0>(T, sa, n_tokens, lo2, hi2, q, n, lane, eq2, bad);
       if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
       if (lane == 0) s.ub[n] = ub;
     }
@@ -312,7 +371,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   const int64_t cnt = hi - lo;
   const int Kp = (int)(cnt < (int64_t)a.K ? cnt : (int64_t)a.K);
   const int nwords = a.nwords;
-  const int niter = (Kp + kThreads - 1) / kThreads;
+  const int niter = (Kp + NT - 1) / NT;
 
   // ---- phase 2: gather rows, common-prefix lengths, node-start bitmaps --------------------
   // the suffix-array entry of the next iteration's row is fetched one iteration ahead, so
@@ -324,13 +383,13 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   if (lane == 0 && tid > 0 && tid <= Kp)
     pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid - 1));
   for (int it = 0; it < niter; ++it) {
-    const int jbase = it * kThreads + warp * 32;
+    const int jbase = it * NT + warp * 32;
     const int j = jbase + lane;
     int64_t p = p_next;
     const int64_t pp = pp_next;
-    if (j + kThreads < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + kThreads));
-    if (lane == 0 && j + kThreads <= Kp)
-      pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + kThreads - 1));
+    if (j + NT < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT));
+    if (lane == 0 && j + NT <= Kp)
+      pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT - 1));
     if (jbase >= Kp) continue;   // warp-uniform
     const bool valid = j < Kp;
     int row[kMaxM], prev[kMaxM];
@@ -399,11 +458,11 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
     return;
   }
 
-  // jump table: for every depth (one warp each) a suffix scan over the bitmap words, last chunk
+  // jump table: for every depth (a warp each) a suffix scan over the bitmap words, last chunk
   // of 32 words first: jump[w] = position of the first set bit in any word after w
-  if (warp < m) {
-    const uint32_t* row = bm + warp * nwords;
-    uint16_t* jrow = jump + warp * nwords;
+  for (int dd = warp; dd < m; dd += NW) {
+    const uint32_t* row = bm + dd * nwords;
+    uint16_t* jrow = jump + dd * nwords;
     const int last = (Kp + 31) >> 5;              // the sentinel word
     int carry = 0x7FFFFFFF;
     for (int c = last >> 5; c >= 0; --c) {
@@ -426,7 +485,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   // ---- phase 3a: histogram of (weight, depth) over all Trie nodes --------------------------
   // key = weight << 5 | (16 - depth): larger key = better node.
   for (int it = 0; it < niter; ++it) {
-    const int jbase = it * kThreads + warp * 32;
+    const int jbase = it * NT + warp * 32;
     if (jbase >= Kp) continue;
     const int j = jbase + lane;
     const bool valid = j < Kp;
@@ -471,7 +530,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
     __syncthreads();
     const int bin_hi = s.bin_hi;
     for (int it = 0; it < niter; ++it) {
-      const int jbase = it * kThreads + warp * 32;
+      const int jbase = it * NT + warp * 32;
       if (jbase >= Kp) continue;
       const int j = jbase + lane;
       if (j >= Kp) continue;
@@ -506,7 +565,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   // ---- phase 3c: collect the kept nodes -----------------------------------------------------
   uint32_t tie_base = 0;
   for (int it = 0; it < niter; ++it) {
-    const int j = it * kThreads + tid;
+    const int j = it * NT + tid;
     const bool valid = j < Kp;
     bool tie = false;
     if (valid) {
@@ -529,7 +588,7 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       if (lane == 0) s.warp_cnt[warp] = __popc(bal);
       __syncthreads();
       uint32_t before = tie_base, total = 0;
-      for (int w = 0; w < kWarps; ++w) {
+      for (int w = 0; w < NW; ++w) {
         uint32_t c = s.warp_cnt[w];
         if (w < warp) before += c;
         total += c;
@@ -548,16 +607,16 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
   if (s.nsel > (uint32_t)N && tid == 0) atomicOr(&s.err, REST_CTX_INTERNAL);
 
   // ---- phase 4: breadth-first order, parents, masks, tokens ---------------------------------
-  if (tid < nn) {
-    const uint32_t me = s.sel[tid];
+  for (int i = tid; i < nn; i += NT) {
+    const uint32_t me = s.sel[i];
     int rank = 0;
     for (int k = 0; k < nn; ++k) rank += (s.sel[k] < me);
     s.sorted[rank] = me;
-    s.sortedcnt[rank] = s.selcnt[tid];
+    s.sortedcnt[rank] = s.selcnt[i];
   }
   __syncthreads();
-  if (tid < nn) {
-    const uint32_t me = s.sorted[tid];
+  for (int i = tid; i < nn; i += NT) {
+    const uint32_t me = s.sorted[i];
     const int d = (int)(me >> 16), j = (int)(me & 0xFFFFu);
     int par = -1;
     if (d > 1) {
@@ -573,28 +632,28 @@ __global__ void __launch_bounds__(kThreads) rest_draft_kernel(DraftArgs a) {
       }
       if (par < 0) { atomicOr(&s.err, REST_CTX_INTERNAL); par = -1; }
     }
-    s.par[tid] = par;
+    s.par[i] = par;
     int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
-    int64_t o = (int64_t)b * N + tid;
+    int64_t o = (int64_t)b * N + i;
     a.tokens[o] = __ldg(T + p + n_win + d - 1);
     a.parents[o] = par;
     a.depth[o] = d;
     a.pos_ids[o] = clen + d - 1;
-    if (a.node_count) a.node_count[o] = (int32_t)s.sortedcnt[tid];
+    if (a.node_count) a.node_count[o] = (int32_t)s.sortedcnt[i];
   }
   __syncthreads();
-  if (tid < nn) {
+  for (int i = tid; i < nn; i += NT) {
     uint32_t bits[(kMaxN + 31) / 32];
 #pragma unroll
     for (int w = 0; w < (kMaxN + 31) / 32; ++w) bits[w] = 0;
-    int k = tid;
+    int k = i;
     for (int step = 0; step <= kMaxM && k >= 0; ++step) {
 #pragma unroll
       for (int w = 0; w < (kMaxN + 31) / 32; ++w)
         if (w == (k >> 5)) bits[w] |= 1u << (k & 31);
       k = s.par[k];
     }
-    int64_t o = ((int64_t)b * N + tid) * Wm;
+    int64_t o = ((int64_t)b * N + i) * Wm;
 #pragma unroll
     for (int w = 0; w < (kMaxN + 31) / 32; ++w)
       if (w < Wm) a.mask[o + w] = bits[w];
@@ -637,7 +696,11 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     return REST_INVALID_ARG;
   if (prm->n_min < 1 || prm->n_max < prm->n_min || prm->K < 1 || prm->m < 1 || prm->N < 1)
     return REST_INVALID_ARG;
-  if (prm->sample_mode != REST_SAMPLE_STRIDED && prm->sample_mode != REST_SAMPLE_FIRST_K)
+  const int sample_mode = prm->sample_mode & REST_SAMPLE_MASK;
+  const int search = prm->sample_mode & ~REST_SAMPLE_MASK;
+  if (sample_mode != REST_SAMPLE_STRIDED && sample_mode != REST_SAMPLE_FIRST_K)
+    return REST_INVALID_ARG;
+  if (search != REST_SEARCH_AUTO && search != REST_SEARCH_SINGLE && search != REST_SEARCH_BATCHED)
     return REST_INVALID_ARG;
   if (prm->n_max > REST_MAX_SUFFIX || prm->m > REST_MAX_M || prm->N > REST_MAX_N ||
       prm->K > REST_MAX_K || prm->n_max - prm->n_min + 1 > kWarps)
@@ -646,17 +709,29 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   DraftArgs a;
   a.T = ds->v.tokens; a.sa = ds->v.sa; a.n_tokens = ds->v.n_tokens; a.vocab = ds->v.vocab;
   a.n_max = prm->n_max; a.n_min = prm->n_min; a.K = prm->K; a.m = prm->m; a.N = prm->N;
-  a.sample_mode = prm->sample_mode;
+  a.sample_mode = sample_mode;
   a.ctx = d_ctx; a.ctx_stride = ctx_stride; a.ctx_len = d_ctx_len;
   a.tokens = d_tokens; a.parents = d_parents; a.depth = d_depth; a.pos_ids = d_pos_ids;
   a.mask = d_mask; a.n_nodes = d_n_nodes; a.match_n = d_match_n; a.match_range = d_match_range;
   a.node_count = d_node_count; a.status = d_status;
   size_t smem = draft_smem_bytes(prm->K, prm->m, &a.kcap, &a.nwords);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  auto kern = ds->v.sa_bytes == 4 ? rest_draft_kernel<int32_t> : rest_draft_kernel<int64_t>;
+  // the batched path pays off once the call has several times more contexts than the GPU holds
+  // at the same time (measured crossover: between 1024 and 4096 contexts on 148 SMs); below
+  // that a call lasts as long as its slowest contexts and the shortest dependent chain wins
+  bool batched = search == REST_SEARCH_BATCHED;
+  if (search == REST_SEARCH_AUTO) {
+    int dev = 0, sms = 0;
+    REST_CUDA_TRY(cudaGetDevice(&dev));
+    REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    batched = B >= 16 * sms;
+  }
+  const bool narrow = ds->v.sa_bytes == 4;
+  auto kern = batched ? (narrow ? rest_draft_kernel<int32_t, true> : rest_draft_kernel<int64_t, true>)
+                      : (narrow ? rest_draft_kernel<int32_t, false> : rest_draft_kernel<int64_t, false>);
   REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
-                                          ds->v.sa_bytes == 4 ? 0 : 1, smem));
-  kern<<<B, kThreads, smem, st>>>(a);
+                                          (batched ? 4 : 0) + (narrow ? 0 : 1), smem));
+  kern<<<B, batched ? kTpThreads : kThreads, smem, st>>>(a);
   rest::count_launch();
   REST_CUDA_TRY(cudaGetLastError());
   return REST_OK;

@@ -2,7 +2,7 @@
 
     python -m paper_2311_08252_b200.draft_bench [--workloads single_stream stress]
                                                 [--n-tokens 1000000 100000000] [--n-max 4 16]
-                                                [--batches 1 256 4096]
+                                                [--batches 1 256 4096] [--search auto|single|batched]
 
 The datastore is the workload's recipe at --n-tokens tokens; its suffix array is built on the
 device (rest_suffix_array_build).  Contexts follow the workload's context recipe.
@@ -42,6 +42,9 @@ def main():
                     help="longest suffix lengths to try (default: the workload's n_max)")
     ap.add_argument("--batches", nargs="*", type=int, default=[1, 64, 256, 1024, 4096])
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--search", choices=["auto", "single", "batched"], default="auto",
+                    help="suffix-array search of rest_draft (auto: batched when B exceeds what "
+                         "the GPU holds at once)")
     args = ap.parse_args()
     peak, peak_kind = bench.measured_peaks()
     dev = torch.device("cuda:0")
@@ -62,7 +65,9 @@ def main():
                    for s in range(nsets)]
             ctx_len = torch.full((B,), Lc, dtype=torch.int32, device=dev)
             out = rest.alloc_draft_output(B, w.N, dev)
-            kw = dict(n_max=n_max, n_min=min(w.n_min, n_max), K=w.K, m=w.m, N=w.N, out=out)
+            kw = dict(n_max=n_max, n_min=min(w.n_min, n_max), K=w.K, m=w.m, N=w.N, out=out,
+                      search={"auto": rest.REST_SEARCH_AUTO, "single": rest.REST_SEARCH_SINGLE,
+                              "batched": rest.REST_SEARCH_BATCHED}[args.search])
             kp, matched, match_n, nodes = 0, 0, 0, 0
             for s in range(nsets):
                 rest.rest_draft(ds, ctx[s], ctx_len, **kw)
@@ -85,7 +90,7 @@ def main():
             chain = bench.draft_chain_reads(w.n_tokens, kp_mean)
             print(json.dumps({
                 "workload": name, "datastore_tokens": w.n_tokens, "suffix_array_build_s": t_build,
-                "B": B, "K": w.K, "m": w.m, "N": w.N, "n_max": n_max,
+                "B": B, "K": w.K, "m": w.m, "N": w.N, "n_max": n_max, "search": args.search,
                 "mean_candidates": kp_mean, "mean_nodes": nodes / (nsets * B),
                 "contexts_with_a_match": matched / (nsets * B),
                 "mean_matched_length": match_n / max(matched, 1),

@@ -5,9 +5,13 @@ import pytest
 
 import datagen
 import oracle
+import paper_2311_08252_b200 as rest
 from gpu_util import assert_draft_equal, gpu_draft
 
 pytestmark = pytest.mark.gpu
+
+# the single-context and the batched suffix-array search must give the same trees
+SEARCHES = (rest.REST_SEARCH_SINGLE, rest.REST_SEARCH_BATCHED)
 
 
 def test_worked_example():
@@ -50,8 +54,9 @@ def test_small_alphabets_match_oracle(seed, vocab, n_tok, K, m, N, sa_bytes):
     for mode in (0, 1):
         kw = dict(K=K, m=m, N=N, sample_mode=mode)
         ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
-        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, **kw)
-        assert_draft_equal(got, ref, f"mode {mode}")
+        for search in SEARCHES:
+            got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, search=search, **kw)
+            assert_draft_equal(got, ref, f"mode {mode}, search {search:#x}")
 
 
 @pytest.mark.parametrize("name,n_tok,B", [
@@ -65,9 +70,30 @@ def test_workload_recipes_match_oracle(name, n_tok, B):
     ctx_len = np.full(B, ctx.shape[1], np.int32)
     kw = dict(K=w.K, m=w.m, N=w.N, n_max=w.n_max, n_min=w.n_min)
     ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
-    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, **kw)
-    assert_draft_equal(got, ref, name)
+    for search in SEARCHES:
+        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, search=search, **kw)
+        assert_draft_equal(got, ref, f"{name}, search {search:#x}")
     assert (ref["n_nodes"] > 0).sum() > B // 2
+
+
+def test_more_contexts_than_the_gpu_holds_at_once():
+    """B = 2500 contexts (more than 16 per SM): the call picks the batched path by itself; all
+    three settings agree with the oracle."""
+    w = datagen.WORKLOADS["batched"].scaled(n_tokens=3_000_000)
+    T = datagen.make_tokens(w)
+    sa = datagen.build_suffix_array(T, w.vocab, W=32, sa_bytes=w.sa_bytes)
+    B = 2500
+    ctx = datagen.make_contexts(w, T, B=B, Lc=48)
+    ctx_len = np.full(B, 48, np.int32)
+    ctx_len[::7] = np.arange(len(ctx_len[::7])) % 20      # short contexts: fewer lengths to search
+    kw = dict(K=w.K, m=w.m, N=w.N)
+    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+    for search in (rest.REST_SEARCH_AUTO,) + SEARCHES:
+        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, **kw)
+        assert_draft_equal(got, ref, f"search {search:#x}")
+    assert len(set(ref["match_n"].tolist())) > 8          # matched lengths all over 2 ... 16
+    with pytest.raises(rest.RestError):
+        gpu_draft(T, sa, w.vocab, ctx[:2], ctx_len[:2], search=0x400, **kw)
 
 
 def test_largest_trees_on_the_stress_recipe():
@@ -94,10 +120,11 @@ def test_other_suffix_limits_and_repeatability():
     for n_max, n_min in ((16, 1), (8, 3), (4, 4), (1, 1)):
         kw = dict(K=300, m=7, N=48, n_max=n_max, n_min=n_min)
         ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
-        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, **kw)
-        assert_draft_equal(got, ref, f"n_max={n_max} n_min={n_min}")
-        again, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, **kw)
-        assert_draft_equal(again, got, "second run")
+        for search in SEARCHES:
+            got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, **kw)
+            assert_draft_equal(got, ref, f"n_max={n_max} n_min={n_min} search {search:#x}")
+            again, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, **kw)
+            assert_draft_equal(again, got, "second run")
 
 
 def test_bad_context_tokens_and_corrupt_datastore():
@@ -165,5 +192,6 @@ def test_random_parameters_against_the_oracle():
                   N=int(rng.choice([1, 16, 64, 100, 128, 256])), n_max=n_max,
                   n_min=int(rng.integers(1, n_max + 1)), sample_mode=int(rng.integers(0, 2)))
         ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
-        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, **kw)
-        assert_draft_equal(got, ref, f"case {case}: vocab {vocab}, {n_tok} tokens, {kw}")
+        search = SEARCHES[case % 2]
+        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=search, **kw)
+        assert_draft_equal(got, ref, f"case {case}: vocab {vocab}, {n_tok} tokens, {kw}, search {search:#x}")
