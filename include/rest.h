@@ -56,8 +56,8 @@ enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1, REST_SAMPLE_MASK = 0xFF
  * (fewest dependent reads, the fastest single context).  BATCHED: 256 threads per context, six
  * or seven searches instead of fifteen (the lengths that match are n_min ... n* without a gap)
  * and eight probes per round once the probes leave L2: more dependent rounds, fewer random
- * DRAM reads, twice the contexts in flight.  AUTO picks BATCHED when the call has at least
- * 16 contexts per SM. */
+ * DRAM reads, more contexts in flight (most of all with the scratch that rest_draft_workspace_bytes
+ * asks for, see d_ws).  AUTO picks BATCHED when the call has at least 16 contexts per SM. */
 enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 0x100, REST_SEARCH_BATCHED = 0x200 };
 enum { REST_DS_VALIDATE = 1u };
 
@@ -132,7 +132,12 @@ void rest_datastore_destroy(rest_datastore* ds);
  *   d_match_range int64[B,2] lo, hi of the matched suffix-array range
  *   d_node_count int32[B,N]  weight of each kept node (may be NULL)
  *   d_status     int32[B]    REST_CTX_* code
- *   d_ws         scratch of rest_draft_workspace_bytes() bytes (may be NULL when that is 0)
+ *   d_ws         optional scratch of rest_draft_workspace_bytes() bytes (the query answers for
+ *                the current device; 0 when the call takes the single-context path).  With it
+ *                the batched path runs as three launches (search; build of the contexts with
+ *                few candidates on small blocks; build of the others on large blocks) and the
+ *                scratch holds the two context lists; with NULL or fewer bytes it runs as one
+ *                launch.  The outputs are the same.
  */
 size_t rest_draft_workspace_bytes(const rest_draft_params* params, int32_t B);
 rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params,

@@ -211,12 +211,22 @@ def alloc_draft_output(B: int, N: int, device) -> DraftOutput:
         torch.empty((B, N), **i32), torch.empty(B, **i32))
 
 
+def draft_workspace_bytes(B: int, n_max=16, n_min=2, K=5000, m=10, N=64,
+                          sample_mode=REST_SAMPLE_STRIDED, search=REST_SEARCH_AUTO) -> int:
+    """Scratch bytes rest_draft can use for a call of B contexts on the current device (0 when
+    the call takes the single-context path)."""
+    prm = _Params(n_max, n_min, K, m, N, sample_mode | search)
+    return int(lib().rest_draft_workspace_bytes(ctypes.byref(prm), B))
+
+
 def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=64,
                sample_mode=REST_SAMPLE_STRIDED, out: DraftOutput | None = None, stream=None,
-               search=REST_SEARCH_AUTO) -> DraftOutput:
+               search=REST_SEARCH_AUTO, workspace=None) -> DraftOutput:
     """Draft trees for contexts ctx int32[B, Lc] (row b holds ctx_len[b] tokens).  The mask
     tensor is int32 storage of the uint32 words.  `search` (REST_SEARCH_*) picks the
-    single-context or the batched suffix-array search; the results do not depend on it."""
+    single-context or the batched path; the results do not depend on it.  `workspace`: a uint8
+    CUDA tensor of rest_draft_workspace_bytes() bytes, None to allocate one when the library
+    asks for it, False to pass none (the batched path then runs as a single launch)."""
     L = lib()
     _dev_i32(ctx_len, "ctx_len")
     import torch
@@ -226,11 +236,18 @@ def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=6
     if out is None:
         out = alloc_draft_output(B, N, ctx.device)
     prm = _Params(n_max, n_min, K, m, N, sample_mode | search)
+    ws_ptr, ws_bytes = 0, 0
+    if workspace is None:
+        need = L.rest_draft_workspace_bytes(ctypes.byref(prm), B)
+        if need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=ctx.device)
+    if workspace is not None and workspace is not False:
+        ws_ptr, ws_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     rc = L.rest_draft(ds._h, ctypes.byref(prm), ctx.data_ptr(), ctx.stride(0), ctx_len.data_ptr(), B,
                       out.tokens.data_ptr(), out.parents.data_ptr(), out.depth.data_ptr(),
                       out.pos_ids.data_ptr(), out.mask.data_ptr(), out.n_nodes.data_ptr(),
                       out.match_n.data_ptr(), out.match_range.data_ptr(), _ptr(out.node_count),
-                      out.status.data_ptr(), 0, 0, _stream(stream))
+                      out.status.data_ptr(), ws_ptr, ws_bytes, _stream(stream))
     _check(rc, "rest_draft")
     return out
 

@@ -40,6 +40,11 @@ constexpr int kTpThreads = 256;
 constexpr int kTpArity = 8;
 constexpr bool kTpStaged = true;
 constexpr int kWideRounds = 3;
+// three-launch form: block sizes of the search and of the build of contexts with at most
+// kLightRows candidates (the others are built by kThreads-wide blocks)
+constexpr int kSearchThreads = 128;
+constexpr int kLightThreads = 128;
+constexpr int kLightRows = 256;
 
 struct DraftArgs {
   const int32_t* T;
@@ -56,7 +61,14 @@ struct DraftArgs {
   int64_t* match_range;
   int32_t *node_count, *status;
   int nwords;   // bitmap words per depth
-  int kcap;     // K rounded up to a multiple of 32
+  int kcap;     // rows the block's shared memory holds, a multiple of 32
+  // three-launch form of the batched path: the search launch sorts the contexts that matched
+  // into two lists by candidate count, the two build launches take one list each
+  int32_t* list;          // [2][B] context indices
+  int32_t* list_count;    // [2]
+  int B;
+  int which;              // list of this build launch
+  int light_rows;         // candidate counts up to this go to list 0
 };
 
 // Three-way comparison of the first n tokens of the suffix stored in slot `slot` with q.
@@ -225,10 +237,13 @@ struct Smem {
 // TP = false: the single-context path, tuned for the fewest dependent reads.  TP = true: the
 // batched path, for calls with more contexts than the GPU holds at once; the same results by
 // fewer random DRAM reads per context (see phase 1).
-template <typename SaT, bool TP>
-__global__ void __launch_bounds__(TP ? kTpThreads : kThreads, TP ? 1024 / kTpThreads : 2)
+// PART: kWhole = search and build in one launch; kSearch = phase 1 only (writes match_n and
+// match_range, the defaults of every output slot, and the context's index into one of two
+// lists); kBuild = phases 2-4 for the contexts of one list.
+enum { kWhole = 0, kSearch = 1, kBuild = 2 };
+template <typename SaT, bool TP, int NT, int PART>
+__global__ void __launch_bounds__(NT, 1024 / NT)
 rest_draft_kernel(DraftArgs a) {
-  constexpr int NT = TP ? kTpThreads : kThreads;   // threads of this block
   constexpr int NW = NT / 32;
   static_assert(NT % 32 == 0 && NT >= 64, "whole warps; at least kMaxM + 2 threads");
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -237,7 +252,10 @@ rest_draft_kernel(DraftArgs a) {
   uint32_t* bm = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Smem) + 2 * a.kcap); // [m][nwords]
   uint16_t* jump = reinterpret_cast<uint16_t*>(bm + a.m * a.nwords);                // [m][nwords]
 
-  const int b = blockIdx.x;
+  if constexpr (PART == kBuild) {
+    if ((int)blockIdx.x >= a.list_count[a.which]) return;
+  }
+  const int b = PART == kBuild ? a.list[(int64_t)a.which * a.B + blockIdx.x] : (int)blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int N = a.N, m = a.m, Wm = (N + 31) >> 5;
   // a kernel launched behind this one with programmatic stream serialisation may begin its
@@ -249,7 +267,9 @@ rest_draft_kernel(DraftArgs a) {
   const int clen = a.ctx_len[b];
   const int32_t* ctx = a.ctx + (int64_t)b * a.ctx_stride;
 
-  // Unused-slot defaults; thread i owns slots i, i + NT, ... for the whole kernel.
+  // Unused-slot defaults; thread i owns slots i, i + NT, ... for the whole kernel (a build
+  // launch finds them written by the search launch).
+  if constexpr (PART != kBuild)
   for (int i = tid; i < N; i += NT) {
     int64_t o = (int64_t)b * N + i;
     a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
@@ -261,9 +281,17 @@ rest_draft_kernel(DraftArgs a) {
   if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; }
   if (tid <= kMaxM) s.e1[tid] = 0;
   if (tid <= kMaxM + 1) s.e1diff[tid] = 0;
-  for (int i = tid; i < kHistHi; i += NT) s.hist_hi[i] = 0;
-  for (int i = tid; i < kHistLo; i += NT) s.hist_lo[i] = 0;
+  if constexpr (PART != kSearch) {
+    for (int i = tid; i < kHistHi; i += NT) s.hist_hi[i] = 0;
+    for (int i = tid; i < kHistLo; i += NT) s.hist_lo[i] = 0;
+  }
   __syncthreads();
+  int n_win = 0;
+  if constexpr (PART == kBuild) {
+    n_win = a.match_n[b];
+    if (tid == 0) { s.lb[n_win] = a.match_range[2 * b]; s.ub[n_win] = a.match_range[2 * b + 1]; }
+    __syncthreads();
+  } else {
   if (tid < nq) {
     int t = ctx[clen - nq + tid];
     s.q[tid] = t;
@@ -317,7 +345,6 @@ rest_draft_kernel(DraftArgs a) {
     }
   }
   __syncthreads();
-  int n_win = 0;
   for (int n = nq; n >= a.n_min; --n)
     if (s.ub[n] != s.lb[n]) { n_win = n; break; }
   // 1b: only the winning length needs its upper bound, and only if the last round of its lower
@@ -367,8 +394,20 @@ rest_draft_kernel(DraftArgs a) {
     }
     return;
   }
+  }  // PART != kBuild
   const int64_t lo = s.lb[n_win], hi = s.ub[n_win];
   const int64_t cnt = hi - lo;
+  if constexpr (PART == kSearch) {
+    // hand the context to the build launch that fits its candidate count
+    if (tid == 0) {
+      a.status[b] = 0; a.n_nodes[b] = 0; a.match_n[b] = n_win;
+      a.match_range[2 * b] = lo; a.match_range[2 * b + 1] = hi;
+      const int heavy = (cnt < (int64_t)a.K ? cnt : (int64_t)a.K) > (int64_t)a.light_rows;
+      const int at = atomicAdd(a.list_count + heavy, 1);
+      a.list[(int64_t)heavy * a.B + at] = b;
+    }
+    return;
+  }
   const int Kp = (int)(cnt < (int64_t)a.K ? cnt : (int64_t)a.K);
   const int nwords = a.nwords;
   const int niter = (Kp + NT - 1) / NT;
@@ -679,7 +718,29 @@ size_t draft_smem_bytes(int K, int m, int* kcap_out, int* nwords_out) {
 
 }  // namespace
 
-extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params*, int32_t) { return 0; }
+// Whether a call of B contexts takes the batched path (search = the REST_SEARCH_* bits).
+static rest_status wants_batched(int search, int B, bool* batched) {
+  *batched = search == REST_SEARCH_BATCHED;
+  if (search == REST_SEARCH_AUTO) {
+    // the batched path pays off once the call has several times more contexts than the GPU
+    // holds at the same time (measured crossover: between 1024 and 4096 contexts on 148 SMs);
+    // below that a call lasts as long as its slowest contexts and the shortest dependent chain wins
+    int dev = 0, sms = 0;
+    REST_CUDA_TRY(cudaGetDevice(&dev));
+    REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    *batched = B >= 16 * sms;
+  }
+  return REST_OK;
+}
+
+static size_t split_workspace_bytes(int B) { return (2 * (size_t)B + 16) * sizeof(int32_t); }
+
+extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params* prm, int32_t B) {
+  if (!prm || B <= 0) return 0;
+  bool batched = false;
+  if (wants_batched(prm->sample_mode & ~REST_SAMPLE_MASK, B, &batched) != REST_OK || !batched) return 0;
+  return split_workspace_bytes(B);
+}
 
 extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* prm,
                                   const int32_t* d_ctx, int64_t ctx_stride,
@@ -687,7 +748,7 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
                                   int32_t* d_parents, int32_t* d_depth, int32_t* d_pos_ids,
                                   uint32_t* d_mask, int32_t* d_n_nodes, int32_t* d_match_n,
                                   int64_t* d_match_range, int32_t* d_node_count,
-                                  int32_t* d_status, void* /*d_ws*/, size_t /*ws_bytes*/,
+                                  int32_t* d_status, void* d_ws, size_t ws_bytes,
                                   void* stream) {
   if (!ds || !prm || B < 0) return REST_INVALID_ARG;
   if (B == 0) return REST_OK;
@@ -716,23 +777,46 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   a.node_count = d_node_count; a.status = d_status;
   size_t smem = draft_smem_bytes(prm->K, prm->m, &a.kcap, &a.nwords);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the batched path pays off once the call has several times more contexts than the GPU holds
-  // at the same time (measured crossover: between 1024 and 4096 contexts on 148 SMs); below
-  // that a call lasts as long as its slowest contexts and the shortest dependent chain wins
-  bool batched = search == REST_SEARCH_BATCHED;
-  if (search == REST_SEARCH_AUTO) {
-    int dev = 0, sms = 0;
-    REST_CUDA_TRY(cudaGetDevice(&dev));
-    REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    batched = B >= 16 * sms;
-  }
+  bool batched = false;
+  if (rest_status rc = wants_batched(search, B, &batched); rc != REST_OK) return rc;
   const bool narrow = ds->v.sa_bytes == 4;
-  auto kern = batched ? (narrow ? rest_draft_kernel<int32_t, true> : rest_draft_kernel<int64_t, true>)
-                      : (narrow ? rest_draft_kernel<int32_t, false> : rest_draft_kernel<int64_t, false>);
-  REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
-                                          (batched ? 4 : 0) + (narrow ? 0 : 1), smem));
-  kern<<<B, batched ? kTpThreads : kThreads, smem, st>>>(a);
-  rest::count_launch();
-  REST_CUDA_TRY(cudaGetLastError());
-  return REST_OK;
+  a.list = nullptr; a.list_count = nullptr; a.B = B; a.which = 0; a.light_rows = 0;
+  auto launch = [&](auto kern, int slot, int threads, int blocks, size_t bytes) -> rest_status {
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern), slot + (narrow ? 0 : 1), bytes));
+    kern<<<blocks, threads, bytes, st>>>(a);
+    rest::count_launch();
+    REST_CUDA_TRY(cudaGetLastError());
+    return REST_OK;
+  };
+  if (!batched) {
+    return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWhole>, 0, kThreads, B, smem)
+                  : launch(rest_draft_kernel<int64_t, false, kThreads, kWhole>, 0, kThreads, B, smem);
+  }
+  if (!d_ws || ws_bytes < split_workspace_bytes(B)) {
+    // no scratch for the context lists: search and build in one launch
+    return narrow ? launch(rest_draft_kernel<int32_t, true, kTpThreads, kWhole>, 2, kTpThreads, B, smem)
+                  : launch(rest_draft_kernel<int64_t, true, kTpThreads, kWhole>, 2, kTpThreads, B, smem);
+  }
+  // Three launches: the search with a small block per context; then the contexts that matched,
+  // those with few candidates on small blocks (many per SM) and the others on large ones.  A
+  // build launch has one block per context of the call; the blocks beyond its list leave at once.
+  a.list_count = static_cast<int32_t*>(d_ws);
+  a.list = a.list_count + 16;
+  a.light_rows = prm->K < kLightRows ? prm->K : kLightRows;
+  REST_CUDA_TRY(cudaMemsetAsync(a.list_count, 0, 2 * sizeof(int32_t), st));
+  rest_status rc = narrow ? launch(rest_draft_kernel<int32_t, true, kSearchThreads, kSearch>, 4, kSearchThreads, B, sizeof(Smem))
+                          : launch(rest_draft_kernel<int64_t, true, kSearchThreads, kSearch>, 4, kSearchThreads, B, sizeof(Smem));
+  if (rc != REST_OK) return rc;
+  const int kcap_all = a.kcap, nwords_all = a.nwords;
+  const size_t smem_light = draft_smem_bytes(a.light_rows, prm->m, &a.kcap, &a.nwords);
+  a.which = 0;
+  rc = narrow ? launch(rest_draft_kernel<int32_t, true, kLightThreads, kBuild>, 6, kLightThreads, B, smem_light)
+              : launch(rest_draft_kernel<int64_t, true, kLightThreads, kBuild>, 6, kLightThreads, B, smem_light);
+  if (rc != REST_OK) return rc;
+  if (prm->K > a.light_rows) {
+    a.kcap = kcap_all; a.nwords = nwords_all; a.which = 1;
+    rc = narrow ? launch(rest_draft_kernel<int32_t, true, kThreads, kBuild>, 8, kThreads, B, smem)
+                : launch(rest_draft_kernel<int64_t, true, kThreads, kBuild>, 8, kThreads, B, smem);
+  }
+  return rc;
 }

@@ -45,6 +45,8 @@ def main():
     ap.add_argument("--search", choices=["auto", "single", "batched"], default="auto",
                     help="suffix-array search of rest_draft (auto: batched when B exceeds what "
                          "the GPU holds at once)")
+    ap.add_argument("--no-workspace", action="store_true",
+                    help="pass no scratch: the batched path then runs as a single launch")
     args = ap.parse_args()
     peak, peak_kind = bench.measured_peaks()
     dev = torch.device("cuda:0")
@@ -65,9 +67,12 @@ def main():
                    for s in range(nsets)]
             ctx_len = torch.full((B,), Lc, dtype=torch.int32, device=dev)
             out = rest.alloc_draft_output(B, w.N, dev)
-            kw = dict(n_max=n_max, n_min=min(w.n_min, n_max), K=w.K, m=w.m, N=w.N, out=out,
+            kw = dict(n_max=n_max, n_min=min(w.n_min, n_max), K=w.K, m=w.m, N=w.N,
                       search={"auto": rest.REST_SEARCH_AUTO, "single": rest.REST_SEARCH_SINGLE,
                               "batched": rest.REST_SEARCH_BATCHED}[args.search])
+            ws_bytes = 0 if args.no_workspace else rest.draft_workspace_bytes(B, **kw)
+            kw.update(out=out, workspace=torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+                      if ws_bytes else False)
             kp, matched, match_n, nodes = 0, 0, 0, 0
             for s in range(nsets):
                 rest.rest_draft(ds, ctx[s], ctx_len, **kw)

@@ -57,6 +57,8 @@ def test_small_alphabets_match_oracle(seed, vocab, n_tok, K, m, N, sa_bytes):
         for search in SEARCHES:
             got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, search=search, **kw)
             assert_draft_equal(got, ref, f"mode {mode}, search {search:#x}")
+        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=rest.REST_SEARCH_BATCHED, workspace=False, **kw)
+        assert_draft_equal(got, ref, f"mode {mode}, batched in one launch")
 
 
 @pytest.mark.parametrize("name,n_tok,B", [
@@ -91,6 +93,9 @@ def test_more_contexts_than_the_gpu_holds_at_once():
     for search in (rest.REST_SEARCH_AUTO,) + SEARCHES:
         got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, **kw)
         assert_draft_equal(got, ref, f"search {search:#x}")
+    # without scratch for the context lists the batched path runs as one launch
+    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=rest.REST_SEARCH_BATCHED, workspace=False, **kw)
+    assert_draft_equal(got, ref, "batched, one launch")
     assert len(set(ref["match_n"].tolist())) > 8          # matched lengths all over 2 ... 16
     with pytest.raises(rest.RestError):
         gpu_draft(T, sa, w.vocab, ctx[:2], ctx_len[:2], search=0x400, **kw)
