@@ -57,7 +57,8 @@ enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1, REST_SAMPLE_MASK = 0xFF
  * or seven searches instead of fifteen (the lengths that match are n_min ... n* without a gap)
  * and eight probes per round once the probes leave L2: more dependent rounds, fewer random
  * DRAM reads, more contexts in flight (most of all with the scratch that rest_draft_workspace_bytes
- * asks for, see d_ws).  AUTO picks BATCHED when the call has at least 16 contexts per SM. */
+ * asks for, see d_ws).  AUTO picks BATCHED when the call has at least 5 contexts per SM and
+ * that scratch, or at least 16 contexts per SM without it. */
 enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 0x100, REST_SEARCH_BATCHED = 0x200 };
 enum { REST_DS_VALIDATE = 1u };
 

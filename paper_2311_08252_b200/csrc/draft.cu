@@ -718,17 +718,18 @@ size_t draft_smem_bytes(int K, int m, int* kcap_out, int* nwords_out) {
 
 }  // namespace
 
-// Whether a call of B contexts takes the batched path (search = the REST_SEARCH_* bits).
-static rest_status wants_batched(int search, int B, bool* batched) {
+// Whether a call of B contexts takes the batched path (search = the REST_SEARCH_* bits;
+// with_scratch: the caller gives the scratch of the three-launch form).
+static rest_status wants_batched(int search, int B, bool with_scratch, bool* batched) {
   *batched = search == REST_SEARCH_BATCHED;
   if (search == REST_SEARCH_AUTO) {
-    // the batched path pays off once the call has several times more contexts than the GPU
-    // holds at the same time (measured crossover: between 1024 and 4096 contexts on 148 SMs);
-    // below that a call lasts as long as its slowest contexts and the shortest dependent chain wins
+    // Below a few contexts per SM a call lasts as long as its slowest contexts and the shortest
+    // dependent chain wins.  Measured crossover on 148 SMs: between 512 and 1024 contexts for the
+    // three-launch form, between 1024 and 4096 for the one-launch form.
     int dev = 0, sms = 0;
     REST_CUDA_TRY(cudaGetDevice(&dev));
     REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    *batched = B >= 16 * sms;
+    *batched = B >= (with_scratch ? 5 : 16) * sms;
   }
   return REST_OK;
 }
@@ -738,7 +739,7 @@ static size_t split_workspace_bytes(int B) { return (2 * (size_t)B + 16) * sizeo
 extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params* prm, int32_t B) {
   if (!prm || B <= 0) return 0;
   bool batched = false;
-  if (wants_batched(prm->sample_mode & ~REST_SAMPLE_MASK, B, &batched) != REST_OK || !batched) return 0;
+  if (wants_batched(prm->sample_mode & ~REST_SAMPLE_MASK, B, true, &batched) != REST_OK || !batched) return 0;
   return split_workspace_bytes(B);
 }
 
@@ -777,8 +778,9 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   a.node_count = d_node_count; a.status = d_status;
   size_t smem = draft_smem_bytes(prm->K, prm->m, &a.kcap, &a.nwords);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool with_scratch = d_ws && ws_bytes >= split_workspace_bytes(B);
   bool batched = false;
-  if (rest_status rc = wants_batched(search, B, &batched); rc != REST_OK) return rc;
+  if (rest_status rc = wants_batched(search, B, with_scratch, &batched); rc != REST_OK) return rc;
   const bool narrow = ds->v.sa_bytes == 4;
   a.list = nullptr; a.list_count = nullptr; a.B = B; a.which = 0; a.light_rows = 0;
   auto launch = [&](auto kern, int slot, int threads, int blocks, size_t bytes) -> rest_status {
@@ -792,7 +794,7 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWhole>, 0, kThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, false, kThreads, kWhole>, 0, kThreads, B, smem);
   }
-  if (!d_ws || ws_bytes < split_workspace_bytes(B)) {
+  if (!with_scratch) {
     // no scratch for the context lists: search and build in one launch
     return narrow ? launch(rest_draft_kernel<int32_t, true, kTpThreads, kWhole>, 2, kTpThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, true, kTpThreads, kWhole>, 2, kTpThreads, B, smem);

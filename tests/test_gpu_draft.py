@@ -79,8 +79,8 @@ def test_workload_recipes_match_oracle(name, n_tok, B):
 
 
 def test_more_contexts_than_the_gpu_holds_at_once():
-    """B = 2500 contexts (more than 16 per SM): the call picks the batched path by itself; all
-    three settings agree with the oracle."""
+    """B = 2500 contexts (more than 16 per SM): the call picks the batched path by itself, with
+    and without scratch; every setting agrees with the oracle."""
     w = datagen.WORKLOADS["batched"].scaled(n_tokens=3_000_000)
     T = datagen.make_tokens(w)
     sa = datagen.build_suffix_array(T, w.vocab, W=32, sa_bytes=w.sa_bytes)
@@ -94,8 +94,10 @@ def test_more_contexts_than_the_gpu_holds_at_once():
         got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, **kw)
         assert_draft_equal(got, ref, f"search {search:#x}")
     # without scratch for the context lists the batched path runs as one launch
-    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=rest.REST_SEARCH_BATCHED, workspace=False, **kw)
-    assert_draft_equal(got, ref, "batched, one launch")
+    for search in (rest.REST_SEARCH_AUTO, rest.REST_SEARCH_BATCHED):
+        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, workspace=False, **kw)
+        assert_draft_equal(got, ref, f"one launch, search {search:#x}")
+    assert rest.draft_workspace_bytes(B, **kw) >= 8 * B and rest.draft_workspace_bytes(8, **kw) == 0
     assert len(set(ref["match_n"].tolist())) > 8          # matched lengths all over 2 ... 16
     with pytest.raises(rest.RestError):
         gpu_draft(T, sa, w.vocab, ctx[:2], ctx_len[:2], search=0x400, **kw)
