@@ -41,10 +41,16 @@ constexpr int kTpArity = 8;
 constexpr bool kTpStaged = true;
 constexpr int kWideRounds = 3;
 // three-launch form: block sizes of the search and of the build of contexts with at most
-// kLightRows candidates (the others are built by kThreads-wide blocks)
+// kLightRows candidates, and of the build of the others
 constexpr int kSearchThreads = 128;
 constexpr int kLightThreads = 128;
 constexpr int kLightRows = 256;
+// Blocks of contexts with long candidate lists: kThreads (two per SM by registers) unless the
+// K cap is so large that shared memory allows only two blocks per SM anyway; then kBigThreads,
+// which doubles the threads an SM gives to such a context (K = 20000, m = 16: 880 -> 415 us at
+// 1024 contexts, 1670 -> 1181 us at 4096; at K = 5000 the same change loses 4-13 % in large calls).
+constexpr int kBigThreads = 1024;
+constexpr size_t kBigSmemBytes = 56 * 1024;
 
 struct DraftArgs {
   const int32_t* T;
@@ -224,7 +230,7 @@ struct Smem {
   int bin_lo;
   uint32_t above_lo;
   uint32_t nsel;
-  uint32_t warp_cnt[kWarps];
+  uint32_t warp_cnt[32];
   uint32_t sel[kMaxN];         // depth << 16 | row
   uint32_t selcnt[kMaxN];
   uint32_t sorted[kMaxN];
@@ -790,7 +796,11 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     REST_CUDA_TRY(cudaGetLastError());
     return REST_OK;
   };
+  const bool big = smem > kBigSmemBytes;
   if (!batched) {
+    if (big)
+      return narrow ? launch(rest_draft_kernel<int32_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem)
+                    : launch(rest_draft_kernel<int64_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem);
     return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWhole>, 0, kThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, false, kThreads, kWhole>, 0, kThreads, B, smem);
   }
@@ -817,8 +827,12 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   if (rc != REST_OK) return rc;
   if (prm->K > a.light_rows) {
     a.kcap = kcap_all; a.nwords = nwords_all; a.which = 1;
-    rc = narrow ? launch(rest_draft_kernel<int32_t, true, kThreads, kBuild>, 8, kThreads, B, smem)
-                : launch(rest_draft_kernel<int64_t, true, kThreads, kBuild>, 8, kThreads, B, smem);
+    if (big)
+      rc = narrow ? launch(rest_draft_kernel<int32_t, true, kBigThreads, kBuild>, 12, kBigThreads, B, smem)
+                  : launch(rest_draft_kernel<int64_t, true, kBigThreads, kBuild>, 12, kBigThreads, B, smem);
+    else
+      rc = narrow ? launch(rest_draft_kernel<int32_t, true, kThreads, kBuild>, 8, kThreads, B, smem)
+                  : launch(rest_draft_kernel<int64_t, true, kThreads, kBuild>, 8, kThreads, B, smem);
   }
   return rc;
 }
