@@ -23,7 +23,7 @@ rest_status note_cuda_error(cudaError_t e, const char* where) {
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t bytes) {
-  constexpr int kMaxDev = 64, kSlots = 16;
+  constexpr int kMaxDev = 64, kSlots = kSmemSlots;
   static std::atomic<size_t> set_bytes[kMaxDev][kSlots];
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);

@@ -790,7 +790,8 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   const bool narrow = ds->v.sa_bytes == 4;
   a.list = nullptr; a.list_count = nullptr; a.B = B; a.which = 0; a.light_rows = 0;
   auto launch = [&](auto kern, int slot, int threads, int blocks, size_t bytes) -> rest_status {
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern), slot + (narrow ? 0 : 1), bytes));
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
+                                            rest::kSmemSlotDraft + slot + (narrow ? 0 : 1), bytes));
     kern<<<blocks, threads, bytes, st>>>(a);
     rest::count_launch();
     REST_CUDA_TRY(cudaGetLastError());
@@ -798,7 +799,13 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   };
   const bool big = smem > kBigSmemBytes;
   if (!batched) {
-    if (big)
+    // a call with at most one context per SM lasts as long as its slowest context: give each
+    // context the whole SM (not the single context: its typical candidate list is short and
+    // the larger block only adds barrier time)
+    int dev = 0, sms = 0;
+    REST_CUDA_TRY(cudaGetDevice(&dev));
+    REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (big || (B > 1 && B <= sms))
       return narrow ? launch(rest_draft_kernel<int32_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem)
                     : launch(rest_draft_kernel<int64_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem);
     return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWhole>, 0, kThreads, B, smem)

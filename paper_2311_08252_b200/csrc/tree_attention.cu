@@ -1279,7 +1279,7 @@ int cluster_capacity(bool wide, int c) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (rest::ensure_dynamic_smem(fn, wide ? 3 : 2, smem) != cudaSuccess ||
+    if (rest::ensure_dynamic_smem(fn, wide ? rest::kSmemSlotAttnWide : rest::kSmemSlotAttn, smem) != cudaSuccess ||
         cudaOccupancyMaxActiveClusters(&n, fn, &cfg) != cudaSuccess || n <= 0) {
       (void)cudaGetLastError();
       return nominal;
@@ -1392,9 +1392,9 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   a.NBLK = N > 64 ? (N + 127) / 128 : 1;
   const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
   if (wide)
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_wide_kernel), 3, smem));
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_wide_kernel), rest::kSmemSlotAttnWide, smem));
   else
-    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), 2, smem));
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(tree_attention_ws_kernel), rest::kSmemSlotAttn, smem));
   if ((int64_t)B * H * a.NBLK * a.S > 0x7FFFFFFFll) return REST_UNSUPPORTED;
   // Units that need no key split but do not fill a whole number of waves: the units of the last,
   // partial wave go into a second launch with their key range cut over one cluster each, so that
