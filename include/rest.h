@@ -6,7 +6,8 @@
  * Draft side:   rest_draft                                 (Sec. 3.2, Algorithms 1 and 2)
  * Verify side:  rest_tree_attention, rest_accept           (Sec. 3.2, draft verification / acceptance)
  * Between steps: rest_kv_commit                            (the accepted path joins the prefix)
- * Aids:         rest_tree_attention_plan, rest_probe_dependent_reads, rest_device_error_flags
+ * Health:       rest_device_error_flags
+ * (measurement and planning aids live in rest_aids.h)
  *
  * Conventions
  *   - Every pointer named d_* is a DEVICE pointer owned by the caller.  The library borrows
@@ -50,16 +51,16 @@ enum {
   REST_CTX_INTERNAL = 3
 };
 
-enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1, REST_SAMPLE_MASK = 0xFF };
-/* How rest_draft searches the suffix array, OR-ed into sample_mode; the results are the same
- * either way.  SINGLE: all suffix lengths at once, 32 probes per round, 512 threads per context
- * (fewest dependent reads, the fastest single context).  BATCHED: 256 threads per context, six
- * or seven searches instead of fifteen (the lengths that match are n_min ... n* without a gap)
- * and eight probes per round once the probes leave L2: more dependent rounds, fewer random
- * DRAM reads, more contexts in flight (most of all with the scratch that rest_draft_workspace_bytes
- * asks for, see d_ws).  AUTO picks BATCHED when the call has at least 5 contexts per SM and
- * that scratch, or at least 16 contexts per SM without it. */
-enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 0x100, REST_SEARCH_BATCHED = 0x200 };
+enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1 };
+/* How rest_draft searches the suffix array (rest_draft_params.search_path); the results are the
+ * same either way.  SINGLE: all suffix lengths at once, 32 probes per round, 512 threads per
+ * context (fewest dependent reads, the fastest single context).  BATCHED: 256 threads per
+ * context, six or seven searches instead of fifteen (the lengths that match are n_min ... n*
+ * without a gap) and eight probes per round once the probes leave L2: more dependent rounds,
+ * fewer random DRAM reads, more contexts in flight (most of all with the scratch that
+ * rest_draft_workspace_bytes asks for, see d_ws).  AUTO picks BATCHED when the call has at
+ * least 5 contexts per SM and that scratch, or at least 16 contexts per SM without it. */
+enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 1, REST_SEARCH_BATCHED = 2 };
 enum { REST_DS_VALIDATE = 1u };
 
 /* Limits of this implementation. */
@@ -79,9 +80,10 @@ typedef struct rest_datastore rest_datastore;   /* opaque host object holding de
  *   m             continuation length (1..16)
  *   N             maximum number of draft tokens, the paper's c (1..256)
  *   sample_mode   which K of cnt > K matches are used: REST_SAMPLE_STRIDED takes suffix-array
- *                 slot lo + floor(j*cnt/K), REST_SAMPLE_FIRST_K takes lo + j, j = 0..K-1      */
+ *                 slot lo + floor(j*cnt/K), REST_SAMPLE_FIRST_K takes lo + j, j = 0..K-1
+ *   search_path   REST_SEARCH_AUTO / SINGLE / BATCHED: a performance switch, never a result */
 typedef struct {
-  int32_t n_max, n_min, K, m, N, sample_mode;
+  int32_t n_max, n_min, K, m, N, sample_mode, search_path;
 } rest_draft_params;
 
 /*
@@ -170,7 +172,7 @@ rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params
  *             output is built from, so it carries bf16 precision (a few 1e-3 absolute)
  *   d_ws      scratch of rest_tree_attention_workspace_bytes() bytes
  *   scale     softmax scale, finite and > 0 (else REST_INVALID_ARG)
- *   Limits: D = 128; N in {16, 32, 48, ..., 256}; H % H_kv == 0.
+ *   Limits: D = 128; 1 <= N <= 256 (any tree rest_draft can write); H % H_kv == 0.
  */
 size_t rest_tree_attention_workspace_bytes(int32_t B, int32_t H, int32_t N, int32_t D,
                                            int32_t max_kv);
@@ -179,16 +181,6 @@ rest_status rest_tree_attention(const void* d_q, const void* d_k, const void* d_
                                 const uint32_t* d_mask, int32_t B, int32_t H, int32_t H_kv,
                                 int32_t N, int32_t D, int32_t max_kv, float scale, void* d_out,
                                 float* d_lse, void* d_ws, size_t ws_bytes, void* stream);
-
-/*
- * rest_tree_attention_plan - how rest_tree_attention would cut the key range for this shape on
- * the current device (a planning aid; the paper has no counterpart).  out[0] = key ranges per
- * (context, head), out[1] = blocks per cluster (ranges merged on chip), out[2] = clusters per
- * (context, head) (merged through the workspace when > 1), out[3] = clusters of that size the
- * device can run at once.  Host pointers.
- */
-rest_status rest_tree_attention_plan(int32_t B, int32_t H, int32_t N, int32_t D, int32_t max_kv,
-                                     int32_t* out);
 
 /*
  * rest_tree_attention_static_scratch - rest_tree_attention for callers that cannot allocate.
@@ -286,19 +278,6 @@ rest_status rest_suffix_array_build(const int32_t* d_tokens, uint64_t n_tokens, 
                                     void* d_sa, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
- * rest_probe_dependent_reads - measurement aid (the paper has no counterpart).
- *
- * One device thread follows `steps` dependent loads idx = d_next[idx] from `start` and writes
- * d_out[0] = elapsed nanoseconds (device global timer), d_out[1] = the final index.  With a
- * random cyclic table much larger than L2 this is the latency of one dependent DRAM read; the
- * searches of Algorithm 1 are chains of such reads, so it bounds a single draft from below.
- *   d_next  uint32[n] device table (entries >= n are treated as 0), n <= 2^32 - 1
- *   d_out   uint64[2] device
- */
-rest_status rest_probe_dependent_reads(const uint32_t* d_next, uint64_t n, uint32_t start,
-                                       uint32_t steps, uint64_t* d_out, void* stream);
-
-/*
  * Device-side trouble that no per-call status can carry.  Every wait inside the kernels is
  * bounded; a kernel that gives up sets a bit here instead of spinning, and its output is then
  * undefined.  Reads and clears the flags of the current device (synchronises the device).
@@ -310,8 +289,6 @@ rest_status rest_device_error_flags(uint32_t* h_flags);
 const char* rest_status_string(rest_status s);
 /* Text of the last CUDA runtime error seen by this library on the calling thread. */
 const char* rest_last_cuda_error(void);
-/* Number of kernels the library has launched in this process (for launch accounting). */
-uint64_t rest_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -23,8 +23,8 @@ REST_OK = 0
 REST_SAMPLE_STRIDED = 0
 REST_SAMPLE_FIRST_K = 1
 REST_SEARCH_AUTO = 0
-REST_SEARCH_SINGLE = 0x100
-REST_SEARCH_BATCHED = 0x200
+REST_SEARCH_SINGLE = 1
+REST_SEARCH_BATCHED = 2
 REST_DS_VALIDATE = 1
 
 EXPORTS = (
@@ -43,7 +43,8 @@ class RestError(RuntimeError):
 
 
 class _Params(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("n_max", "n_min", "K", "m", "N", "sample_mode")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("n_max", "n_min", "K", "m", "N", "sample_mode",
+                                              "search_path")]
 
 
 _lib = None
@@ -215,7 +216,7 @@ def draft_workspace_bytes(B: int, n_max=16, n_min=2, K=5000, m=10, N=64,
                           sample_mode=REST_SAMPLE_STRIDED, search=REST_SEARCH_AUTO) -> int:
     """Scratch bytes rest_draft can use for a call of B contexts on the current device (0 when
     the call takes the single-context path)."""
-    prm = _Params(n_max, n_min, K, m, N, sample_mode | search)
+    prm = _Params(n_max, n_min, K, m, N, sample_mode, search)
     return int(lib().rest_draft_workspace_bytes(ctypes.byref(prm), B))
 
 
@@ -235,7 +236,7 @@ def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=6
     B = ctx.shape[0]
     if out is None:
         out = alloc_draft_output(B, N, ctx.device)
-    prm = _Params(n_max, n_min, K, m, N, sample_mode | search)
+    prm = _Params(n_max, n_min, K, m, N, sample_mode, search)
     ws_ptr, ws_bytes = 0, 0
     if workspace is None:
         need = L.rest_draft_workspace_bytes(ctypes.byref(prm), B)

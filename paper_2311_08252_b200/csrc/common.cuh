@@ -4,6 +4,7 @@
 #include <stdint.h>
 
 #include "rest.h"
+#include "rest_aids.h"
 
 namespace rest {
 
@@ -13,6 +14,9 @@ void count_launch(int n = 1);
 // Raises a kernel's dynamic shared-memory limit on the current device when `bytes` exceeds
 // what was set before (kernel_slot: small per-kernel index used for the per-device cache).
 cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t bytes);
+// Streaming multiprocessors of the current device (asked once per device); 0 when there is no
+// usable device.
+int sm_count();
 // One slot per kernel instance, library-wide: two kernels on one slot would skip each other's
 // attribute call.  The draft kernel's instances take kSmemSlotDraft + 0 ... 13.
 constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 14, kSmemSlotAttnWide = 15, kSmemSlots = 16;

@@ -36,6 +36,25 @@ cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t byte
   return e;
 }
 
+int sm_count() {
+  constexpr int kMaxDev = 64;
+  static std::atomic<int> cache[kMaxDev];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+  const bool cached = dev >= 0 && dev < kMaxDev;
+  if (cached) {
+    const int have = cache[dev].load(std::memory_order_relaxed);
+    if (have > 0) return have;
+  }
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  if (cached) cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 }  // namespace rest
 
 namespace {
@@ -98,7 +117,8 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
     uint32_t* d_flags = static_cast<uint32_t*>(d_aux);
     uint32_t* d_seen = d_flags + 64;
     REST_CUDA_TRY(cudaMemsetAsync(d_aux, 0, need, st));
-    int blocks = (int)((n_tokens + 255) / 256 < 148 * 16 ? (n_tokens + 255) / 256 : 148 * 16);
+    const uint64_t wave = (uint64_t)(rest::sm_count() > 0 ? rest::sm_count() : 148) * 16;
+    int blocks = (int)((n_tokens + 255) / 256 < wave ? (n_tokens + 255) / 256 : wave);
     if (sa_bytes == 4)
       validate_kernel<int32_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int32_t*>(d_sa),
                                                        (int64_t)n_tokens, vocab, d_seen, d_flags);

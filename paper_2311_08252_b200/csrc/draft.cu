@@ -704,12 +704,23 @@ rest_draft_kernel(DraftArgs a) {
       if (w < Wm) a.mask[o + w] = bits[w];
   }
   __syncthreads();
+  if (s.err != 0) {
+    // an inconsistency met while the tree was being written: the caller gets the empty tree
+    // that every other reported problem gives, not a half-built one
+    for (int i = tid; i < N; i += NT) {
+      int64_t o = (int64_t)b * N + i;
+      a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
+      for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (i >> 5)) ? (1u << (i & 31)) : 0u;
+      if (a.node_count) a.node_count[o] = 0;
+    }
+  }
   if (tid == 0) {
+    const bool ok = s.err == 0;
     a.status[b] = s.err;
-    a.n_nodes[b] = nn;
-    a.match_n[b] = n_win;
-    a.match_range[2 * b] = lo;
-    a.match_range[2 * b + 1] = hi;
+    a.n_nodes[b] = ok ? nn : 0;
+    a.match_n[b] = ok ? n_win : 0;
+    a.match_range[2 * b] = ok ? lo : 0;
+    a.match_range[2 * b + 1] = ok ? hi : 0;
   }
 }
 
@@ -732,9 +743,8 @@ static rest_status wants_batched(int search, int B, bool with_scratch, bool* bat
     // Below a few contexts per SM a call lasts as long as its slowest contexts and the shortest
     // dependent chain wins.  Measured crossover on 148 SMs: between 512 and 1024 contexts for the
     // three-launch form, between 1024 and 4096 for the one-launch form.
-    int dev = 0, sms = 0;
-    REST_CUDA_TRY(cudaGetDevice(&dev));
-    REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int sms = rest::sm_count();
+    if (sms <= 0) return rest::note_cuda_error(cudaErrorNoDevice, "sm_count");
     *batched = B >= (with_scratch ? 5 : 16) * sms;
   }
   return REST_OK;
@@ -745,7 +755,7 @@ static size_t split_workspace_bytes(int B) { return (2 * (size_t)B + 16) * sizeo
 extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params* prm, int32_t B) {
   if (!prm || B <= 0) return 0;
   bool batched = false;
-  if (wants_batched(prm->sample_mode & ~REST_SAMPLE_MASK, B, true, &batched) != REST_OK || !batched) return 0;
+  if (wants_batched(prm->search_path, B, true, &batched) != REST_OK || !batched) return 0;
   return split_workspace_bytes(B);
 }
 
@@ -764,8 +774,8 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     return REST_INVALID_ARG;
   if (prm->n_min < 1 || prm->n_max < prm->n_min || prm->K < 1 || prm->m < 1 || prm->N < 1)
     return REST_INVALID_ARG;
-  const int sample_mode = prm->sample_mode & REST_SAMPLE_MASK;
-  const int search = prm->sample_mode & ~REST_SAMPLE_MASK;
+  const int sample_mode = prm->sample_mode;
+  const int search = prm->search_path;
   if (sample_mode != REST_SAMPLE_STRIDED && sample_mode != REST_SAMPLE_FIRST_K)
     return REST_INVALID_ARG;
   if (search != REST_SEARCH_AUTO && search != REST_SEARCH_SINGLE && search != REST_SEARCH_BATCHED)
@@ -802,9 +812,7 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     // a call with at most one context per SM lasts as long as its slowest context: give each
     // context the whole SM (not the single context: its typical candidate list is short and
     // the larger block only adds barrier time)
-    int dev = 0, sms = 0;
-    REST_CUDA_TRY(cudaGetDevice(&dev));
-    REST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int sms = rest::sm_count();
     if (big || (B > 1 && B <= sms))
       return narrow ? launch(rest_draft_kernel<int32_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem)
                     : launch(rest_draft_kernel<int64_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem);

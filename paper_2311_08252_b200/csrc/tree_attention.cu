@@ -51,7 +51,6 @@ constexpr int kRowBytes = kD * 2;     // 256
 constexpr int kTileBytes = kBN * kRowBytes;   // 16 KB
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr int kNumSMs = 148;
 
 struct AttnArgs {
   const __nv_bfloat16 *q, *k, *v;
@@ -682,7 +681,8 @@ tree_attention_ws_kernel(AttnArgs a, const __grid_constant__ CUtensorMap tm_q,
 // exponentials is only raised when a tile's maximum exceeds it by more than 2^8, and only then
 // is the O row rescaled in TMEM (rare after the first tiles), so the per-tile work is
 // load S, mask, exp2, pack P.  Probabilities are at most 2^8, harmless in bf16 / fp32.
-// Splits write un-normalised partials to the caller's workspace; the combine kernel merges.
+// Key splits are merged inside a cluster of up to 8 blocks through distributed shared memory;
+// only beyond 8 splits do the cluster results go to the caller's workspace for the combine kernel.
 // =======================================================================================
 constexpr int kWideQBytes = 128 * kRowBytes;            // 32 KB: 128 rows x 128 dims
 constexpr int kWidePBytes = 128 * 128;                  // 16 KB: 128 rows x 64 keys
@@ -1208,8 +1208,44 @@ EncodeTiledFn encode_tiled_fn() {
   }();
   return fn;
 }
+// A tensor map depends only on (base, extents, strides); a decoding loop passes the same few
+// tensors call after call, so each host thread remembers the maps it has encoded in a small
+// direct-mapped table and a repeated call costs a key comparison instead of a driver call.
+struct MapKey {
+  const void* base;
+  int64_t rows, heads, batch, row_stride, head_stride, batch_stride;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && rows == o.rows && heads == o.heads && batch == o.batch &&
+           row_stride == o.row_stride && head_stride == o.head_stride && batch_stride == o.batch_stride;
+  }
+};
+struct MapEntry { MapKey key; CUtensorMap map; int slot[3]; bool valid; };
+constexpr int kMapCacheEntries = 256;
+
+bool encode_box_map_uncached(CUtensorMap* map, const void* base, int64_t rows, int64_t heads, int64_t batch,
+                             int64_t row_stride, int64_t head_stride, int64_t batch_stride, int (&slot)[3]);
+
 bool encode_box_map(CUtensorMap* map, const void* base, int64_t rows, int64_t heads, int64_t batch,
                     int64_t row_stride, int64_t head_stride, int64_t batch_stride, int (&slot)[3]) {
+  static thread_local MapEntry cache[kMapCacheEntries];
+  const MapKey key{base, rows, heads, batch, row_stride, head_stride, batch_stride};
+  uint64_t hsh = reinterpret_cast<uintptr_t>(base) >> 8;
+  hsh = (hsh ^ (hsh >> 17) ^ (uint64_t)rows * 0x9E3779B97F4A7C15ull) * 0xD6E8FEB86659FD93ull;
+  MapEntry& e = cache[(hsh >> 40) % kMapCacheEntries];
+  if (e.valid && e.key == key) {
+    *map = e.map;
+    slot[0] = e.slot[0]; slot[1] = e.slot[1]; slot[2] = e.slot[2];
+    return true;
+  }
+  if (!encode_box_map_uncached(map, base, rows, heads, batch, row_stride, head_stride, batch_stride, slot))
+    return false;
+  e.key = key; e.map = *map; e.valid = true;
+  e.slot[0] = slot[0]; e.slot[1] = slot[1]; e.slot[2] = slot[2];
+  return true;
+}
+
+bool encode_box_map_uncached(CUtensorMap* map, const void* base, int64_t rows, int64_t heads, int64_t batch,
+                             int64_t row_stride, int64_t head_stride, int64_t batch_stride, int (&slot)[3]) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   // outer dimensions in order of increasing stride (size-1 dimensions last: their stride is unused)
@@ -1252,7 +1288,8 @@ bool encode_box_map(CUtensorMap* map, const void* base, int64_t rows, int64_t he
 int cluster_capacity(bool wide, int c) {
   constexpr int kMaxDev = 64;
   static std::atomic<int> cache[kMaxDev][2][kMaxCluster + 1];
-  const int nominal = (2 * kNumSMs) / c;
+  const int sms = rest::sm_count();
+  const int nominal = (2 * (sms > 0 ? sms : 148)) / c;     // 148: size queries on a machine without a GPU
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { (void)cudaGetLastError(); return nominal; }
   const int have = cache[dev][wide ? 1 : 0][c].load(std::memory_order_relaxed);
@@ -1355,9 +1392,15 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   if (B == 0) return REST_OK;
   if (!d_q || !d_k || !d_v || !d_kv_len || !d_mask || !d_out) return REST_INVALID_ARG;
   if (!(scale > 0.f) || !(scale < INFINITY)) return REST_INVALID_ARG;
-  if (D != kD || N > REST_MAX_N || (N % 16) != 0 || (H % H_kv) != 0) return REST_UNSUPPORTED;
+  if (D != kD || N > REST_MAX_N || (H % H_kv) != 0) return REST_UNSUPPORTED;
   for (int i = 0; i < 9; ++i)
     if (strides[i] < 0 || (strides[i] % 8) != 0) return REST_INVALID_ARG;
+  {
+    // a dimension that is actually stepped through must advance by at least one row of D elements
+    const int64_t extent[9] = {B, N, H, B, H_kv, max_kv, B, N, H};
+    for (int i = 0; i < 9; ++i)
+      if (extent[i] > 1 && strides[i] < D) return REST_INVALID_ARG;
+  }
   if ((reinterpret_cast<uintptr_t>(d_q) | reinterpret_cast<uintptr_t>(d_k) |
        reinterpret_cast<uintptr_t>(d_v) | reinterpret_cast<uintptr_t>(d_out)) & 15)
     return REST_INVALID_ARG;
@@ -1387,7 +1430,7 @@ extern "C" rest_status rest_tree_attention(const void* d_q, const void* d_k, con
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Grouped KV heads with N = 64 and a batch that fills the GPU without key splits: two query
   // heads of a group share one 128-row block of the wide kernel (their K/V is streamed once)
-  a.pack = (N == 64 && (a.group % 2) == 0 && (int64_t)B * H / 2 >= 2 * kNumSMs) ? 2 : 1;
+  a.pack = (N == 64 && (a.group % 2) == 0 && (int64_t)B * H / 2 >= 2 * rest::sm_count()) ? 2 : 1;
   const bool wide = N > 64 || a.pack == 2;
   a.NBLK = N > 64 ? (N + 127) / 128 : 1;
   const size_t smem = wide ? (size_t)wide_smem_bytes() : (size_t)ws_smem_bytes();
@@ -1477,18 +1520,19 @@ constexpr size_t kStaticScratchBytes = REST_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device
+std::atomic<void*> g_static_scratch_addr[kMaxDevices];   // device address of g_static_scratch, per device
 
 rest_status static_scratch_pointer(void** out) {
   int dev = 0;
   REST_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return REST_UNSUPPORTED;
-  if (g_static_scratch_addr[dev] == nullptr) {
-    void* p = nullptr;
+  void* p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
+    // two threads may both ask the first time; they get the same address
     REST_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
-    g_static_scratch_addr[dev] = p;
+    g_static_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_static_scratch_addr[dev];
+  *out = p;
   return REST_OK;
 }
 

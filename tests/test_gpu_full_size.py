@@ -14,7 +14,7 @@ import torch
 import datagen
 import oracle
 import paper_2311_08252_b200 as rest
-from gpu_util import assert_draft_equal, attention_errors, bits, gpu_draft, to_dev
+from gpu_util import DRAFT_KEYS, assert_draft_equal, attention_errors, bits, gpu_draft, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -71,23 +71,44 @@ def test_draft_full_single_stream_datastore():
     assert (ref["n_nodes"] > 0).mean() > 0.5
 
 
+def host_memory_available():
+    import psutil
+    return psutil.virtual_memory().available
+
+
 @pytest.mark.parametrize("name,n_tokens", [("stress", 500_000_000), ("batched", 1_000_000_000),
                                            ("large", 1_000_000_000)])
 def test_draft_largest_datastores(name, n_tokens):
     """The 500 M-token stress datastore, the 1 B-token batched one, and the large recipe with its
-    int64 suffix array at 1 B tokens (the 4 B-token array cannot be built in this host's memory).
-    Building these suffix arrays on the host takes minutes, so the test only runs when
-    REST_FULL_DATASTORES=1."""
-    import os
-    if os.environ.get("REST_FULL_DATASTORES") != "1":
-        pytest.skip("set REST_FULL_DATASTORES=1 to build the 0.5-1 B-token suffix arrays")
+    int64 suffix array at 1 B tokens, each at its configuration's batch size.  The suffix array
+    is built on the device (rest_suffix_array_build) and copied back, so that the oracle searches
+    the very same array."""
     w = datagen.WORKLOADS[name].scaled(n_tokens=n_tokens)
+    need_dev = n_tokens * (4 + w.sa_bytes) + rest.lib().rest_suffix_array_workspace_bytes(n_tokens)
+    free, _ = torch.cuda.mem_get_info()
+    if free < need_dev + (2 << 30):
+        pytest.skip(f"needs {need_dev / 2**30:.0f} GiB of device memory, {free / 2**30:.0f} GiB free")
+    need_host = n_tokens * (4 + w.sa_bytes) * 2
+    if host_memory_available() < need_host + (4 << 30):
+        pytest.skip(f"needs {need_host / 2**30:.0f} GiB of host memory")
     T = datagen.make_tokens(w)
-    sa = datagen.build_suffix_array(T, w.vocab, sa_bytes=w.sa_bytes)
+    d_T = to_dev(T)
+    d_sa = rest.rest_suffix_array_build(d_T, w.sa_bytes)
+    torch.cuda.empty_cache()
+    ds = rest.Datastore(d_T, d_sa, w.vocab, validate=True)
+    sa = d_sa.cpu().numpy()
     B, Lc = w.B, 64
     ctx = datagen.make_contexts(w, T, B=B, Lc=Lc)
     ctx_len = np.full(B, Lc, np.int32)
-    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, K=w.K, m=w.m, N=w.N)
-    got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, K=w.K, m=w.m, N=w.N)
-    assert_draft_equal(got, ref, f"{name}, {n_tokens} tokens")
+    kw = dict(K=w.K, m=w.m, N=w.N)
+    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+    for search in (rest.REST_SEARCH_SINGLE, rest.REST_SEARCH_BATCHED):
+        out = rest.rest_draft(ds, to_dev(ctx), to_dev(ctx_len), search=search, **kw)
+        torch.cuda.synchronize()
+        got = {k: getattr(out, k).cpu().numpy() for k in DRAFT_KEYS}
+        got["mask"] = out.mask.cpu().numpy().view(np.uint32)
+        assert_draft_equal(got, ref, f"{name}, {n_tokens} tokens, search {search}")
     assert (ref["n_nodes"] > 0).mean() > 0.5
+    ds.close()
+    del d_T, d_sa, ds
+    torch.cuda.empty_cache()

@@ -71,6 +71,28 @@ def test_strided_cache_and_aliased_length():
     assert np.array_equal(d_len.cpu().numpy(), want_len)
 
 
+def test_aliased_length_with_a_grid_far_beyond_one_wave():
+    """Thousands of blocks with the new length written over the old one: no block of a context
+    may see the updated length (which would move the wrong rows)."""
+    rng = np.random.default_rng(11)
+    B, H, N, D, Lcap, md = 2048, 8, 16, 128, 40, 16
+    kb = rng.integers(0, 65536, size=(B, H, Lcap, D)).astype(np.uint16)
+    vb = rng.integers(0, 65536, size=(B, H, Lcap, D)).astype(np.uint16)
+    kv_len = rng.integers(0, Lcap - N - md, size=B).astype(np.int32)
+    lens = rng.integers(1, md + 1, size=B).astype(np.int32)
+    nodes = np.full((B, md), -1, np.int32)
+    for b in range(B):
+        nodes[b, :lens[b]] = np.sort(rng.choice(N, size=lens[b], replace=False))
+    want_k, want_v, want_len = oracle.kv_commit(kb, vb, kv_len, nodes, lens)
+    k, v = bf16_from_bits(kb), bf16_from_bits(vb)
+    d_len = to_dev(kv_len)
+    rest.rest_kv_commit(k, v, d_len, to_dev(nodes), to_dev(lens), N, new_kv_len=d_len)
+    torch.cuda.synchronize()
+    assert np.array_equal(d_len.cpu().numpy(), want_len)
+    assert np.array_equal(bits_of(k), want_k)
+    assert np.array_equal(bits_of(v), want_v)
+
+
 def test_empty_batch_and_zero_depth():
     k = torch.zeros((0, 2, 64, 128), dtype=torch.bfloat16, device="cuda")
     e = torch.zeros((0,), dtype=torch.int32, device="cuda")
