@@ -61,7 +61,7 @@ enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1 };
  * rest_draft_workspace_bytes asks for, see d_ws).  AUTO picks BATCHED when the call has at
  * least 5 contexts per SM and that scratch, or at least 16 contexts per SM without it. */
 enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 1, REST_SEARCH_BATCHED = 2 };
-enum { REST_DS_VALIDATE = 1u };
+enum { REST_DS_VALIDATE = 1u, REST_DS_INDEX = 2u };
 
 /* Limits of this implementation. */
 enum {
@@ -96,9 +96,16 @@ typedef struct {
  *              as unsigned integers, a suffix that is a proper prefix of another sorts first).
  *              Only the order on the first n_max + m tokens matters to rest_draft.
  *   flags      REST_DS_VALIDATE: check on the device that d_sa is a permutation ordered on the
- *              first 32 tokens and that tokens are in range; needs d_aux of
- *              rest_datastore_aux_bytes() bytes; synchronises `stream`; returns
- *              REST_BAD_DATASTORE on failure.  Without the flag d_aux may be NULL.
+ *              first 32 tokens and that tokens are in range; synchronises `stream`; returns
+ *              REST_BAD_DATASTORE on failure.
+ *              REST_DS_INDEX: build a bucket index into d_aux (asynchronously on `stream`): for
+ *              every token the suffix-array range of the suffixes that start with it, and a hash
+ *              table with the ranges of the frequent token pairs (up to 256 MiB).  rest_draft
+ *              then starts each search inside such a range instead of over the whole array:
+ *              fewer dependent reads, identical results.  Needs vocab <= 2^22 (ignored beyond).
+ *   d_aux      device scratch of rest_datastore_aux_bytes() bytes, 256-byte aligned, needed with
+ *              either flag (NULL otherwise).  With REST_DS_INDEX the handle keeps using it: it
+ *              must stay allocated and untouched until rest_datastore_destroy.
  *   out        receives a host handle; free it with rest_datastore_destroy (device arrays stay
  *              the caller's).
  */

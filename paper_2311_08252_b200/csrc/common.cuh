@@ -27,12 +27,37 @@ constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 14, kSmemSlotAttnWide = 15, kS
     if (e_ != cudaSuccess) return ::rest::note_cuda_error(e_, #expr);    \
   } while (0)
 
+// Bucket index over the suffix array (an accelerator built by rest_datastore_create; results
+// never depend on it).  `first[t]` is the first suffix-array slot whose suffix starts with token
+// t (first[vocab] = n_tokens), so suffixes starting with t occupy [first[t], first[t + 1]).
+// `table` is a hash table over the frequent token pairs (t0, t1): groups of four 32-byte
+// entries {key, lo, hi, unused}; an entry says that the suffixes starting with (t0, t1) occupy
+// slots [lo, hi).  Pairs that occur fewer times than a size-dependent minimum are not stored;
+// a search for them starts from the first-token range instead.
+struct BucketIndex {
+  const long long* first;               // null: no index
+  const unsigned long long* table;      // 4 words per entry
+  uint32_t group_mask;                  // number of groups - 1 (a group = 4 entries = 128 bytes)
+};
+constexpr unsigned long long kIndexEmptyKey = ~0ull;
+__host__ __device__ inline unsigned long long index_pair_key(uint32_t t0, uint32_t t1) {
+  return ((unsigned long long)t0 << 32) | (unsigned long long)t1;
+}
+__host__ __device__ inline uint32_t index_group_of(unsigned long long key, uint32_t group_mask) {
+  key ^= key >> 29;
+  key *= 0xBF58476D1CE4E5B9ull;
+  key ^= key >> 32;
+  key *= 0x94D049BB133111EBull;
+  return (uint32_t)(key >> 35) & group_mask;
+}
+
 struct DatastoreView {
   const int32_t* tokens;
   const void* sa;
   int64_t n_tokens;
   int32_t sa_bytes;
   uint32_t vocab;
+  BucketIndex idx;
 };
 
 }  // namespace rest

@@ -91,11 +91,120 @@ __global__ void validate_kernel(const int32_t* __restrict__ T, const SaT* __rest
   if (bad) atomicOr(flags, bad);
 }
 
+// ---- bucket index ------------------------------------------------------------------------
+constexpr uint32_t kIndexMaxVocab = 1u << 22;       // the first-token table has vocab + 1 entries
+constexpr uint64_t kIndexMinEntries = 1ull << 12, kIndexMaxEntries = 1ull << 23;
+
+struct IndexLayout {
+  uint64_t entries;      // hash-table entries (a power of two; 0 = no index for this datastore)
+  int64_t min_run;       // token pairs with fewer occurrences are not stored
+  size_t first_bytes, table_bytes, total;
+};
+IndexLayout index_layout(uint64_t n, uint32_t vocab) {
+  IndexLayout l = {};
+  if (vocab > kIndexMaxVocab || n < 2) return l;
+  uint64_t e = kIndexMinEntries;
+  while (e < n / 2 && e < kIndexMaxEntries) e <<= 1;
+  l.entries = e;
+  // at most n / min_run pairs are stored: the table stays at most one eighth full, so a group
+  // of four overflows practically never (and a pair that finds its group full is just left out)
+  l.min_run = (int64_t)((8 * n + e - 1) / e);
+  if (l.min_run < 1) l.min_run = 1;
+  l.first_bytes = (((size_t)vocab + 1) * 8 + 255) / 256 * 256;
+  l.table_bytes = (size_t)e * 32;
+  l.total = l.first_bytes + l.table_bytes;
+  return l;
+}
+size_t validation_bytes(uint64_t n) {
+  // one "seen" bit per position, rounded up to 32-bit words, plus one 256-byte block of flags
+  return ((n + 31) / 32) * 4 + 256;
+}
+
+// The token pair a suffix starts with; t1 = -1 for the one suffix that is a single token long.
+// false when the entry or a token is out of range (such a datastore gets no usable index).
+template <typename SaT>
+__device__ __forceinline__ bool pair_at(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
+                                        int64_t n, uint32_t vocab, int64_t slot, int32_t& t0, int32_t& t1) {
+  const int64_t p = (int64_t)sa[slot];
+  if (p < 0 || p >= n) return false;
+  t0 = T[p];
+  t1 = p + 1 < n ? T[p + 1] : -1;
+  return t0 >= 0 && (uint32_t)t0 < vocab && (t1 == -1 || (t1 >= 0 && (uint32_t)t1 < vocab));
+}
+
+// One thread per suffix-array slot.  The slot where a first token begins writes first[t]; the
+// slots where a run of one token pair begins and ends write that pair's lo and hi, provided the
+// run has at least min_run members (seen by looking min_run - 1 slots ahead or back).
+template <typename SaT>
+__global__ void index_build_kernel(const int32_t* __restrict__ T, const SaT* __restrict__ sa, int64_t n,
+                                   uint32_t vocab, int64_t min_run, long long* __restrict__ first,
+                                   unsigned long long* __restrict__ table, uint32_t group_mask) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    int32_t t0, t1, a0 = -2, a1 = -2, b0 = -2, b1 = -2;
+    if (!pair_at(T, sa, n, vocab, i, t0, t1)) continue;
+    if (i > 0 && !pair_at(T, sa, n, vocab, i - 1, a0, a1)) a0 = -2;
+    if (i + 1 < n && !pair_at(T, sa, n, vocab, i + 1, b0, b1)) b0 = -2;
+    if (i == 0 || a0 != t0) first[t0] = i;
+    if (t1 < 0) continue;
+    const bool starts = i == 0 || a0 != t0 || a1 != t1;
+    const bool ends = i + 1 == n || b0 != t0 || b1 != t1;
+    if (!starts && !ends) continue;
+    bool long_enough = true;
+    if (min_run > 1) {
+      long_enough = false;                       // a run of one is shorter than any minimum above one
+      if (!(starts && ends)) {
+        const int64_t far = starts ? i + min_run - 1 : i - min_run + 1;
+        int32_t f0, f1;
+        long_enough = far >= 0 && far < n && pair_at(T, sa, n, vocab, far, f0, f1) && f0 == t0 && f1 == t1;
+      }
+    }
+    if (!long_enough) continue;
+    const unsigned long long key = rest::index_pair_key((uint32_t)t0, (uint32_t)t1);
+    unsigned long long* grp = table + (size_t)rest::index_group_of(key, group_mask) * 16;
+    for (int e = 0; e < 4; ++e) {
+      const unsigned long long cur = atomicCAS(grp + e * 4, rest::kIndexEmptyKey, key);
+      if (cur == rest::kIndexEmptyKey || cur == key) {
+        if (starts) grp[e * 4 + 1] = (unsigned long long)i;
+        if (ends) grp[e * 4 + 2] = (unsigned long long)(i + 1);
+        break;
+      }
+    }
+  }
+}
+
+// first[t] of a token that never starts a suffix = first[] of the next token that does:
+// a suffix minimum from the right, 1024 entries at a time (one block).
+__global__ void __launch_bounds__(1024)
+index_fill_kernel(long long* __restrict__ first, uint32_t vocab, int64_t n) {
+  __shared__ long long buf[1024];
+  __shared__ long long carry;
+  if (threadIdx.x == 0) { carry = n; first[vocab] = n; }
+  __syncthreads();
+  for (int64_t top = (int64_t)vocab; top > 0; top -= 1024) {
+    const int64_t t = top - 1 - threadIdx.x;          // thread 0 takes the rightmost entry
+    long long v = t >= 0 ? first[t] : -1;
+    buf[threadIdx.x] = v < 0 ? 0x7FFFFFFFFFFFFFFFll : v;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {              // inclusive minimum over threads 0 .. x
+      long long u = threadIdx.x >= o ? buf[threadIdx.x - o] : 0x7FFFFFFFFFFFFFFFll;
+      __syncthreads();
+      if (u < buf[threadIdx.x]) buf[threadIdx.x] = u;
+      __syncthreads();
+    }
+    const long long c = carry;
+    const long long r = buf[threadIdx.x] < c ? buf[threadIdx.x] : c;
+    if (t >= 0) first[t] = r;
+    __syncthreads();
+    if (threadIdx.x == 1023) carry = r;
+    __syncthreads();
+  }
+}
+
 }  // namespace
 
-extern "C" size_t rest_datastore_aux_bytes(uint64_t n_tokens, int32_t, uint32_t) {
-  // one "seen" bit per position, rounded up to 32-bit words, plus one 256-byte block of flags
-  return ((n_tokens + 31) / 32) * 4 + 256;
+extern "C" size_t rest_datastore_aux_bytes(uint64_t n_tokens, int32_t, uint32_t vocab) {
+  return index_layout(n_tokens, vocab).total + validation_bytes(n_tokens);
 }
 
 extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n_tokens,
@@ -109,14 +218,19 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
   if (sa_bytes != 4 && sa_bytes != 8) return REST_INVALID_ARG;
   if (sa_bytes == 4 && n_tokens > 0x7FFFFFFFull) return REST_INVALID_ARG;
   if (n_tokens > (1ull << 40)) return REST_UNSUPPORTED;
+  if (flags & ~(REST_DS_VALIDATE | REST_DS_INDEX)) return REST_INVALID_ARG;
+  const IndexLayout il = (flags & REST_DS_INDEX) ? index_layout(n_tokens, vocab) : IndexLayout{};
+  const size_t aux_need = il.total + ((flags & REST_DS_VALIDATE) ? validation_bytes(n_tokens) : 0);
+  if (aux_need > 0) {
+    if (!d_aux || (reinterpret_cast<uintptr_t>(d_aux) & 255)) return REST_INVALID_ARG;
+    if (aux_bytes < aux_need) return REST_WORKSPACE_TOO_SMALL;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (flags & REST_DS_VALIDATE) {
-    size_t need = rest_datastore_aux_bytes(n_tokens, sa_bytes, vocab);
-    if (!d_aux) return REST_INVALID_ARG;
-    if (aux_bytes < need) return REST_WORKSPACE_TOO_SMALL;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    uint32_t* d_flags = static_cast<uint32_t*>(d_aux);
+    const size_t need = validation_bytes(n_tokens);
+    uint32_t* d_flags = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(d_aux) + il.total);
     uint32_t* d_seen = d_flags + 64;
-    REST_CUDA_TRY(cudaMemsetAsync(d_aux, 0, need, st));
+    REST_CUDA_TRY(cudaMemsetAsync(d_flags, 0, need, st));
     const uint64_t wave = (uint64_t)(rest::sm_count() > 0 ? rest::sm_count() : 148) * 16;
     int blocks = (int)((n_tokens + 255) / 256 < wave ? (n_tokens + 255) / 256 : wave);
     if (sa_bytes == 4)
@@ -132,8 +246,31 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
     REST_CUDA_TRY(cudaStreamSynchronize(st));
     if (h_flags != 0) return REST_BAD_DATASTORE;
   }
+  rest::BucketIndex idx = {nullptr, nullptr, 0};
+  if (il.entries > 0) {
+    // built after a successful validation (when asked for), on the same stream, without a sync:
+    // calls that use the handle on this stream see the finished index
+    unsigned char* base = static_cast<unsigned char*>(d_aux);
+    long long* first = reinterpret_cast<long long*>(base);
+    unsigned long long* table = reinterpret_cast<unsigned long long*>(base + il.first_bytes);
+    REST_CUDA_TRY(cudaMemsetAsync(base, 0xFF, il.total, st));      // first[] = -1, keys = empty, lo = hi = -1
+    const uint32_t group_mask = (uint32_t)(il.entries / 4 - 1);
+    const uint64_t wave = (uint64_t)(rest::sm_count() > 0 ? rest::sm_count() : 148) * 16;
+    const int blocks = (int)((n_tokens + 255) / 256 < wave ? (n_tokens + 255) / 256 : wave);
+    if (sa_bytes == 4)
+      index_build_kernel<int32_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int32_t*>(d_sa),
+                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask);
+    else
+      index_build_kernel<int64_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int64_t*>(d_sa),
+                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask);
+    index_fill_kernel<<<1, 1024, 0, st>>>(first, vocab, (int64_t)n_tokens);
+    rest::count_launch(2);
+    REST_CUDA_TRY(cudaGetLastError());
+    idx.first = first; idx.table = table; idx.group_mask = group_mask;
+  }
   rest_datastore* ds = static_cast<rest_datastore*>(malloc(sizeof(rest_datastore)));
   if (!ds) return REST_INVALID_ARG;
+  ds->v.idx = idx;
   ds->v.tokens = d_tokens;
   ds->v.sa = d_sa;
   ds->v.n_tokens = (int64_t)n_tokens;

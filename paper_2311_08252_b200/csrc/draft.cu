@@ -2,18 +2,25 @@
 // (Trie weights and the c heaviest nodes) and the breadth-first pseudo sequence with its
 // ancestor mask (Sec. 3.2), one thread block per context, everything in one launch.
 //
-// Phases inside the block (16 warps):
-//   1 search   warp w looks for suffix length n_min + w: a 32-ary lower bound (every lane
-//              probes one suffix-array slot per round, a ballot narrows the interval), then,
-//              if the slot matches, a galloping + 32-ary upper bound.  The longest length
-//              with a non-empty range wins.
-//   2 gather   one candidate row per thread, in suffix-array order, which is also the
-//              lexicographic order of the continuations.  Only the common-prefix length with
-//              the previous row (by warp shuffle) and the row length are kept: for every
-//              depth d the bitmap "row j starts a new Trie node at depth d" (lcp_j < d).
-//   3 select   weight of node (d, j) = distance to the next set bit of bitmap d.  The N
-//              largest by (weight desc, depth asc, row asc) are found with a two-level radix
-//              histogram over (weight, depth) and an ordered scan over rows for the ties.
+// Phases inside the block:
+//   1 search   a warp per suffix length: the bucket index (when the datastore has one) gives the
+//              suffix-array range of the query's first token pair, a 32-ary lower bound inside
+//              it (every lane probes one slot per round, a ballot narrows the interval) finds
+//              the first match, and for the longest length that matched a galloping + 32-ary
+//              upper bound finds the end of the run.
+//   2 gather   candidate rows in suffix-array order, which is also the lexicographic order of
+//              the continuations.  A warp fetches its 32 rows (and the row before them) with
+//              coalesced loads: lane l reads word l, 32 + l, ... of the rows laid end to end,
+//              so a load touches three or four rows instead of 32, and the rows pass through
+//              a shared-memory staging area.  Only the common-prefix length with the previous
+//              row survives: for every depth d the bitmap "row j starts a new Trie node at
+//              depth d" (lcp_j < d).
+//   3 select   weight of node (d, j) = distance to the next set bit of bitmap d.  All passes
+//              run over (depth, bitmap word) pairs, not over rows: two adjacent set bits are a
+//              node of weight 1 (counted with one popcount per word), a set bit followed by a
+//              clear one is a heavier node (visited one by one).  The N largest by (weight
+//              desc, depth asc, row asc) come from a two-level radix histogram over (weight,
+//              depth) and a prefix sum over the words of the tie depth.
 //   4 emit     rank the kept nodes by (depth, row), look up parents through the bitmap of the
 //              depth above, build ancestor masks, fetch the node tokens.
 #include <cuda_runtime.h>
@@ -66,6 +73,7 @@ struct DraftArgs {
   int32_t *n_nodes, *match_n;
   int64_t* match_range;
   int32_t *node_count, *status;
+  rest::BucketIndex idx;
   int nwords;   // bitmap words per depth
   int kcap;     // rows the block's shared memory holds, a multiple of 32
   // three-launch form of the batched path: the search launch sorts the contexts that matched
