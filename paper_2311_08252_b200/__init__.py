@@ -26,6 +26,7 @@ REST_SEARCH_AUTO = 0
 REST_SEARCH_SINGLE = 1
 REST_SEARCH_BATCHED = 2
 REST_DS_VALIDATE = 1
+REST_DS_INDEX = 2
 
 EXPORTS = (
     "rest_datastore_aux_bytes", "rest_datastore_create", "rest_datastore_destroy",
@@ -147,9 +148,12 @@ def launch_count() -> int:
 
 class Datastore:
     """Handle over device-resident tokens int32[n] and suffix array int32[n] / int64[n].
-    The tensors are borrowed: this object keeps references so they outlive the handle."""
+    The tensors are borrowed: this object keeps references so they outlive the handle.
+    index=True also builds the bucket index (token and token-pair ranges of the suffix array)
+    that lets rest_draft start its searches inside a small range; results do not depend on it."""
 
-    def __init__(self, tokens, sa, vocab: int, validate: bool = False, stream=None):
+    def __init__(self, tokens, sa, vocab: int, validate: bool = False, stream=None,
+                 index: bool = True):
         import torch
         if not (tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()):
             raise RestError("tokens must be a contiguous int32 CUDA tensor")
@@ -161,15 +165,17 @@ class Datastore:
         self.sa_bytes = sa.element_size()
         L = lib()
         aux, aux_bytes = None, 0
-        if validate:
+        flags = (REST_DS_VALIDATE if validate else 0) | (REST_DS_INDEX if index else 0)
+        if flags:
             aux_bytes = L.rest_datastore_aux_bytes(self.n_tokens, self.sa_bytes, self.vocab)
             aux = torch.empty(aux_bytes, dtype=torch.uint8, device=tokens.device)
         h = ctypes.c_void_p()
         rc = L.rest_datastore_create(tokens.data_ptr(), self.n_tokens, sa.data_ptr(), self.sa_bytes,
-                                     self.vocab, REST_DS_VALIDATE if validate else 0, _ptr(aux),
-                                     aux_bytes, _stream(stream), ctypes.byref(h))
+                                     self.vocab, flags, _ptr(aux), aux_bytes, _stream(stream),
+                                     ctypes.byref(h))
         _check(rc, "rest_datastore_create")
         self._h = h
+        self._aux = aux if index else None      # the handle reads the index for its whole life
 
     def close(self):
         if getattr(self, "_h", None):
@@ -183,8 +189,8 @@ class Datastore:
             pass
 
 
-def rest_datastore_create(tokens, sa, vocab, validate=False, stream=None) -> Datastore:
-    return Datastore(tokens, sa, vocab, validate, stream)
+def rest_datastore_create(tokens, sa, vocab, validate=False, stream=None, index=True) -> Datastore:
+    return Datastore(tokens, sa, vocab, validate, stream, index)
 
 
 @dataclass

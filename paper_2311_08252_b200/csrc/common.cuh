@@ -38,6 +38,7 @@ struct BucketIndex {
   const long long* first;               // null: no index
   const unsigned long long* table;      // 4 words per entry
   uint32_t group_mask;                  // number of groups - 1 (a group = 4 entries = 128 bytes)
+  const uint32_t* unusable;             // non-zero: the build met an entry or token out of range
 };
 constexpr unsigned long long kIndexEmptyKey = ~0ull;
 __host__ __device__ inline unsigned long long index_pair_key(uint32_t t0, uint32_t t1) {

@@ -95,6 +95,7 @@ __global__ void validate_kernel(const int32_t* __restrict__ T, const SaT* __rest
 constexpr uint32_t kIndexMaxVocab = 1u << 22;       // the first-token table has vocab + 1 entries
 constexpr uint64_t kIndexMinEntries = 1ull << 12, kIndexMaxEntries = 1ull << 23;
 
+constexpr size_t kIndexHeaderBytes = 256;           // word 0: "the datastore has an entry or token out of range"
 struct IndexLayout {
   uint64_t entries;      // hash-table entries (a power of two; 0 = no index for this datastore)
   int64_t min_run;       // token pairs with fewer occurrences are not stored
@@ -112,7 +113,7 @@ IndexLayout index_layout(uint64_t n, uint32_t vocab) {
   if (l.min_run < 1) l.min_run = 1;
   l.first_bytes = (((size_t)vocab + 1) * 8 + 255) / 256 * 256;
   l.table_bytes = (size_t)e * 32;
-  l.total = l.first_bytes + l.table_bytes;
+  l.total = kIndexHeaderBytes + l.first_bytes + l.table_bytes;
   return l;
 }
 size_t validation_bytes(uint64_t n) {
@@ -138,11 +139,14 @@ __device__ __forceinline__ bool pair_at(const int32_t* __restrict__ T, const SaT
 template <typename SaT>
 __global__ void index_build_kernel(const int32_t* __restrict__ T, const SaT* __restrict__ sa, int64_t n,
                                    uint32_t vocab, int64_t min_run, long long* __restrict__ first,
-                                   unsigned long long* __restrict__ table, uint32_t group_mask) {
+                                   unsigned long long* __restrict__ table, uint32_t group_mask,
+                                   uint32_t* __restrict__ unusable) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
     int32_t t0, t1, a0 = -2, a1 = -2, b0 = -2, b1 = -2;
-    if (!pair_at(T, sa, n, vocab, i, t0, t1)) continue;
+    // a datastore with an entry or a token out of range gets no index: searches then run over
+    // the whole array, where such an entry is reported when it is met
+    if (!pair_at(T, sa, n, vocab, i, t0, t1)) { *unusable = 1u; continue; }
     if (i > 0 && !pair_at(T, sa, n, vocab, i - 1, a0, a1)) a0 = -2;
     if (i + 1 < n && !pair_at(T, sa, n, vocab, i + 1, b0, b1)) b0 = -2;
     if (i == 0 || a0 != t0) first[t0] = i;
@@ -246,27 +250,29 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
     REST_CUDA_TRY(cudaStreamSynchronize(st));
     if (h_flags != 0) return REST_BAD_DATASTORE;
   }
-  rest::BucketIndex idx = {nullptr, nullptr, 0};
+  rest::BucketIndex idx = {nullptr, nullptr, 0, nullptr};
   if (il.entries > 0) {
     // built after a successful validation (when asked for), on the same stream, without a sync:
     // calls that use the handle on this stream see the finished index
     unsigned char* base = static_cast<unsigned char*>(d_aux);
-    long long* first = reinterpret_cast<long long*>(base);
-    unsigned long long* table = reinterpret_cast<unsigned long long*>(base + il.first_bytes);
+    uint32_t* unusable = reinterpret_cast<uint32_t*>(base);
+    long long* first = reinterpret_cast<long long*>(base + kIndexHeaderBytes);
+    unsigned long long* table = reinterpret_cast<unsigned long long*>(base + kIndexHeaderBytes + il.first_bytes);
     REST_CUDA_TRY(cudaMemsetAsync(base, 0xFF, il.total, st));      // first[] = -1, keys = empty, lo = hi = -1
+    REST_CUDA_TRY(cudaMemsetAsync(base, 0, kIndexHeaderBytes, st));
     const uint32_t group_mask = (uint32_t)(il.entries / 4 - 1);
     const uint64_t wave = (uint64_t)(rest::sm_count() > 0 ? rest::sm_count() : 148) * 16;
     const int blocks = (int)((n_tokens + 255) / 256 < wave ? (n_tokens + 255) / 256 : wave);
     if (sa_bytes == 4)
       index_build_kernel<int32_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int32_t*>(d_sa),
-                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask);
+                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask, unusable);
     else
       index_build_kernel<int64_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int64_t*>(d_sa),
-                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask);
+                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask, unusable);
     index_fill_kernel<<<1, 1024, 0, st>>>(first, vocab, (int64_t)n_tokens);
     rest::count_launch(2);
     REST_CUDA_TRY(cudaGetLastError());
-    idx.first = first; idx.table = table; idx.group_mask = group_mask;
+    idx.first = first; idx.table = table; idx.group_mask = group_mask; idx.unusable = unusable;
   }
   rest_datastore* ds = static_cast<rest_datastore*>(malloc(sizeof(rest_datastore)));
   if (!ds) return REST_INVALID_ARG;

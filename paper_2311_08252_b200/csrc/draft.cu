@@ -35,9 +35,12 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxM = REST_MAX_M;
 constexpr int kMaxN = REST_MAX_N;
-constexpr int kHistHi = 1056;   // bins of key >> 10, key < 2^20 + 32
+constexpr int kHistHi = 2080;   // first-level bins: weights below 1024 one by one, then 1024 + weight / 32
 constexpr int kHistLo = 1024;
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kMaxTrunc = 32;                         // rows cut short by the end of the stream (at most m exist)
+constexpr int kMaxLoads = (33 * kMaxM + 31) / 32;     // load instructions for a warp's 33 rows
+constexpr int kPositionCacheRows = 1024;              // rows whose suffix position stays in shared memory for phase 4
 // Batched path (calls with far more contexts than the GPU holds at once): threads per block,
 // lanes per probe round once the probes leave L2, the number of 32-wide rounds before that,
 // and whether the suffix lengths are searched in two steps.  Measured at 4096 contexts on a
@@ -57,7 +60,7 @@ constexpr int kLightRows = 256;
 // which doubles the threads an SM gives to such a context (K = 20000, m = 16: 880 -> 415 us at
 // 1024 contexts, 1670 -> 1181 us at 4096; at K = 5000 the same change loses 4-13 % in large calls).
 constexpr int kBigThreads = 1024;
-constexpr size_t kBigSmemBytes = 56 * 1024;
+constexpr size_t kBigRowsTimesM = 160000;   // K * m from which a context gets a 1024-thread block
 
 struct DraftArgs {
   const int32_t* T;
@@ -76,6 +79,7 @@ struct DraftArgs {
   rest::BucketIndex idx;
   int nwords;   // bitmap words per depth
   int kcap;     // rows the block's shared memory holds, a multiple of 32
+  int pcache_rows;   // rows whose suffix position is kept in shared memory
   // three-launch form of the batched path: the search launch sorts the contexts that matched
   // into two lists by candidate count, the two build launches take one list each
   int32_t* list;          // [2][B] context indices
@@ -229,24 +233,61 @@ __device__ void warp_threshold_desc(const uint32_t* hist, int nbins, uint32_t ne
 struct Smem {
   int q[16];
   long long lb[17], ub[17];
-  uint32_t e1[kMaxM + 1];      // nodes of weight 1 per depth
-  int e1diff[kMaxM + 2];       // the same as a difference array over depths, before the prefix sum
-  uint32_t heavy_total;        // nodes of weight >= 2
+  long long bhi[17];           // end of the range the lower bound of each length was searched in
+  uint32_t small[5][kMaxM + 1];   // [c][d]: nodes of weight c = 1 ... 4 at depth d
+  uint32_t big_total;          // nodes of weight >= 5
   int err;
   int bin_hi;
   uint32_t above_hi;
   int bin_lo;
   uint32_t above_lo;
   uint32_t nsel;
-  uint32_t warp_cnt[32];
+  int ntrunc;
+  int warp_first[32];          // block-wide searches: first probe of each warp that compared greater
+  uint32_t trunc[kMaxTrunc];   // len << 16 | row: rows cut short by the end of the token stream
   uint32_t sel[kMaxN];         // depth << 16 | row
   uint32_t selcnt[kMaxN];
   uint32_t sorted[kMaxN];
   uint32_t sortedcnt[kMaxN];
   int par[kMaxN];
-  uint32_t hist_hi[kHistHi];
-  uint32_t hist_lo[kHistLo];
+  uint32_t hist_hi[kHistHi];   // nodes of weight >= 5 by weight: exact below 1024, in steps of 32 above
+  uint32_t hist_lo[kHistLo];   // inside the threshold bin: by depth (and the weight's low bits)
 };
+
+// Suffix-array range of the suffixes that start with the token pair (t0, t1), from the bucket
+// index.  Warp-cooperative: four lanes read the four entries of the pair's group (one 128-byte
+// line).  false when the pair is not stored.
+__device__ __forceinline__ bool index_pair_range(const rest::BucketIndex& idx, uint32_t t0, uint32_t t1,
+                                                 int lane, int64_t n_tokens, int64_t& lo, int64_t& hi) {
+  const unsigned long long key = rest::index_pair_key(t0, t1);
+  const unsigned long long* grp = idx.table + (size_t)rest::index_group_of(key, idx.group_mask) * 16;
+  unsigned long long k = rest::kIndexEmptyKey;
+  long long l = -1, h = -1;
+  if (lane < 4) {
+    k = __ldg(grp + lane * 4);
+    l = (long long)__ldg(grp + lane * 4 + 1);
+    h = (long long)__ldg(grp + lane * 4 + 2);
+  }
+  const unsigned hit = __ballot_sync(kFull, lane < 4 && k == key && l >= 0 && h > l && h <= n_tokens);
+  if (hit == 0) return false;
+  const int src = __ffs(hit) - 1;
+  lo = __shfl_sync(kFull, l, src);
+  hi = __shfl_sync(kFull, h, src);
+  return true;
+}
+
+// Rows in bitmap word w whose continuation is shorter than d tokens (they end a run like any
+// row that starts a node, but are no node at depth d themselves).  The list is almost always
+// empty: only matches within m tokens of the end of the stream are cut short.
+__device__ __forceinline__ uint32_t cut_short_mask(const Smem& s, int ntrunc, int d, int w) {
+  uint32_t t = 0;
+  for (int k = 0; k < ntrunc; ++k) {
+    const uint32_t e = s.trunc[k];
+    const int j = (int)(e & 0xFFFFu), len = (int)(e >> 16);
+    if ((j >> 5) == w && len < d) t |= 1u << (j & 31);
+  }
+  return t;
+}
 
 // TP = false: the single-context path, tuned for the fewest dependent reads.  TP = true: the
 // batched path, for calls with more contexts than the GPU holds at once; the same results by
@@ -259,12 +300,18 @@ template <typename SaT, bool TP, int NT, int PART>
 __global__ void __launch_bounds__(NT, 1024 / NT)
 rest_draft_kernel(DraftArgs a) {
   constexpr int NW = NT / 32;
-  static_assert(NT % 32 == 0 && NT >= 64, "whole warps; at least kMaxM + 2 threads");
+  static_assert(NT % 32 == 0 && NT >= 128, "whole warps; enough threads for the set-up loops");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& s = *reinterpret_cast<Smem*>(smem_raw);
-  uint16_t* lenlcp = reinterpret_cast<uint16_t*>(smem_raw + sizeof(Smem));          // [kcap]
-  uint32_t* bm = reinterpret_cast<uint32_t*>(smem_raw + sizeof(Smem) + 2 * a.kcap); // [m][nwords]
-  uint16_t* jump = reinterpret_cast<uint16_t*>(bm + a.m * a.nwords);                // [m][nwords]
+  // per warp: start position, length and comparable length of its 33 slots (the row before the
+  // warp's first one, then its 32 rows); the suffix positions of the first rows (phase 4 reads
+  // the kept nodes' tokens through them); then the block's bitmaps
+  long long* slot_base = reinterpret_cast<long long*>(smem_raw + sizeof(Smem));            // [NW][34]
+  long long* pcache = slot_base + NW * 34;                                                  // [pcache_rows]
+  int* slot_len = reinterpret_cast<int*>(pcache + a.pcache_rows);                           // [NW][66]
+  uint32_t* bm = reinterpret_cast<uint32_t*>(slot_len + NW * 66);                           // [m][nwords]
+  uint16_t* jump = reinterpret_cast<uint16_t*>(bm + a.m * a.nwords);                        // [m][nwords]
+  uint16_t* tiecnt = jump + a.m * a.nwords;                                                 // [nwords]
 
   if constexpr (PART == kBuild) {
     if ((int)blockIdx.x >= a.list_count[a.which]) return;
@@ -280,21 +327,29 @@ rest_draft_kernel(DraftArgs a) {
   const int64_t n_tokens = a.n_tokens;
   const int clen = a.ctx_len[b];
   const int32_t* ctx = a.ctx + (int64_t)b * a.ctx_stride;
+  // read early, beside the context: whether the bucket index may be used (not when its build
+  // met a suffix-array entry or a token out of range)
+  const uint32_t index_unusable = (PART != kBuild && a.idx.first != nullptr) ? __ldg(a.idx.unusable) : 1u;
 
   // Unused-slot defaults; thread i owns slots i, i + NT, ... for the whole kernel (a build
   // launch finds them written by the search launch).
-  if constexpr (PART != kBuild)
-  for (int i = tid; i < N; i += NT) {
-    int64_t o = (int64_t)b * N + i;
-    a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
-    for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (i >> 5)) ? (1u << (i & 31)) : 0u;
-    if (a.node_count) a.node_count[o] = 0;
-  }
+  auto write_defaults = [&]() {
+    for (int i = tid; i < N; i += NT) {
+      int64_t o = (int64_t)b * N + i;
+      a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
+      for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (i >> 5)) ? (1u << (i & 31)) : 0u;
+      if (a.node_count) a.node_count[o] = 0;
+    }
+  };
+  auto report_empty = [&]() {                      // by thread 0, after a barrier
+    a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
+    a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
+  };
+  if constexpr (PART != kBuild) write_defaults();
   const int nq = min(a.n_max, max(clen, 0));   // context tokens that can take part
-  if (tid == 0) { s.err = 0; s.heavy_total = 0; s.nsel = 0; }
-  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; }
-  if (tid <= kMaxM) s.e1[tid] = 0;
-  if (tid <= kMaxM + 1) s.e1diff[tid] = 0;
+  if (tid == 0) { s.err = 0; s.big_total = 0; s.nsel = 0; s.ntrunc = 0; }
+  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; s.bhi[tid] = n_tokens; }
+  if (tid < 5 * (kMaxM + 1)) (&s.small[0][0])[tid] = 0;
   if constexpr (PART != kSearch) {
     for (int i = tid; i < kHistHi; i += NT) s.hist_hi[i] = 0;
     for (int i = tid; i < kHistLo; i += NT) s.hist_lo[i] = 0;
@@ -313,10 +368,7 @@ rest_draft_kernel(DraftArgs a) {
   }
   __syncthreads();
   if (s.err != 0 || nq < a.n_min) {
-    if (tid == 0) {
-      a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
-      a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
-    }
+    if (tid == 0) report_empty();
     return;
   }
 
@@ -324,15 +376,41 @@ rest_draft_kernel(DraftArgs a) {
   // 1a: lower bound of every suffix length, one warp each.  ub = -1 marks "matches, end of the
   // run not known yet".
   constexpr int kArity = TP ? kTpArity : 32;
+  const bool have_index = index_unusable == 0u;
   auto lower_bound_of = [&](int n) {     // executed by one whole warp
     int q[16];
 #pragma unroll
     for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
     bool bad = false, eq = false;
-    int64_t next_gt = -1;
-    int64_t lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
+    int64_t next_gt = -1, lb;
+    if (have_index) {
+      // every suffix that starts with the query's first token lies in [f0, f1); when the index
+      // also stores the query's first token pair, every suffix that starts with that pair lies
+      // in [lo0, hi0).  Slot hi0 (or the end of the array) compares greater than the query.
+      int64_t lo0 = __ldg(a.idx.first + q[0]), hi0 = __ldg(a.idx.first + q[0] + 1);
+      lo0 = lo0 < 0 ? 0 : (lo0 > n_tokens ? n_tokens : lo0);
+      hi0 = hi0 < lo0 ? lo0 : (hi0 > n_tokens ? n_tokens : hi0);
+      if (n == 1) {                       // the first-token range is the answer
+        if (lane == 0) { s.lb[1] = lo0; s.ub[1] = hi0; s.bhi[1] = hi0; }
+        return;
+      }
+      int64_t plo, phi;
+      if (index_pair_range(a.idx, (uint32_t)q[0], (uint32_t)q[1], lane, n_tokens, plo, phi) &&
+          plo >= lo0 && phi <= hi0) {
+        if (n == 2) {                     // the pair's range is the answer
+          if (lane == 0) { s.lb[2] = plo; s.ub[2] = phi; s.bhi[2] = phi; }
+          return;
+        }
+        lo0 = plo; hi0 = phi;
+      }
+      if (lane == 0) s.bhi[n] = hi0;
+      lb = warp_first_true<SaT, false, kArity, 0>(T, sa, n_tokens, lo0, hi0, q, n, lane, eq, bad, &next_gt);
+      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < hi0) ? next_gt : lb; }
+    } else {
+      lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
+      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_tokens) ? next_gt : lb; }
+    }
     if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
-    if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_tokens) ? next_gt : lb; }
   };
   if constexpr (!TP || !kTpStaged) {
     for (int n = a.n_min + warp; n <= nq; n += NW) lower_bound_of(n);   // one length per warp when NW = 16
@@ -362,50 +440,62 @@ rest_draft_kernel(DraftArgs a) {
   for (int n = nq; n >= a.n_min; --n)
     if (s.ub[n] != s.lb[n]) { n_win = n; break; }
   // 1b: only the winning length needs its upper bound, and only if the last round of its lower
-  // bound did not already show where the run ends (shorter lengths match far more slots and
-  // would need the most rounds: they are never looked at again)
+  // bound did not already show where the run ends.  The whole block searches: in the first
+  // round the first half of the threads probes the slots right behind the first match one by
+  // one and the second half probes at geometrically growing distances (so a short run is
+  // settled in one round whatever the size of the range); the rounds after that cut what is
+  // left into NT + 1 parts.
   if (n_win != 0 && s.ub[n_win] < 0) {       // block-uniform
-    if (warp == (n_win - a.n_min) % NW) {
-      const int n = n_win;
-      int q[16];
+    const int n = n_win;
+    int q[16];
 #pragma unroll
-      for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
-      bool bad = false;
-      const int64_t lb = s.lb[n];
-      // gallop: slot lb + 2^e for e = 0 ... 31, all at once or kArity exponents per round; f =
-      // the first exponent whose slot compares greater or lies past the end (-1: none)
-      int f = -1;
-      for (int g = 0; g < 32 / kArity; ++g) {
-        bool t = false;
-        if (lane < kArity) {
-          const int64_t pos = lb + ((int64_t)1 << (g * kArity + lane));
-          t = true;
-          if (pos < n_tokens) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
-        }
-        const unsigned bal = __ballot_sync(kFull, t);
-        if (bal != 0) { f = g * kArity + __ffs(bal) - 1; break; }
-      }
-      int64_t lo2, hi2 = n_tokens;
-      bool eq2 = false;
-      if (f < 0) {
-        lo2 = lb + ((int64_t)1 << 31) + 1;
+    for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
+    bool bad = false;
+    const int64_t end = s.bhi[n];            // slots from here on are known to compare greater
+    int64_t lo2 = s.lb[n] + 1, hi2 = end;    // the answer lies in [lo2, hi2]
+    constexpr int H = NT / 2, S = (H / 34) > 0 ? (H / 34) : 1;     // linear probes; geometric steps per octave
+    auto first_round_pos = [&](int t) -> int64_t {
+      if (t < H) return lo2 + t;
+      const int e = t - H + 1, oct = e / S, frac = e - oct * S;
+      if (oct > 44) return (int64_t)1 << 60;
+      const int64_t base = (int64_t)H << oct;
+      return lo2 + base + base * frac / S - 1;
+    };
+    bool first = true;
+    while (hi2 > lo2) {                      // block-uniform
+      const int64_t size = hi2 - lo2;
+      const bool exact = !first && size <= NT;            // one probe per remaining slot
+      auto pos_of = [&](int t) -> int64_t {
+        if (first) return first_round_pos(t);
+        if (exact) return lo2 + t;
+        return lo2 + (int64_t)(((unsigned long long)(t + 1) * (unsigned long long)size) / (unsigned long long)(NT + 1));
+      };
+      const int64_t pos = pos_of(tid);
+      bool t = true;                                      // slots from hi2 on compare greater
+      if (pos < hi2) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
+      const unsigned bal = __ballot_sync(kFull, t);
+      if (lane == 0) s.warp_first[warp] = bal ? warp * 32 + __ffs(bal) - 1 : 0x7FFFFFFF;
+      __syncthreads();
+      int tf = 0x7FFFFFFF;
+      for (int w = 0; w < NW; ++w) tf = min(tf, s.warp_first[w]);
+      __syncthreads();
+      if (tf == 0x7FFFFFFF) {
+        lo2 = pos_of(NT - 1) + 1;
+        if (lo2 > hi2) lo2 = hi2;
       } else {
-        int64_t pf = lb + ((int64_t)1 << f);
-        hi2 = pf < n_tokens ? pf : n_tokens;
-        lo2 = f > 0 ? lb + ((int64_t)1 << (f - 1)) + 1 : lb + 1;
+        const int64_t pf = pos_of(tf);
+        const int64_t nlo = tf > 0 ? pos_of(tf - 1) + 1 : lo2;
+        hi2 = pf < hi2 ? pf : hi2;
+        lo2 = nlo < hi2 ? nlo : hi2;
       }
-      if (lo2 > hi2) lo2 = hi2;
-      const int64_t ub = warp_first_true<SaT, true, kArity, 0>(T, sa, n_tokens, lo2, hi2, q, n, lane, eq2, bad);
-      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
-      if (lane == 0) s.ub[n] = ub;
+      first = false;
     }
+    if (bad) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+    if (tid == 0) s.ub[n] = hi2;
     __syncthreads();
   }
   if (s.err != 0 || n_win == 0) {
-    if (tid == 0) {
-      a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
-      a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
-    }
+    if (tid == 0) report_empty();
     return;
   }
   }  // PART != kBuild
@@ -425,91 +515,127 @@ rest_draft_kernel(DraftArgs a) {
   const int Kp = (int)(cnt < (int64_t)a.K ? cnt : (int64_t)a.K);
   const int nwords = a.nwords;
   const int niter = (Kp + NT - 1) / NT;
+  const int nw = (Kp + 31) >> 5;            // bitmap words that hold rows
 
   // ---- phase 2: gather rows, common-prefix lengths, node-start bitmaps --------------------
-  // the suffix-array entry of the next iteration's row is fetched one iteration ahead, so
-  // that the two dependent reads (entry, then tokens) of consecutive iterations overlap
-  // (lane 0 also needs the row before its own, which another warp holds: it fetches that
-  // entry ahead as well and reads both rows' tokens side by side)
-  int64_t p_next = 0, pp_next = 0;
-  if (tid < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid));
-  if (lane == 0 && tid > 0 && tid <= Kp)
-    pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid - 1));
-  for (int it = 0; it < niter; ++it) {
-    const int jbase = it * NT + warp * 32;
-    const int j = jbase + lane;
-    int64_t p = p_next;
-    const int64_t pp = pp_next;
-    if (j + NT < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT));
-    if (lane == 0 && j + NT <= Kp)
-      pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT - 1));
-    if (jbase >= Kp) continue;   // warp-uniform
-    const bool valid = j < Kp;
-    int row[kMaxM], prev[kMaxM];
-    int len = 0, plen = 0;
-    bool bad = false;
-    if (valid) {
-      if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
-      int64_t base = p + n_win;
-      int64_t rem = n_tokens - base;
-      len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
-#pragma unroll
-      for (int d = 0; d < kMaxM; ++d) row[d] = (d < len) ? __ldg(T + base + d) : 0;
-    } else {
-#pragma unroll
-      for (int d = 0; d < kMaxM; ++d) row[d] = 0;
-    }
-#pragma unroll
-    for (int d = 0; d < kMaxM; ++d) prev[d] = __shfl_up_sync(kFull, row[d], 1);
-    plen = __shfl_up_sync(kFull, len, 1);
-    if (lane == 0 && j > 0) {   // previous row belongs to another warp: fetch it again
-      int64_t p = pp;
-      if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
-      int64_t base = p + n_win;
-      int64_t rem = n_tokens - base;
-      plen = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
-#pragma unroll
-      for (int d = 0; d < kMaxM; ++d) prev[d] = (d < plen) ? __ldg(T + base + d) : 0;
-    }
-    int lcp = 0;
-    if (valid && j > 0) {
+  // Slot 0 of a warp is the row before its first row, slot l + 1 the row of lane l.  The 33
+  // rows are read as one run of 33 m words, word f by lane f mod 32 in load f / 32: consecutive
+  // lanes read consecutive tokens of a row, so a load instruction touches three or four rows
+  // (a few cache lines) instead of 32.  Word f is compared with word f - m (the same column of
+  // the row before: lane - m of the same load, or of the load before) right where it sits; a
+  // ballot turns the "equal" and "smaller" outcomes of each load into bit strings, and lane l
+  // cuts the m bits of its row out of them: the number of leading equal columns is the common
+  // prefix.  The suffix-array entries of the next iteration are fetched one iteration ahead.
+  {
+    long long* sb = slot_base + warp * 34;
+    int* sl = slot_len + warp * 66;          // lengths, then comparable lengths min(len, len of the row before)
+    int* slim = sl + 33;
+    const uint32_t magic = (65536u + (uint32_t)m - 1u) / (uint32_t)m;    // f / m = (f * magic) >> 16 for f < 600
+    const int nload = (33 * m + 31) >> 5;
+    const int src_lane = (lane - m) & 31;
+    int64_t p_next = 0, pp_next = 0;
+    if (tid < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid));
+    if (lane == 0 && tid > 0 && tid <= Kp)
+      pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid - 1));
+    for (int it = 0; it < niter; ++it) {
+      const int jbase = it * NT + warp * 32;
+      const int j = jbase + lane;
+      int64_t p = p_next;
+      int64_t pp = pp_next;
+      if (j + NT < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT));
+      if (lane == 0 && j + NT <= Kp)
+        pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT - 1));
+      if (jbase >= Kp) continue;   // warp-uniform
+      const bool valid = j < Kp;
+      bool bad = false;
+      int len = 0;
+      int64_t base = 0;
+      if (valid) {
+        if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
+        if (j < a.pcache_rows) pcache[j] = p;
+        base = p + n_win;
+        const int64_t rem = n_tokens - base;
+        len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+      }
+      int plen = __shfl_up_sync(kFull, len, 1);
+      if (lane == 0) {
+        plen = 0;
+        int64_t pbase = 0;
+        if (j > 0) {                 // the row before this warp's rows belongs to another warp
+          if (pp < 0 || pp >= n_tokens) { bad = true; pp = 0; }
+          pbase = pp + n_win;
+          const int64_t rem = n_tokens - pbase;
+          plen = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+        }
+        sb[0] = pbase; sl[0] = plen; slim[0] = 0;
+      }
       const int lim = min(len, plen);
-      bool run = true;
-      bool ordered = plen <= len;   // decides when one row is a prefix of the other
+      sb[lane + 1] = base; sl[lane + 1] = len; slim[lane + 1] = lim;
+      __syncwarp();
+      uint32_t vals[kMaxLoads];
 #pragma unroll
-      for (int d = 0; d < kMaxM; ++d) {
-        if (run && d < lim) {
-          if (row[d] == prev[d]) {
-            lcp = d + 1;
-          } else {
-            run = false;
-            ordered = (uint32_t)prev[d] < (uint32_t)row[d];
-          }
+      for (int i = 0; i < kMaxLoads; ++i) {
+        vals[i] = 0;
+        if (i < nload) {
+          const uint32_t f = (uint32_t)(i * 32 + lane);
+          const uint32_t r = (f * magic) >> 16, c = f - r * (uint32_t)m;
+          if (r < 33u && (int)c < sl[r]) vals[i] = (uint32_t)__ldg(T + sb[r] + c);
         }
       }
-      if (!ordered) bad = true;
-    }
-    if (valid) lenlcp[j] = (uint16_t)(lcp | (len << 8));
-    uint32_t myword = 0;
+      uint32_t my_eq = 0, my_lt = 0;         // lane i keeps the bit strings of load i
 #pragma unroll
-    for (int d = 1; d <= kMaxM; ++d) {
-      if (d <= m) {
-        uint32_t w = __ballot_sync(kFull, !valid || lcp < d);
-        if (lane == d - 1) myword = w;
+      for (int i = 0; i < kMaxLoads; ++i) {
+        if (i < nload) {                     // warp-uniform
+          const uint32_t f = (uint32_t)(i * 32 + lane);
+          const uint32_t r = (f * magic) >> 16, c = f - r * (uint32_t)m;
+          const uint32_t x = __shfl_sync(kFull, vals[i], src_lane);
+          const uint32_t y = i > 0 ? __shfl_sync(kFull, vals[i > 0 ? i - 1 : 0], src_lane) : 0u;
+          const uint32_t before = lane >= m ? x : y;
+          const bool comparable = r >= 1u && r < 33u && (int)c < slim[r];
+          const uint32_t eq = __ballot_sync(kFull, comparable && vals[i] == before);
+          const uint32_t lt = __ballot_sync(kFull, comparable && before < vals[i]);
+          if (lane == i) { my_eq = eq; my_lt = lt; }
+        }
       }
+      // this lane's row is slot lane + 1: its m outcome bits start at bit (lane + 1) m
+      const int bitpos = (lane + 1) * m, wi = bitpos >> 5, sh = bitpos & 31;
+      const uint32_t e0 = __shfl_sync(kFull, my_eq, wi), e1 = __shfl_sync(kFull, my_eq, (wi + 1) & 31);
+      const uint32_t l0 = __shfl_sync(kFull, my_lt, wi), l1 = __shfl_sync(kFull, my_lt, (wi + 1) & 31);
+      const uint32_t eqf = (uint32_t)((((unsigned long long)e1 << 32) | e0) >> sh);
+      const uint32_t ltf = (uint32_t)((((unsigned long long)l1 << 32) | l0) >> sh);
+      int lcp = __ffs((int)(~eqf | (1u << m))) - 1;      // leading equal columns, at most m
+      if (!valid || j == 0) lcp = 0;
+      if (valid && j > 0) {
+        // the first differing column decides the order; when one row is a prefix of the
+        // other the shorter one must come first
+        const bool ordered = lcp < lim ? ((ltf >> lcp) & 1u) != 0u : plen <= len;
+        if (!ordered) bad = true;
+      }
+      if (valid && len < m) {        // cut short by the end of the stream: at most m such rows exist
+        const int at = atomicAdd(&s.ntrunc, 1);
+        if (at < kMaxTrunc) s.trunc[at] = ((uint32_t)len << 16) | (uint32_t)j;
+        else atomicOr(&s.err, REST_CTX_INTERNAL);
+      }
+      uint32_t myword = 0;
+#pragma unroll
+      for (int d = 1; d <= kMaxM; ++d) {
+        if (d <= m) {
+          uint32_t w = __ballot_sync(kFull, !valid || lcp < d);
+          if (lane == d - 1) myword = w;
+        }
+      }
+      if (lane < m) bm[lane * nwords + (jbase >> 5)] = myword;
+      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+      __syncwarp();                  // the slot tables are rewritten by the next iteration
     }
-    if (lane < m) bm[lane * nwords + (jbase >> 5)] = myword;
-    if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
   }
   if (tid < m) bm[tid * nwords + ((Kp + 31) >> 5)] = kFull;   // sentinel past the last row
   __syncthreads();
   if (s.err != 0) {
-    if (tid == 0) {
-      a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
-      a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
-    }
+    if (tid == 0) report_empty();
     return;
   }
+  const int ntrunc = min(s.ntrunc, kMaxTrunc);
 
   // jump table: for every depth (a warp each) a suffix scan over the bitmap words, last chunk
   // of 32 words first: jump[w] = position of the first set bit in any word after w
@@ -535,124 +661,176 @@ rest_draft_kernel(DraftArgs a) {
   }
   __syncthreads();
 
-  // ---- phase 3a: histogram of (weight, depth) over all Trie nodes --------------------------
-  // key = weight << 5 | (16 - depth): larger key = better node.
-  for (int it = 0; it < niter; ++it) {
-    const int jbase = it * NT + warp * 32;
-    if (jbase >= Kp) continue;
-    const int j = jbase + lane;
-    const bool valid = j < Kp;
-    const int ll = valid ? lenlcp[j] : 0;
-    const int lcp = ll & 0xFF, len = ll >> 8;
-    // Weights along a row never grow with depth: walk down from the first depth at which the
-    // row starts a node until the weight drops to 1; every deeper node of the row weighs 1.
-    uint32_t nheavy = 0;
-    int d1 = len + 1;                      // first depth of weight 1 (len + 1: none)
-    if (valid) {
-      for (int d = lcp + 1; d <= len; ++d) {
-        const int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
-        if (c < 2) { d1 = d; break; }
-        atomicAdd(&s.hist_hi[((c << 5) | (16 - d)) >> 10], 1u);
-        ++nheavy;
+  // The passes of phase 3 run over the pairs (depth d, bitmap word w).  In word w of depth d a
+  // set bit marks a row that starts a node (unless the row is shorter than d) and the node's
+  // weight is the distance to the next set bit.  Weights 1 to 4 are read off the bit pattern
+  // (set bit, then 0 to 3 clear bits, then a set bit) for the whole word at once and counted
+  // with one popcount each; only nodes of weight >= 5 are visited one by one.
+  struct WordNodes { uint32_t c[5]; uint32_t big; };     // c[1..4]: node starts of that weight
+  const int items = m * nw;
+  auto word_nodes = [&](int d, int w) -> WordNodes {
+    const uint32_t* row = bm + (d - 1) * nwords;
+    const uint32_t S = row[w], nx = row[w + 1];
+    uint32_t nodes = S;
+    if (w == nw - 1 && (Kp & 31)) nodes &= (1u << (Kp & 31)) - 1u;     // bits past the last row
+    if (ntrunc) nodes &= ~cut_short_mask(s, ntrunc, d, w);
+    const unsigned long long W = (unsigned long long)S | ((unsigned long long)nx << 32);
+    const uint32_t a1 = (uint32_t)(W >> 1), a2 = (uint32_t)(W >> 2), a3 = (uint32_t)(W >> 3), a4 = (uint32_t)(W >> 4);
+    WordNodes r;
+    r.c[0] = 0;
+    r.c[1] = nodes & a1;
+    uint32_t rest_ = nodes & ~a1;
+    r.c[2] = rest_ & a2; rest_ &= ~a2;
+    r.c[3] = rest_ & a3; rest_ &= ~a3;
+    r.c[4] = rest_ & a4;
+    r.big = rest_ & ~a4;
+    return r;
+  };
+  // key of a node = weight << 5 | (16 - depth): larger key = better node.  First-level bin of a
+  // node of weight >= 5: the weight itself below 1024, 1024 + weight / 32 above.
+  auto key_of = [](int c, int d) -> uint32_t { return ((uint32_t)c << 5) | (uint32_t)(16 - d); };
+  auto bin_of = [](int c) -> int { return c < 1024 ? c : 1024 + (c >> 5); };
+  auto sub_of = [](int c, int d) -> int { return c < 1024 ? 16 - d : ((c & 31) << 5) | (16 - d); };
+
+  // ---- phase 3a: counts of the light nodes, histogram of the others ------------------------
+  {
+    uint32_t nbig = 0;
+    for (int item = tid; item < items; item += NT) {
+      const int d = item / nw + 1, w = item - (d - 1) * nw;
+      const WordNodes wn = word_nodes(d, w);
+#pragma unroll
+      for (int c = 1; c <= 4; ++c)
+        if (wn.c[c]) atomicAdd(&s.small[c][d], (uint32_t)__popc(wn.c[c]));
+      const uint32_t* row = bm + (d - 1) * nwords;
+      const uint16_t* jrow = jump + (d - 1) * nwords;
+      uint32_t big = wn.big;
+      while (big) {
+        const int j = (w << 5) + __ffs(big) - 1;
+        big &= big - 1;
+        atomicAdd(&s.hist_hi[bin_of(next_set(row, jrow, j) - j)], 1u);
+        ++nbig;
       }
     }
-    // weight-1 nodes per depth: d1 <= d <= len, counted as starts minus ends per warp
-    for (int d = 1; d <= m + 1; ++d) {
-      const uint32_t st = __ballot_sync(kFull, valid && d1 == d && d1 <= len);
-      const uint32_t en = __ballot_sync(kFull, valid && d1 <= len && len + 1 == d);
-      if (lane == 0 && (st | en)) atomicAdd(&s.e1diff[d], __popc(st) - __popc(en));
-    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) nheavy += __shfl_xor_sync(kFull, nheavy, o);
-    if (lane == 0 && nheavy) atomicAdd(&s.heavy_total, nheavy);
-  }
-  __syncthreads();
-
-  if (tid == 0) {
-    int run = 0;
-    for (int d = 1; d <= m; ++d) { run += s.e1diff[d]; s.e1[d] = (uint32_t)run; }
+    for (int o = 16; o > 0; o >>= 1) nbig += __shfl_xor_sync(kFull, nbig, o);
+    if (lane == 0 && nbig) atomicAdd(&s.big_total, nbig);
   }
   __syncthreads();
 
   // ---- phase 3b: threshold key t*, number of ties wanted ------------------------------------
-  uint32_t tstar;      // nodes with key > tstar are kept
-  uint32_t r_tie;      // plus the first r_tie nodes (by row) with key == tstar
-  const uint32_t heavy_total = s.heavy_total;
-  if (heavy_total >= (uint32_t)N) {
+  uint32_t tstar = 0;  // nodes with key > tstar are kept
+  uint32_t r_tie = 0;  // plus the first r_tie nodes (by row) with key == tstar
+  int c_tie = 0, d_tie = 0;
+  const uint32_t big_total = s.big_total;
+  if (big_total >= (uint32_t)N) {
     if (warp == 0) warp_threshold_desc(s.hist_hi, kHistHi, (uint32_t)N, lane, &s.bin_hi, &s.above_hi);
     __syncthreads();
     const int bin_hi = s.bin_hi;
-    for (int it = 0; it < niter; ++it) {
-      const int jbase = it * NT + warp * 32;
-      if (jbase >= Kp) continue;
-      const int j = jbase + lane;
-      if (j >= Kp) continue;
-      const int ll = lenlcp[j];
-      const int lcp = ll & 0xFF, len = ll >> 8;
-      for (int d = lcp + 1; d <= len; ++d) {
-        int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
-        if (c < 2) break;   // weights do not grow with depth
-        uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
-        if ((int)(key >> 10) == bin_hi) atomicAdd(&s.hist_lo[key & 1023u], 1u);
+    for (int item = tid; item < items; item += NT) {
+      const int d = item / nw + 1, w = item - (d - 1) * nw;
+      uint32_t big = word_nodes(d, w).big;
+      const uint32_t* row = bm + (d - 1) * nwords;
+      const uint16_t* jrow = jump + (d - 1) * nwords;
+      while (big) {
+        const int j = (w << 5) + __ffs(big) - 1;
+        big &= big - 1;
+        const int c = next_set(row, jrow, j) - j;
+        if (bin_of(c) == bin_hi) atomicAdd(&s.hist_lo[sub_of(c, d)], 1u);
       }
     }
     __syncthreads();
     if (warp == 0)
       warp_threshold_desc(s.hist_lo, kHistLo, (uint32_t)N - s.above_hi, lane, &s.bin_lo, &s.above_lo);
     __syncthreads();
-    tstar = ((uint32_t)bin_hi << 10) | (uint32_t)s.bin_lo;
+    const int sub = s.bin_lo;
+    d_tie = 16 - (sub & 31);
+    c_tie = bin_hi < 1024 ? bin_hi : (((bin_hi - 1024) << 5) | (sub >> 5));
+    tstar = key_of(c_tie, d_tie);
     r_tie = (uint32_t)N - s.above_hi - s.above_lo;
   } else {
-    // every node of weight >= 2 is kept; weight-1 nodes fill up by depth, then by row
-    uint32_t need = (uint32_t)N - heavy_total, cum = 0;
-    tstar = 0; r_tie = 0;
-    for (int d = 1; d <= m; ++d) {
-      uint32_t e = s.e1[d];
-      if (cum + e >= need) { tstar = (1u << 5) | (uint32_t)(16 - d); r_tie = need - cum; break; }
-      cum += e;
+    // every node of weight >= 5 is kept; the lighter ones fill up by weight, then depth, then row
+    uint32_t need = (uint32_t)N - big_total, cum = 0;
+    for (int c = 4; c >= 1 && tstar == 0; --c) {
+      for (int d = 1; d <= m; ++d) {
+        const uint32_t e = s.small[c][d];
+        if (cum + e >= need) { c_tie = c; d_tie = d; tstar = key_of(c, d); r_tie = need - cum; break; }
+        cum += e;
+      }
     }
   }
-  const int d_tie = 16 - (int)(tstar & 31u);
-  const int c_tie = (int)(tstar >> 5);
 
   // ---- phase 3c: collect the kept nodes -----------------------------------------------------
-  uint32_t tie_base = 0;
-  for (int it = 0; it < niter; ++it) {
-    const int j = it * NT + tid;
-    const bool valid = j < Kp;
-    bool tie = false;
-    if (valid) {
-      const int ll = lenlcp[j];
-      const int lcp = ll & 0xFF, len = ll >> 8;
-      for (int d = lcp + 1; d <= len; ++d) {
-        int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
-        uint32_t key = ((uint32_t)c << 5) | (uint32_t)(16 - d);
-        if (key > tstar) {
-          uint32_t slot = atomicAdd(&s.nsel, 1u);
-          if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)j; s.selcnt[slot] = c; }
-        } else {
-          tie = key == tstar;
-          break;                           // keys only fall with depth along a row
+  // everything above the threshold now; the ties (same weight, same depth) by row order after a
+  // prefix sum over the words of their depth
+  auto keep = [&](int d, int j, int c) {
+    const uint32_t slot = atomicAdd(&s.nsel, 1u);
+    if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)j; s.selcnt[slot] = (uint32_t)c; }
+  };
+  auto tie_bits = [&](int w) -> uint32_t {         // tie candidates in word w of the tie depth
+    const WordNodes wn = word_nodes(d_tie, w);
+    if (c_tie <= 4) return c_tie == 1 ? wn.c[1] : c_tie == 2 ? wn.c[2] : c_tie == 3 ? wn.c[3] : wn.c[4];
+    const uint32_t* row = bm + (d_tie - 1) * nwords;
+    const uint16_t* jrow = jump + (d_tie - 1) * nwords;
+    uint32_t big = wn.big, t = 0;
+    while (big) {
+      const int bit = __ffs(big) - 1;
+      big &= big - 1;
+      const int j = (w << 5) + bit;
+      if (next_set(row, jrow, j) - j == c_tie) t |= 1u << bit;
+    }
+    return t;
+  };
+  for (int item = tid; item < items; item += NT) {
+    const int d = item / nw + 1, w = item - (d - 1) * nw;
+    const WordNodes wn = word_nodes(d, w);
+#pragma unroll
+    for (int c = 1; c <= 4; ++c) {
+      if (key_of(c, d) > tstar) {
+        uint32_t bits = wn.c[c];
+        while (bits) {
+          keep(d, (w << 5) + __ffs(bits) - 1, c);
+          bits &= bits - 1;
         }
       }
     }
-    if (r_tie > 0) {   // block-uniform
-      uint32_t bal = __ballot_sync(kFull, tie);
-      if (lane == 0) s.warp_cnt[warp] = __popc(bal);
-      __syncthreads();
-      uint32_t before = tie_base, total = 0;
-      for (int w = 0; w < NW; ++w) {
-        uint32_t c = s.warp_cnt[w];
-        if (w < warp) before += c;
-        total += c;
+    const uint32_t* row = bm + (d - 1) * nwords;
+    const uint16_t* jrow = jump + (d - 1) * nwords;
+    uint32_t big = wn.big;
+    while (big) {
+      const int j = (w << 5) + __ffs(big) - 1;
+      big &= big - 1;
+      const int c = next_set(row, jrow, j) - j;
+      if (key_of(c, d) > tstar) keep(d, j, c);
+    }
+  }
+  if (r_tie > 0) {   // block-uniform
+    for (int w = tid; w < nw; w += NT) tiecnt[w] = (uint16_t)__popc(tie_bits(w));
+    __syncthreads();
+    if (warp == 0) {                               // exclusive prefix sum over the words, in place
+      uint32_t carry = 0;
+      for (int c0 = 0; c0 < nw; c0 += 32) {
+        const int w = c0 + lane;
+        const uint32_t v = w < nw ? tiecnt[w] : 0u;
+        uint32_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t u = __shfl_up_sync(kFull, incl, o);
+          if (lane >= o) incl += u;
+        }
+        if (w < nw) tiecnt[w] = (uint16_t)min(carry + incl - v, 0xFFFFu);
+        carry += __shfl_sync(kFull, incl, 31);
       }
-      uint32_t rank = before + __popc(bal & ((1u << lane) - 1u));
-      if (tie && rank < r_tie) {
-        uint32_t slot = atomicAdd(&s.nsel, 1u);
-        if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d_tie << 16) | (uint32_t)j; s.selcnt[slot] = c_tie; }
+    }
+    __syncthreads();
+    for (int w = tid; w < nw; w += NT) {
+      uint32_t rank = tiecnt[w];
+      if (rank >= r_tie) continue;
+      uint32_t t = tie_bits(w);
+      while (t && rank < r_tie) {
+        keep(d_tie, (w << 5) + __ffs(t) - 1, c_tie);
+        t &= t - 1;
+        ++rank;
       }
-      tie_base += total;
-      __syncthreads();
     }
   }
   __syncthreads();
@@ -686,7 +864,8 @@ rest_draft_kernel(DraftArgs a) {
       if (par < 0) { atomicOr(&s.err, REST_CTX_INTERNAL); par = -1; }
     }
     s.par[i] = par;
-    int64_t p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
+    const int64_t p = j < a.pcache_rows ? (int64_t)pcache[j]
+                                        : (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
     int64_t o = (int64_t)b * N + i;
     a.tokens[o] = __ldg(T + p + n_win + d - 1);
     a.parents[o] = par;
@@ -715,29 +894,36 @@ rest_draft_kernel(DraftArgs a) {
   if (s.err != 0) {
     // an inconsistency met while the tree was being written: the caller gets the empty tree
     // that every other reported problem gives, not a half-built one
-    for (int i = tid; i < N; i += NT) {
-      int64_t o = (int64_t)b * N + i;
-      a.tokens[o] = -1; a.parents[o] = -1; a.depth[o] = 0; a.pos_ids[o] = clen;
-      for (int w = 0; w < Wm; ++w) a.mask[o * Wm + w] = (w == (i >> 5)) ? (1u << (i & 31)) : 0u;
-      if (a.node_count) a.node_count[o] = 0;
-    }
+    write_defaults();
+    if (tid == 0) report_empty();
+    return;
   }
   if (tid == 0) {
-    const bool ok = s.err == 0;
-    a.status[b] = s.err;
-    a.n_nodes[b] = ok ? nn : 0;
-    a.match_n[b] = ok ? n_win : 0;
-    a.match_range[2 * b] = ok ? lo : 0;
-    a.match_range[2 * b + 1] = ok ? hi : 0;
+    a.status[b] = 0;
+    a.n_nodes[b] = nn;
+    a.match_n[b] = n_win;
+    a.match_range[2 * b] = lo;
+    a.match_range[2 * b + 1] = hi;
   }
 }
 
-size_t draft_smem_bytes(int K, int m, int* kcap_out, int* nwords_out) {
-  int kcap = (K + 31) / 32 * 32;
-  int nwords = kcap / 32 + 1;
+// Dynamic shared memory of a block of `threads` threads that builds trees from up to K rows of
+// m tokens (the search-only launch needs sizeof(Smem) alone).
+size_t draft_smem_bytes(int K, int m, int threads, int* kcap_out, int* nwords_out, int* pcache_out) {
+  const int kcap = (K + 31) / 32 * 32;
+  const int nwords = kcap / 32 + 1;
+  const int warps = threads / 32;
+  const int pcache_rows = kcap < kPositionCacheRows ? kcap : kPositionCacheRows;
   if (kcap_out) *kcap_out = kcap;
   if (nwords_out) *nwords_out = nwords;
-  size_t bytes = sizeof(Smem) + 2 * (size_t)kcap + (4 + 2) * (size_t)m * nwords;
+  if (pcache_out) *pcache_out = pcache_rows;
+  size_t bytes = sizeof(Smem);
+  bytes += (size_t)warps * 34 * 8;                         // slots: start positions
+  bytes += (size_t)pcache_rows * 8;                        // suffix positions of the first rows
+  bytes += (size_t)warps * 66 * 4;                         // slots: lengths and comparable lengths
+  bytes += (size_t)m * nwords * 4;                         // node-start bitmaps
+  bytes += (size_t)m * nwords * 2;                         // jump tables
+  bytes += (size_t)nwords * 2;                             // tie counts
   return (bytes + 15) / 16 * 16;
 }
 
@@ -800,13 +986,15 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   a.tokens = d_tokens; a.parents = d_parents; a.depth = d_depth; a.pos_ids = d_pos_ids;
   a.mask = d_mask; a.n_nodes = d_n_nodes; a.match_n = d_match_n; a.match_range = d_match_range;
   a.node_count = d_node_count; a.status = d_status;
-  size_t smem = draft_smem_bytes(prm->K, prm->m, &a.kcap, &a.nwords);
+  a.idx = ds->v.idx;
+  auto smem_for = [&](int K, int threads) { return draft_smem_bytes(K, prm->m, threads, &a.kcap, &a.nwords, &a.pcache_rows); };
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool with_scratch = d_ws && ws_bytes >= split_workspace_bytes(B);
   bool batched = false;
   if (rest_status rc = wants_batched(search, B, with_scratch, &batched); rc != REST_OK) return rc;
   const bool narrow = ds->v.sa_bytes == 4;
   a.list = nullptr; a.list_count = nullptr; a.B = B; a.which = 0; a.light_rows = 0;
+  a.kcap = 0; a.nwords = 0; a.pcache_rows = 0;
   auto launch = [&](auto kern, int slot, int threads, int blocks, size_t bytes) -> rest_status {
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
                                             rest::kSmemSlotDraft + slot + (narrow ? 0 : 1), bytes));
@@ -815,20 +1003,25 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     REST_CUDA_TRY(cudaGetLastError());
     return REST_OK;
   };
-  const bool big = smem > kBigSmemBytes;
+  // candidate lists this long get 1024-thread blocks on every path
+  const bool big = (size_t)prm->K * prm->m >= kBigRowsTimesM;
   if (!batched) {
     // a call with at most one context per SM lasts as long as its slowest context: give each
     // context the whole SM (not the single context: its typical candidate list is short and
     // the larger block only adds barrier time)
     const int sms = rest::sm_count();
-    if (big || (B > 1 && B <= sms))
+    if (big || (B > 1 && B <= sms)) {
+      const size_t smem = smem_for(prm->K, kBigThreads);
       return narrow ? launch(rest_draft_kernel<int32_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem)
                     : launch(rest_draft_kernel<int64_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem);
+    }
+    const size_t smem = smem_for(prm->K, kThreads);
     return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWhole>, 0, kThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, false, kThreads, kWhole>, 0, kThreads, B, smem);
   }
   if (!with_scratch) {
     // no scratch for the context lists: search and build in one launch
+    const size_t smem = smem_for(prm->K, kTpThreads);
     return narrow ? launch(rest_draft_kernel<int32_t, true, kTpThreads, kWhole>, 2, kTpThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, true, kTpThreads, kWhole>, 2, kTpThreads, B, smem);
   }
@@ -842,20 +1035,22 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   rest_status rc = narrow ? launch(rest_draft_kernel<int32_t, true, kSearchThreads, kSearch>, 4, kSearchThreads, B, sizeof(Smem))
                           : launch(rest_draft_kernel<int64_t, true, kSearchThreads, kSearch>, 4, kSearchThreads, B, sizeof(Smem));
   if (rc != REST_OK) return rc;
-  const int kcap_all = a.kcap, nwords_all = a.nwords;
-  const size_t smem_light = draft_smem_bytes(a.light_rows, prm->m, &a.kcap, &a.nwords);
+  const size_t smem_light = smem_for(a.light_rows, kLightThreads);
   a.which = 0;
   rc = narrow ? launch(rest_draft_kernel<int32_t, true, kLightThreads, kBuild>, 6, kLightThreads, B, smem_light)
               : launch(rest_draft_kernel<int64_t, true, kLightThreads, kBuild>, 6, kLightThreads, B, smem_light);
   if (rc != REST_OK) return rc;
   if (prm->K > a.light_rows) {
-    a.kcap = kcap_all; a.nwords = nwords_all; a.which = 1;
-    if (big)
+    a.which = 1;
+    if (big) {
+      const size_t smem = smem_for(prm->K, kBigThreads);
       rc = narrow ? launch(rest_draft_kernel<int32_t, true, kBigThreads, kBuild>, 12, kBigThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, true, kBigThreads, kBuild>, 12, kBigThreads, B, smem);
-    else
+    } else {
+      const size_t smem = smem_for(prm->K, kThreads);
       rc = narrow ? launch(rest_draft_kernel<int32_t, true, kThreads, kBuild>, 8, kThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, true, kThreads, kBuild>, 8, kThreads, B, smem);
+    }
   }
   return rc;
 }

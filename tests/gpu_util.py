@@ -18,8 +18,8 @@ def to_dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).to(dev())
 
 
-def gpu_draft(T, sa, vocab, ctx, ctx_len, validate=False, **kw):
-    ds = rest.Datastore(to_dev(T), to_dev(sa), vocab, validate=validate)
+def gpu_draft(T, sa, vocab, ctx, ctx_len, validate=False, index=True, **kw):
+    ds = rest.Datastore(to_dev(T), to_dev(sa), vocab, validate=validate, index=index)
     out = rest.rest_draft(ds, to_dev(ctx), to_dev(np.asarray(ctx_len, np.int32)), **kw)
     torch.cuda.synchronize()
     res = {k: getattr(out, k).cpu().numpy() for k in DRAFT_KEYS}

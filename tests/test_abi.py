@@ -30,7 +30,10 @@ def test_status_strings_and_size_queries_without_a_gpu():
     L = rest.lib()
     assert L.rest_status_string(0) == b"ok"
     assert b"workspace" in L.rest_status_string(3)
-    assert L.rest_datastore_aux_bytes(64, 4, 10) == 2 * 4 + 256
+    # validation scratch (a bit per position + flags) plus the bucket index (a 256-byte header, the
+    # first-token table rounded to 256 bytes, and at least 4096 pair entries of 32 bytes)
+    assert L.rest_datastore_aux_bytes(64, 4, 10) == (2 * 4 + 256) + (256 + 256 + 4096 * 32)
+    assert L.rest_datastore_aux_bytes(64, 4, (1 << 22) + 1) == 2 * 4 + 256     # vocabulary too large to index
     # many (context, head) units -> a single key split, no scratch
     assert rest.tree_attention_workspace_bytes(256, 32, 64, 128, 4160) == 0
     # single stream, 32 heads -> one 8-block cluster per head merges on chip, no scratch

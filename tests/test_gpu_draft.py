@@ -55,8 +55,9 @@ def test_small_alphabets_match_oracle(seed, vocab, n_tok, K, m, N, sa_bytes):
         kw = dict(K=K, m=m, N=N, sample_mode=mode)
         ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
         for search in SEARCHES:
-            got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, search=search, **kw)
-            assert_draft_equal(got, ref, f"mode {mode}, search {search:#x}")
+            for index in (True, False):
+                got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, index=index, search=search, **kw)
+                assert_draft_equal(got, ref, f"mode {mode}, search {search:#x}, index {index}")
         got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=rest.REST_SEARCH_BATCHED, workspace=False, **kw)
         assert_draft_equal(got, ref, f"mode {mode}, batched in one launch")
 
@@ -73,8 +74,9 @@ def test_workload_recipes_match_oracle(name, n_tok, B):
     kw = dict(K=w.K, m=w.m, N=w.N, n_max=w.n_max, n_min=w.n_min)
     ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
     for search in SEARCHES:
-        got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, search=search, **kw)
-        assert_draft_equal(got, ref, f"{name}, search {search:#x}")
+        for index in (True, False):
+            got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, validate=True, index=index, search=search, **kw)
+            assert_draft_equal(got, ref, f"{name}, search {search:#x}, index {index}")
     assert (ref["n_nodes"] > 0).sum() > B // 2
 
 
@@ -132,6 +134,8 @@ def test_other_suffix_limits_and_repeatability():
             assert_draft_equal(got, ref, f"n_max={n_max} n_min={n_min} search {search:#x}")
             again, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, **kw)
             assert_draft_equal(again, got, "second run")
+            plain, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, index=False, **kw)
+            assert_draft_equal(plain, ref, f"n_max={n_max} n_min={n_min} search {search:#x}, no index")
 
 
 def test_bad_context_tokens_and_corrupt_datastore():
@@ -200,5 +204,7 @@ def test_random_parameters_against_the_oracle():
                   n_min=int(rng.integers(1, n_max + 1)), sample_mode=int(rng.integers(0, 2)))
         ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
         search = SEARCHES[case % 2]
-        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=search, **kw)
-        assert_draft_equal(got, ref, f"case {case}: vocab {vocab}, {n_tok} tokens, {kw}, search {search:#x}")
+        index = (case // 2) % 2 == 0
+        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=search, index=index, **kw)
+        assert_draft_equal(got, ref, f"case {case}: vocab {vocab}, {n_tok} tokens, {kw}, search {search:#x}, "
+                                     f"index {index}")
