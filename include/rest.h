@@ -4,6 +4,8 @@
  *
  * Set-up:       rest_suffix_array_build, rest_datastore_create  (Sec. 3.2, datastore construction)
  * Draft side:   rest_draft                                 (Sec. 3.2, Algorithms 1 and 2)
+ *               rest_retrieve, rest_gather_rows, rest_draft_from_runs: the same in pieces, for a
+ *               datastore spread over several GPUs
  * Verify side:  rest_tree_attention, rest_accept           (Sec. 3.2, draft verification / acceptance)
  * Between steps: rest_kv_commit                            (the accepted path joins the prefix)
  * Health:       rest_device_error_flags
@@ -116,6 +118,20 @@ rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n_tokens, co
 void rest_datastore_destroy(rest_datastore* ds);
 
 /*
+ * rest_datastore_create_shard - a datastore whose suffix array lists only n_sa <= n_tokens of
+ * the positions, e.g. one shard of a token stream that is spread over several GPUs (Sec. 5,
+ * "Effect of the datastore size": the datastore may outgrow one device).  A shard holds the
+ * tokens of its own position range followed by the first tokens of the next shard (at least
+ * n_max + m of them), and its suffix array orders the positions of its own range only, so that
+ * every occurrence in the whole stream is found by exactly one shard and its continuation is
+ * complete.  Everything else as rest_datastore_create; d_sa has n_sa entries, all distinct
+ * positions in [0, n_tokens), ordered like a suffix array.
+ */
+rest_status rest_datastore_create_shard(const int32_t* d_tokens, uint64_t n_tokens, const void* d_sa,
+                                        uint64_t n_sa, int32_t sa_bytes, uint32_t vocab, uint32_t flags,
+                                        void* d_aux, size_t aux_bytes, void* stream, rest_datastore** out);
+
+/*
  * rest_draft - Algorithm 1 (longest-suffix exact-match retrieval), Algorithm 2 (Trie weights,
  * the c heaviest nodes) and the breadth-first pseudo sequence with its tree-attention mask
  * (Sec. 3.2 "Draft verification"), for B independent contexts.
@@ -156,6 +172,56 @@ rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params
                        int32_t* d_pos_ids, uint32_t* d_mask, int32_t* d_n_nodes,
                        int32_t* d_match_n, int64_t* d_match_range, int32_t* d_node_count,
                        int32_t* d_status, void* d_ws, size_t ws_bytes, void* stream);
+
+/*
+ * The draft in pieces, for a datastore spread over several GPUs (Algorithms 1 and 2 over the
+ * union of the shards; Sec. 5 "Effect of the datastore size").  Per decoding step:
+ *   1. every GPU:  rest_retrieve on its shard -> its longest matching suffix length and range;
+ *   2. exchange:   the winning length n* is the maximum over the shards (a shorter suffix of a
+ *                  match is a match, so a shard either matches n* or contributes nothing);
+ *                  shards that match n* report their hit counts cnt_i; with cnt = sum cnt_i,
+ *                  shard i contributes all its rows when cnt <= K, else
+ *                  floor(K C_i / cnt) - floor(K C_(i-1) / cnt) rows (C_i = cnt_1 + ... + cnt_i),
+ *                  spread over its range like rest_draft spreads K over one range.  With one
+ *                  shard this is exactly rest_draft's rule;
+ *   3. every GPU:  rest_gather_rows -> its rows, in lexicographic order (one sorted run);
+ *   4. exchange:   the runs of all shards travel to the GPU that builds the tree;
+ *   5. builder:    rest_draft_from_runs merges the runs and runs Algorithm 2 and the tree
+ *                  emission unchanged.
+ * The exchanges are ordinary collectives on small tensors and belong to the caller (the Python
+ * package does them with torch.distributed).
+ *
+ * rest_retrieve       Algorithm 1 alone: d_match_n[b], d_match_range[b] = {lo, hi}, d_status[b];
+ *                     arguments as in rest_draft (K, m, N, sample_mode of `params` are not used).
+ * rest_gather_rows    candidate j < take[b] of context b: the suffix-array slot
+ *                     lo + floor(j cnt / take[b]) (lo + j with REST_SAMPLE_FIRST_K or when
+ *                     take[b] = cnt), its up to m tokens after the match into d_rows[b][j][0..m)
+ *                     (zero padded) and their number into d_row_len[b][j]; rows j >= take[b] get
+ *                     length 0.  d_match_n / d_match_range as written by rest_retrieve (a shard
+ *                     that lost sets take[b] = 0).  Kr = row capacity per context (<= 32768).
+ *                     d_status[b] is OR-ed with REST_CTX_BAD_DATASTORE on an entry out of range.
+ * rest_draft_from_runs  d_rows int32[B][R][Kr][m], d_row_len int32[B][R][Kr], d_run_rows
+ *                     int32[B][R] (rows of run r in use; each run in lexicographic order, a row
+ *                     that is a prefix of another first; R * Kr <= 32768).  Outputs as rest_draft
+ *                     (d_node_count may be NULL); runs out of order give status
+ *                     REST_CTX_BAD_DATASTORE and an empty tree.  d_ws: scratch of
+ *                     rest_draft_from_runs_workspace_bytes(B, R, Kr) bytes.
+ */
+rest_status rest_retrieve(const rest_datastore* ds, const rest_draft_params* params,
+                          const int32_t* d_ctx, int64_t ctx_stride, const int32_t* d_ctx_len,
+                          int32_t B, int32_t* d_match_n, int64_t* d_match_range, int32_t* d_status,
+                          void* stream);
+rest_status rest_gather_rows(const rest_datastore* ds, const rest_draft_params* params,
+                             const int32_t* d_match_n, const int64_t* d_match_range,
+                             const int32_t* d_take, int32_t B, int32_t Kr, int32_t* d_rows,
+                             int32_t* d_row_len, int32_t* d_status, void* stream);
+size_t rest_draft_from_runs_workspace_bytes(int32_t B, int32_t R, int32_t Kr);
+rest_status rest_draft_from_runs(const rest_draft_params* params, const int32_t* d_rows,
+                                 const int32_t* d_row_len, const int32_t* d_run_rows, int32_t R,
+                                 int32_t Kr, const int32_t* d_ctx_len, int32_t B, int32_t* d_tokens,
+                                 int32_t* d_parents, int32_t* d_depth, int32_t* d_pos_ids,
+                                 uint32_t* d_mask, int32_t* d_n_nodes, int32_t* d_node_count,
+                                 int32_t* d_status, void* d_ws, size_t ws_bytes, void* stream);
 
 /*
  * rest_tree_attention - attention of the N draft positions of each context over the prefix

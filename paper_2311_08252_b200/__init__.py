@@ -29,8 +29,9 @@ REST_DS_VALIDATE = 1
 REST_DS_INDEX = 2
 
 EXPORTS = (
-    "rest_datastore_aux_bytes", "rest_datastore_create", "rest_datastore_destroy",
-    "rest_draft_workspace_bytes", "rest_draft",
+    "rest_datastore_aux_bytes", "rest_datastore_create", "rest_datastore_create_shard",
+    "rest_datastore_destroy", "rest_draft_workspace_bytes", "rest_draft",
+    "rest_retrieve", "rest_gather_rows", "rest_draft_from_runs_workspace_bytes", "rest_draft_from_runs",
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
     "rest_tree_attention_static_scratch",
     "rest_device_error_flags", "rest_kv_commit", "rest_probe_dependent_reads",
@@ -71,6 +72,18 @@ def lib():
     L.rest_datastore_create.restype = i32
     L.rest_datastore_create.argtypes = [vp, u64, vp, i32, u32, u32, vp, sz, vp,
                                         ctypes.POINTER(vp)]
+    L.rest_datastore_create_shard.restype = i32
+    L.rest_datastore_create_shard.argtypes = [vp, u64, vp, u64, i32, u32, u32, vp, sz, vp,
+                                              ctypes.POINTER(vp)]
+    L.rest_retrieve.restype = i32
+    L.rest_retrieve.argtypes = [vp, ctypes.POINTER(_Params), vp, i64, vp, i32, vp, vp, vp, vp]
+    L.rest_gather_rows.restype = i32
+    L.rest_gather_rows.argtypes = [vp, ctypes.POINTER(_Params), vp, vp, vp, i32, i32, vp, vp, vp, vp]
+    L.rest_draft_from_runs_workspace_bytes.restype = sz
+    L.rest_draft_from_runs_workspace_bytes.argtypes = [i32, i32, i32]
+    L.rest_draft_from_runs.restype = i32
+    L.rest_draft_from_runs.argtypes = [ctypes.POINTER(_Params), vp, vp, vp, i32, i32, vp, i32] + [vp] * 8 + \
+        [vp, sz, vp]
     L.rest_datastore_destroy.restype = None
     L.rest_datastore_destroy.argtypes = [vp]
     L.rest_draft_workspace_bytes.restype = sz
@@ -158,8 +171,8 @@ class Datastore:
         if not (tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()):
             raise RestError("tokens must be a contiguous int32 CUDA tensor")
         if not (sa.is_cuda and sa.dtype in (torch.int32, torch.int64) and sa.is_contiguous()
-                and sa.numel() == tokens.numel()):
-            raise RestError("sa must be a contiguous int32/int64 CUDA tensor as long as tokens")
+                and 0 < sa.numel() <= tokens.numel()):
+            raise RestError("sa must be a contiguous int32/int64 CUDA tensor, at most as long as tokens")
         self.tokens, self.sa, self.vocab = tokens, sa, int(vocab)
         self.n_tokens = tokens.numel()
         self.sa_bytes = sa.element_size()
@@ -170,9 +183,10 @@ class Datastore:
             aux_bytes = L.rest_datastore_aux_bytes(self.n_tokens, self.sa_bytes, self.vocab)
             aux = torch.empty(aux_bytes, dtype=torch.uint8, device=tokens.device)
         h = ctypes.c_void_p()
-        rc = L.rest_datastore_create(tokens.data_ptr(), self.n_tokens, sa.data_ptr(), self.sa_bytes,
-                                     self.vocab, flags, _ptr(aux), aux_bytes, _stream(stream),
-                                     ctypes.byref(h))
+        # a suffix array shorter than the token stream lists the positions of a shard's own range
+        rc = L.rest_datastore_create_shard(tokens.data_ptr(), self.n_tokens, sa.data_ptr(), sa.numel(),
+                                           self.sa_bytes, self.vocab, flags, _ptr(aux), aux_bytes,
+                                           _stream(stream), ctypes.byref(h))
         _check(rc, "rest_datastore_create")
         self._h = h
         self._aux = aux if index else None      # the handle reads the index for its whole life
@@ -256,6 +270,69 @@ def rest_draft(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, K=5000, m=10, N=6
                       out.match_n.data_ptr(), out.match_range.data_ptr(), _ptr(out.node_count),
                       out.status.data_ptr(), ws_ptr, ws_bytes, _stream(stream))
     _check(rc, "rest_draft")
+    return out
+
+
+def rest_retrieve(ds: Datastore, ctx, ctx_len, n_max=16, n_min=2, stream=None):
+    """Algorithm 1 alone: returns (match_n int32[B], match_range int64[B,2], status int32[B])."""
+    import torch
+    L = lib()
+    _dev_i32(ctx_len, "ctx_len")
+    if not (ctx.is_cuda and ctx.dtype == torch.int32 and ctx.dim() == 2 and ctx.stride(1) == 1):
+        raise RestError("ctx must be an int32 CUDA tensor [B, Lc] with contiguous rows")
+    B = ctx.shape[0]
+    match_n = torch.empty(B, dtype=torch.int32, device=ctx.device)
+    match_range = torch.empty((B, 2), dtype=torch.int64, device=ctx.device)
+    status = torch.empty(B, dtype=torch.int32, device=ctx.device)
+    prm = _Params(n_max, n_min, 1, 1, 1, 0, 0)
+    _check(L.rest_retrieve(ds._h, ctypes.byref(prm), ctx.data_ptr(), ctx.stride(0), ctx_len.data_ptr(), B,
+                           match_n.data_ptr(), match_range.data_ptr(), status.data_ptr(), _stream(stream)),
+           "rest_retrieve")
+    return match_n, match_range, status
+
+
+def rest_gather_rows(ds: Datastore, match_n, match_range, take, Kr: int, m=10,
+                     sample_mode=REST_SAMPLE_STRIDED, status=None, stream=None):
+    """The take[b] sampled candidate rows of every context's matched range: returns
+    (rows int32[B,Kr,m], row_len int32[B,Kr], status int32[B])."""
+    import torch
+    L = lib()
+    for t, nm in ((match_n, "match_n"), (take, "take")):
+        _dev_i32(t, nm)
+    B = match_n.shape[0]
+    rows = torch.empty((B, Kr, m), dtype=torch.int32, device=match_n.device)
+    row_len = torch.empty((B, Kr), dtype=torch.int32, device=match_n.device)
+    if status is None:
+        status = torch.zeros(B, dtype=torch.int32, device=match_n.device)
+    prm = _Params(16, 2, Kr, m, 1, sample_mode, 0)
+    _check(L.rest_gather_rows(ds._h, ctypes.byref(prm), match_n.data_ptr(), match_range.data_ptr(),
+                              take.data_ptr(), B, Kr, rows.data_ptr(), row_len.data_ptr(),
+                              status.data_ptr(), _stream(stream)), "rest_gather_rows")
+    return rows, row_len, status
+
+
+def rest_draft_from_runs(rows, row_len, run_rows, ctx_len, m=None, N=64, out: DraftOutput | None = None,
+                         stream=None) -> DraftOutput:
+    """Trees from candidate rows handed in as sorted runs: rows int32[B,R,Kr,m], row_len
+    int32[B,R,Kr], run_rows int32[B,R].  match_n / match_range of the result are not written."""
+    import torch
+    L = lib()
+    for t, nm in ((rows, "rows"), (row_len, "row_len"), (run_rows, "run_rows"), (ctx_len, "ctx_len")):
+        _dev_i32(t, nm)
+    B, R, Kr, mm = rows.shape
+    m = mm if m is None else m
+    if m != mm or row_len.shape != (B, R, Kr) or run_rows.shape != (B, R):
+        raise RestError("rows [B,R,Kr,m], row_len [B,R,Kr] and run_rows [B,R] do not fit together")
+    if out is None:
+        out = alloc_draft_output(B, N, rows.device)
+    ws_bytes = L.rest_draft_from_runs_workspace_bytes(B, R, Kr)
+    ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=rows.device)
+    prm = _Params(16, 2, R * Kr, m, N, 0, 0)
+    _check(L.rest_draft_from_runs(ctypes.byref(prm), rows.data_ptr(), row_len.data_ptr(), run_rows.data_ptr(),
+                                  R, Kr, ctx_len.data_ptr(), B, out.tokens.data_ptr(), out.parents.data_ptr(),
+                                  out.depth.data_ptr(), out.pos_ids.data_ptr(), out.mask.data_ptr(),
+                                  out.n_nodes.data_ptr(), _ptr(out.node_count), out.status.data_ptr(),
+                                  ws.data_ptr(), ws_bytes, _stream(stream)), "rest_draft_from_runs")
     return out
 
 

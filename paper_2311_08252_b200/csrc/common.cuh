@@ -18,8 +18,8 @@ cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t byte
 // usable device.
 int sm_count();
 // One slot per kernel instance, library-wide: two kernels on one slot would skip each other's
-// attribute call.  The draft kernel's instances take kSmemSlotDraft + 0 ... 13.
-constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 14, kSmemSlotAttnWide = 15, kSmemSlots = 16;
+// attribute call.  The draft kernel's instances take kSmemSlotDraft + 0 ... 15.
+constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 16, kSmemSlotAttnWide = 17, kSmemSlots = 18;
 
 #define REST_CUDA_TRY(expr)                                              \
   do {                                                                   \
@@ -56,6 +56,7 @@ struct DatastoreView {
   const int32_t* tokens;
   const void* sa;
   int64_t n_tokens;
+  int64_t n_sa;          // suffix-array entries: n_tokens, or fewer when the array lists only some positions
   int32_t sa_bytes;
   uint32_t vocab;
   BucketIndex idx;

@@ -64,13 +64,14 @@ constexpr int kOrderWindow = 32;   // tokens of each suffix that the order check
 // flags[0] |= 1 token out of range, 2 entry out of range, 4 duplicate entry, 8 order violated
 template <typename SaT>
 __global__ void validate_kernel(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
-                                int64_t n, uint32_t vocab, uint32_t* __restrict__ seen,
+                                int64_t n, int64_t n_sa, uint32_t vocab, uint32_t* __restrict__ seen,
                                 uint32_t* __restrict__ flags) {
   int64_t stride = (int64_t)gridDim.x * blockDim.x;
   uint32_t bad = 0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
     int32_t t = T[i];
     if (t < 0 || (uint32_t)t >= vocab) bad |= 1u;
+    if (i >= n_sa) continue;             // the array may list fewer positions than there are tokens
     int64_t p = (int64_t)sa[i];
     if (p < 0 || p >= n) { bad |= 2u; continue; }
     uint32_t bit = 1u << (p & 31);
@@ -138,21 +139,21 @@ __device__ __forceinline__ bool pair_at(const int32_t* __restrict__ T, const SaT
 // run has at least min_run members (seen by looking min_run - 1 slots ahead or back).
 template <typename SaT>
 __global__ void index_build_kernel(const int32_t* __restrict__ T, const SaT* __restrict__ sa, int64_t n,
-                                   uint32_t vocab, int64_t min_run, long long* __restrict__ first,
+                                   int64_t n_sa, uint32_t vocab, int64_t min_run, long long* __restrict__ first,
                                    unsigned long long* __restrict__ table, uint32_t group_mask,
                                    uint32_t* __restrict__ unusable) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_sa; i += stride) {
     int32_t t0, t1, a0 = -2, a1 = -2, b0 = -2, b1 = -2;
     // a datastore with an entry or a token out of range gets no index: searches then run over
     // the whole array, where such an entry is reported when it is met
     if (!pair_at(T, sa, n, vocab, i, t0, t1)) { *unusable = 1u; continue; }
     if (i > 0 && !pair_at(T, sa, n, vocab, i - 1, a0, a1)) a0 = -2;
-    if (i + 1 < n && !pair_at(T, sa, n, vocab, i + 1, b0, b1)) b0 = -2;
+    if (i + 1 < n_sa && !pair_at(T, sa, n, vocab, i + 1, b0, b1)) b0 = -2;
     if (i == 0 || a0 != t0) first[t0] = i;
     if (t1 < 0) continue;
     const bool starts = i == 0 || a0 != t0 || a1 != t1;
-    const bool ends = i + 1 == n || b0 != t0 || b1 != t1;
+    const bool ends = i + 1 == n_sa || b0 != t0 || b1 != t1;
     if (!starts && !ends) continue;
     bool long_enough = true;
     if (min_run > 1) {
@@ -160,7 +161,7 @@ __global__ void index_build_kernel(const int32_t* __restrict__ T, const SaT* __r
       if (!(starts && ends)) {
         const int64_t far = starts ? i + min_run - 1 : i - min_run + 1;
         int32_t f0, f1;
-        long_enough = far >= 0 && far < n && pair_at(T, sa, n, vocab, far, f0, f1) && f0 == t0 && f1 == t1;
+        long_enough = far >= 0 && far < n_sa && pair_at(T, sa, n, vocab, far, f0, f1) && f0 == t0 && f1 == t1;
       }
     }
     if (!long_enough) continue;
@@ -215,9 +216,18 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
                                              const void* d_sa, int32_t sa_bytes, uint32_t vocab,
                                              uint32_t flags, void* d_aux, size_t aux_bytes,
                                              void* stream, rest_datastore** out) {
+  return rest_datastore_create_shard(d_tokens, n_tokens, d_sa, n_tokens, sa_bytes, vocab, flags, d_aux,
+                                     aux_bytes, stream, out);
+}
+
+extern "C" rest_status rest_datastore_create_shard(const int32_t* d_tokens, uint64_t n_tokens,
+                                                   const void* d_sa, uint64_t n_sa, int32_t sa_bytes,
+                                                   uint32_t vocab, uint32_t flags, void* d_aux,
+                                                   size_t aux_bytes, void* stream, rest_datastore** out) {
   if (!out) return REST_INVALID_ARG;
   *out = nullptr;
-  if (!d_tokens || !d_sa || n_tokens == 0 || vocab == 0 || vocab >= 0x80000000u)
+  if (!d_tokens || !d_sa || n_tokens == 0 || n_sa == 0 || n_sa > n_tokens || vocab == 0 ||
+      vocab >= 0x80000000u)
     return REST_INVALID_ARG;
   if (sa_bytes != 4 && sa_bytes != 8) return REST_INVALID_ARG;
   if (sa_bytes == 4 && n_tokens > 0x7FFFFFFFull) return REST_INVALID_ARG;
@@ -239,10 +249,10 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
     int blocks = (int)((n_tokens + 255) / 256 < wave ? (n_tokens + 255) / 256 : wave);
     if (sa_bytes == 4)
       validate_kernel<int32_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int32_t*>(d_sa),
-                                                       (int64_t)n_tokens, vocab, d_seen, d_flags);
+                                                       (int64_t)n_tokens, (int64_t)n_sa, vocab, d_seen, d_flags);
     else
       validate_kernel<int64_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int64_t*>(d_sa),
-                                                       (int64_t)n_tokens, vocab, d_seen, d_flags);
+                                                       (int64_t)n_tokens, (int64_t)n_sa, vocab, d_seen, d_flags);
     rest::count_launch();
     REST_CUDA_TRY(cudaGetLastError());
     uint32_t h_flags = 0;
@@ -262,14 +272,14 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
     REST_CUDA_TRY(cudaMemsetAsync(base, 0, kIndexHeaderBytes, st));
     const uint32_t group_mask = (uint32_t)(il.entries / 4 - 1);
     const uint64_t wave = (uint64_t)(rest::sm_count() > 0 ? rest::sm_count() : 148) * 16;
-    const int blocks = (int)((n_tokens + 255) / 256 < wave ? (n_tokens + 255) / 256 : wave);
+    const int blocks = (int)((n_sa + 255) / 256 < wave ? (n_sa + 255) / 256 : wave);
     if (sa_bytes == 4)
       index_build_kernel<int32_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int32_t*>(d_sa),
-                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask, unusable);
+                                                          (int64_t)n_tokens, (int64_t)n_sa, vocab, il.min_run, first, table, group_mask, unusable);
     else
       index_build_kernel<int64_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int64_t*>(d_sa),
-                                                          (int64_t)n_tokens, vocab, il.min_run, first, table, group_mask, unusable);
-    index_fill_kernel<<<1, 1024, 0, st>>>(first, vocab, (int64_t)n_tokens);
+                                                          (int64_t)n_tokens, (int64_t)n_sa, vocab, il.min_run, first, table, group_mask, unusable);
+    index_fill_kernel<<<1, 1024, 0, st>>>(first, vocab, (int64_t)n_sa);
     rest::count_launch(2);
     REST_CUDA_TRY(cudaGetLastError());
     idx.first = first; idx.table = table; idx.group_mask = group_mask; idx.unusable = unusable;
@@ -280,6 +290,7 @@ extern "C" rest_status rest_datastore_create(const int32_t* d_tokens, uint64_t n
   ds->v.tokens = d_tokens;
   ds->v.sa = d_sa;
   ds->v.n_tokens = (int64_t)n_tokens;
+  ds->v.n_sa = (int64_t)n_sa;
   ds->v.sa_bytes = sa_bytes;
   ds->v.vocab = vocab;
   *out = ds;

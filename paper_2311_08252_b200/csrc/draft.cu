@@ -66,6 +66,7 @@ struct DraftArgs {
   const int32_t* T;
   const void* sa;
   int64_t n_tokens;
+  int64_t n_sa;
   uint32_t vocab;
   int n_max, n_min, K, m, N, sample_mode;
   const int32_t* ctx;
@@ -80,6 +81,12 @@ struct DraftArgs {
   int nwords;   // bitmap words per depth
   int kcap;     // rows the block's shared memory holds, a multiple of 32
   int pcache_rows;   // rows whose suffix position is kept in shared memory
+  // rows handed in by the caller as R sorted runs per context (rest_draft_from_runs): T then
+  // points at the rows [B][R][Kr][m]
+  const int32_t* row_len;     // [B][R][Kr]
+  const int32_t* run_rows;    // [B][R]
+  uint32_t* order;            // [B][kcap] scratch: merged order of the rows
+  int R, Kr;
   // three-launch form of the batched path: the search launch sorts the contexts that matched
   // into two lists by candidate count, the two build launches take one list each
   int32_t* list;          // [2][B] context indices
@@ -258,7 +265,7 @@ struct Smem {
 // index.  Warp-cooperative: four lanes read the four entries of the pair's group (one 128-byte
 // line).  false when the pair is not stored.
 __device__ __forceinline__ bool index_pair_range(const rest::BucketIndex& idx, uint32_t t0, uint32_t t1,
-                                                 int lane, int64_t n_tokens, int64_t& lo, int64_t& hi) {
+                                                 int lane, int64_t n_slots, int64_t& lo, int64_t& hi) {
   const unsigned long long key = rest::index_pair_key(t0, t1);
   const unsigned long long* grp = idx.table + (size_t)rest::index_group_of(key, idx.group_mask) * 16;
   unsigned long long k = rest::kIndexEmptyKey;
@@ -268,7 +275,7 @@ __device__ __forceinline__ bool index_pair_range(const rest::BucketIndex& idx, u
     l = (long long)__ldg(grp + lane * 4 + 1);
     h = (long long)__ldg(grp + lane * 4 + 2);
   }
-  const unsigned hit = __ballot_sync(kFull, lane < 4 && k == key && l >= 0 && h > l && h <= n_tokens);
+  const unsigned hit = __ballot_sync(kFull, lane < 4 && k == key && l >= 0 && h > l && h <= n_slots);
   if (hit == 0) return false;
   const int src = __ffs(hit) - 1;
   lo = __shfl_sync(kFull, l, src);
@@ -294,8 +301,21 @@ __device__ __forceinline__ uint32_t cut_short_mask(const Smem& s, int ntrunc, in
 // fewer random DRAM reads per context (see phase 1).
 // PART: kWhole = search and build in one launch; kSearch = phase 1 only (writes match_n and
 // match_range, the defaults of every output slot, and the context's index into one of two
-// lists); kBuild = phases 2-4 for the contexts of one list.
-enum { kWhole = 0, kSearch = 1, kBuild = 2 };
+// lists); kBuild = phases 2-4 for the contexts of one list; kRetrieve = phase 1 alone, nothing
+// but match_n, match_range and status written (rest_retrieve); kFromRuns = phases 2-4 over rows
+// that the caller hands in as sorted runs, merged first (rest_draft_from_runs).
+enum { kWhole = 0, kSearch = 1, kBuild = 2, kRetrieve = 3, kFromRuns = 4 };
+
+// Three-way comparison of two candidate rows (tokens as unsigned integers; a row that is a
+// proper prefix of the other sorts first).
+__device__ __forceinline__ int compare_rows(const int32_t* __restrict__ y, int ylen, const int (&x)[kMaxM], int xlen) {
+  const int lim = ylen < xlen ? ylen : xlen;
+  for (int k = 0; k < lim; ++k) {
+    const uint32_t a = (uint32_t)y[k], b = (uint32_t)x[k];
+    if (a != b) return a < b ? -1 : 1;
+  }
+  return ylen == xlen ? 0 : (ylen < xlen ? -1 : 1);
+}
 template <typename SaT, bool TP, int NT, int PART>
 __global__ void __launch_bounds__(NT, 1024 / NT)
 rest_draft_kernel(DraftArgs a) {
@@ -325,11 +345,13 @@ rest_draft_kernel(DraftArgs a) {
   const int32_t* __restrict__ T = a.T;
   const SaT* __restrict__ sa = static_cast<const SaT*>(a.sa);
   const int64_t n_tokens = a.n_tokens;
+  const int64_t n_sa = a.n_sa;          // slots of the suffix array (searches), n_tokens bounds positions
   const int clen = a.ctx_len[b];
-  const int32_t* ctx = a.ctx + (int64_t)b * a.ctx_stride;
+  const int32_t* ctx = PART == kFromRuns ? nullptr : a.ctx + (int64_t)b * a.ctx_stride;
   // read early, beside the context: whether the bucket index may be used (not when its build
   // met a suffix-array entry or a token out of range)
-  const uint32_t index_unusable = (PART != kBuild && a.idx.first != nullptr) ? __ldg(a.idx.unusable) : 1u;
+  const uint32_t index_unusable =
+      (PART != kBuild && PART != kFromRuns && a.idx.first != nullptr) ? __ldg(a.idx.unusable) : 1u;
 
   // Unused-slot defaults; thread i owns slots i, i + NT, ... for the whole kernel (a build
   // launch finds them written by the search launch).
@@ -342,15 +364,17 @@ rest_draft_kernel(DraftArgs a) {
     }
   };
   auto report_empty = [&]() {                      // by thread 0, after a barrier
-    a.status[b] = s.err; a.n_nodes[b] = 0; a.match_n[b] = 0;
-    a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0;
+    a.status[b] = s.err;
+    if (a.n_nodes) a.n_nodes[b] = 0;
+    if (a.match_n) a.match_n[b] = 0;
+    if (a.match_range) { a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0; }
   };
-  if constexpr (PART != kBuild) write_defaults();
+  if constexpr (PART == kWhole || PART == kSearch || PART == kFromRuns) write_defaults();
   const int nq = min(a.n_max, max(clen, 0));   // context tokens that can take part
   if (tid == 0) { s.err = 0; s.big_total = 0; s.nsel = 0; s.ntrunc = 0; }
-  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; s.bhi[tid] = n_tokens; }
+  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; s.bhi[tid] = n_sa; }
   if (tid < 5 * (kMaxM + 1)) (&s.small[0][0])[tid] = 0;
-  if constexpr (PART != kSearch) {
+  if constexpr (PART != kSearch && PART != kRetrieve) {
     for (int i = tid; i < kHistHi; i += NT) s.hist_hi[i] = 0;
     for (int i = tid; i < kHistLo; i += NT) s.hist_lo[i] = 0;
   }
@@ -360,6 +384,47 @@ rest_draft_kernel(DraftArgs a) {
     n_win = a.match_n[b];
     if (tid == 0) { s.lb[n_win] = a.match_range[2 * b]; s.ub[n_win] = a.match_range[2 * b + 1]; }
     __syncthreads();
+  } else if constexpr (PART == kFromRuns) {
+    // The rows arrive as R runs, each in lexicographic order (the rows of one suffix-array
+    // range are).  Position of row i of run r in the merged order: i, plus for every other run
+    // the number of its rows that sort before this one (equal rows: the lower run first), found
+    // by bisection.  Runs that are not in order leave slots of the order unwritten, which the
+    // gather below reports as a bad datastore.
+    const int R = a.R, Kr = a.Kr;
+    const int32_t* nrun = a.run_rows + (int64_t)b * R;
+    const int32_t* rows = T + (int64_t)b * R * Kr * m;
+    const int32_t* lens = a.row_len + (int64_t)b * R * Kr;
+    uint32_t* ord = a.order + (int64_t)b * a.kcap;
+    int total = 0;
+    for (int r = 0; r < R; ++r) total += min(max(nrun[r], 0), Kr);
+    for (int x = tid; x < a.kcap; x += NT) ord[x] = 0xFFFFFFFFu;
+    __syncthreads();
+    for (int flat = tid; flat < R * Kr; flat += NT) {
+      const int r = flat / Kr, i = flat - r * Kr;
+      if (i >= min(max(nrun[r], 0), Kr)) continue;
+      int mine[kMaxM];
+      const int mylen = min(max(lens[flat], 0), m);
+#pragma unroll
+      for (int k = 0; k < kMaxM; ++k) mine[k] = k < mylen ? rows[(int64_t)flat * m + k] : 0;
+      int rank = i;
+      for (int r2 = 0; r2 < R; ++r2) {
+        if (r2 == r) continue;
+        int lo2 = 0, hi2 = min(max(nrun[r2], 0), Kr);
+        while (lo2 < hi2) {
+          const int mid = (lo2 + hi2) >> 1, f2 = r2 * Kr + mid;
+          const int c = compare_rows(rows + (int64_t)f2 * m, min(max(lens[f2], 0), m), mine, mylen);
+          if (c < 0 || (c == 0 && r2 < r)) lo2 = mid + 1; else hi2 = mid;
+        }
+        rank += lo2;
+      }
+      if (rank < a.kcap) ord[rank] = (uint32_t)flat;
+    }
+    if (tid == 0) { s.lb[0] = 0; s.ub[0] = total < a.kcap ? total : a.kcap; }
+    __syncthreads();
+    if (total == 0) {
+      if (tid == 0) report_empty();
+      return;
+    }
   } else {
   if (tid < nq) {
     int t = ctx[clen - nq + tid];
@@ -388,14 +453,14 @@ rest_draft_kernel(DraftArgs a) {
       // also stores the query's first token pair, every suffix that starts with that pair lies
       // in [lo0, hi0).  Slot hi0 (or the end of the array) compares greater than the query.
       int64_t lo0 = __ldg(a.idx.first + q[0]), hi0 = __ldg(a.idx.first + q[0] + 1);
-      lo0 = lo0 < 0 ? 0 : (lo0 > n_tokens ? n_tokens : lo0);
-      hi0 = hi0 < lo0 ? lo0 : (hi0 > n_tokens ? n_tokens : hi0);
+      lo0 = lo0 < 0 ? 0 : (lo0 > n_sa ? n_sa : lo0);
+      hi0 = hi0 < lo0 ? lo0 : (hi0 > n_sa ? n_sa : hi0);
       if (n == 1) {                       // the first-token range is the answer
         if (lane == 0) { s.lb[1] = lo0; s.ub[1] = hi0; s.bhi[1] = hi0; }
         return;
       }
       int64_t plo, phi;
-      if (index_pair_range(a.idx, (uint32_t)q[0], (uint32_t)q[1], lane, n_tokens, plo, phi) &&
+      if (index_pair_range(a.idx, (uint32_t)q[0], (uint32_t)q[1], lane, n_sa, plo, phi) &&
           plo >= lo0 && phi <= hi0) {
         if (n == 2) {                     // the pair's range is the answer
           if (lane == 0) { s.lb[2] = plo; s.ub[2] = phi; s.bhi[2] = phi; }
@@ -407,8 +472,8 @@ rest_draft_kernel(DraftArgs a) {
       lb = warp_first_true<SaT, false, kArity, 0>(T, sa, n_tokens, lo0, hi0, q, n, lane, eq, bad, &next_gt);
       if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < hi0) ? next_gt : lb; }
     } else {
-      lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_tokens, q, n, lane, eq, bad, &next_gt);
-      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_tokens) ? next_gt : lb; }
+      lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_sa, q, n, lane, eq, bad, &next_gt);
+      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_sa) ? next_gt : lb; }
     }
     if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
   };
@@ -501,6 +566,13 @@ rest_draft_kernel(DraftArgs a) {
   }  // PART != kBuild
   const int64_t lo = s.lb[n_win], hi = s.ub[n_win];
   const int64_t cnt = hi - lo;
+  if constexpr (PART == kRetrieve) {
+    if (tid == 0) {
+      a.status[b] = 0; a.match_n[b] = n_win;
+      a.match_range[2 * b] = lo; a.match_range[2 * b + 1] = hi;
+    }
+    return;
+  }
   if constexpr (PART == kSearch) {
     // hand the context to the build launch that fits its candidate count
     if (tid == 0) {
@@ -513,6 +585,8 @@ rest_draft_kernel(DraftArgs a) {
     return;
   }
   const int Kp = (int)(cnt < (int64_t)a.K ? cnt : (int64_t)a.K);
+  // where the rows' tokens live: the token stream, or the caller's rows of this context
+  const int32_t* __restrict__ Trow = PART == kFromRuns ? T + (int64_t)b * a.R * a.Kr * m : T;
   const int nwords = a.nwords;
   const int niter = (Kp + NT - 1) / NT;
   const int nw = (Kp + 31) >> 5;            // bitmap words that hold rows
@@ -533,40 +607,51 @@ rest_draft_kernel(DraftArgs a) {
     const uint32_t magic = (65536u + (uint32_t)m - 1u) / (uint32_t)m;    // f / m = (f * magic) >> 16 for f < 600
     const int nload = (33 * m + 31) >> 5;
     const int src_lane = (lane - m) & 31;
+    // where row j comes from: the suffix-array entry of its sampled slot, or (rows handed in
+    // as runs) its place in the caller's row array, through the merged order
+    const uint32_t* ord = PART == kFromRuns ? a.order + (int64_t)b * a.kcap : nullptr;
+    auto row_entry = [&](int j) -> int64_t {
+      if constexpr (PART == kFromRuns) return (int64_t)ord[j];
+      else return (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
+    };
+    // start of the row's tokens (relative to Trow) and its length; `bad` when the entry is out of range
+    auto row_place = [&](int64_t& p, int64_t& base, int& len, bool& bad) {
+      if constexpr (PART == kFromRuns) {
+        if (p < 0 || p >= (int64_t)a.R * a.Kr) { bad = true; p = 0; }
+        p *= m;
+        base = p;
+        len = bad ? 0 : min(max(a.row_len[(int64_t)b * a.R * a.Kr + p / m], 0), m);
+      } else {
+        if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
+        base = p + n_win;
+        const int64_t rem = n_tokens - base;
+        len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+      }
+    };
     int64_t p_next = 0, pp_next = 0;
-    if (tid < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid));
-    if (lane == 0 && tid > 0 && tid <= Kp)
-      pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, tid - 1));
+    if (tid < Kp) p_next = row_entry(tid);
+    if (lane == 0 && tid > 0 && tid <= Kp) pp_next = row_entry(tid - 1);
     for (int it = 0; it < niter; ++it) {
       const int jbase = it * NT + warp * 32;
       const int j = jbase + lane;
       int64_t p = p_next;
       int64_t pp = pp_next;
-      if (j + NT < Kp) p_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT));
-      if (lane == 0 && j + NT <= Kp)
-        pp_next = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j + NT - 1));
+      if (j + NT < Kp) p_next = row_entry(j + NT);
+      if (lane == 0 && j + NT <= Kp) pp_next = row_entry(j + NT - 1);
       if (jbase >= Kp) continue;   // warp-uniform
       const bool valid = j < Kp;
       bool bad = false;
       int len = 0;
       int64_t base = 0;
       if (valid) {
-        if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
+        row_place(p, base, len, bad);
         if (j < a.pcache_rows) pcache[j] = p;
-        base = p + n_win;
-        const int64_t rem = n_tokens - base;
-        len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
       }
       int plen = __shfl_up_sync(kFull, len, 1);
       if (lane == 0) {
         plen = 0;
         int64_t pbase = 0;
-        if (j > 0) {                 // the row before this warp's rows belongs to another warp
-          if (pp < 0 || pp >= n_tokens) { bad = true; pp = 0; }
-          pbase = pp + n_win;
-          const int64_t rem = n_tokens - pbase;
-          plen = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
-        }
+        if (j > 0) row_place(pp, pbase, plen, bad);   // the row before belongs to another warp
         sb[0] = pbase; sl[0] = plen; slim[0] = 0;
       }
       const int lim = min(len, plen);
@@ -579,7 +664,7 @@ rest_draft_kernel(DraftArgs a) {
         if (i < nload) {
           const uint32_t f = (uint32_t)(i * 32 + lane);
           const uint32_t r = (f * magic) >> 16, c = f - r * (uint32_t)m;
-          if (r < 33u && (int)c < sl[r]) vals[i] = (uint32_t)__ldg(T + sb[r] + c);
+          if (r < 33u && (int)c < sl[r]) vals[i] = (uint32_t)__ldg(Trow + sb[r] + c);
         }
       }
       uint32_t my_eq = 0, my_lt = 0;         // lane i keeps the bit strings of load i
@@ -864,10 +949,12 @@ rest_draft_kernel(DraftArgs a) {
       if (par < 0) { atomicOr(&s.err, REST_CTX_INTERNAL); par = -1; }
     }
     s.par[i] = par;
-    const int64_t p = j < a.pcache_rows ? (int64_t)pcache[j]
-                                        : (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
+    int64_t p;
+    if (j < a.pcache_rows) p = (int64_t)pcache[j];
+    else if constexpr (PART == kFromRuns) p = (int64_t)a.order[(int64_t)b * a.kcap + j] * m;
+    else p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
     int64_t o = (int64_t)b * N + i;
-    a.tokens[o] = __ldg(T + p + n_win + d - 1);
+    a.tokens[o] = __ldg(Trow + p + n_win + d - 1);
     a.parents[o] = par;
     a.depth[o] = d;
     a.pos_ids[o] = clen + d - 1;
@@ -901,9 +988,8 @@ rest_draft_kernel(DraftArgs a) {
   if (tid == 0) {
     a.status[b] = 0;
     a.n_nodes[b] = nn;
-    a.match_n[b] = n_win;
-    a.match_range[2 * b] = lo;
-    a.match_range[2 * b + 1] = hi;
+    if (a.match_n) a.match_n[b] = n_win;
+    if (a.match_range) { a.match_range[2 * b] = lo; a.match_range[2 * b + 1] = hi; }
   }
 }
 
@@ -979,7 +1065,7 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     return REST_UNSUPPORTED;
 
   DraftArgs a;
-  a.T = ds->v.tokens; a.sa = ds->v.sa; a.n_tokens = ds->v.n_tokens; a.vocab = ds->v.vocab;
+  a.T = ds->v.tokens; a.sa = ds->v.sa; a.n_tokens = ds->v.n_tokens; a.n_sa = ds->v.n_sa; a.vocab = ds->v.vocab;
   a.n_max = prm->n_max; a.n_min = prm->n_min; a.K = prm->K; a.m = prm->m; a.N = prm->N;
   a.sample_mode = sample_mode;
   a.ctx = d_ctx; a.ctx_stride = ctx_stride; a.ctx_len = d_ctx_len;
@@ -1053,4 +1139,151 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     }
   }
   return rc;
+}
+
+// ---------------------------------------------------------------------------------------
+// The draft in pieces, for a datastore that is spread over several GPUs: every GPU searches
+// its own shard (rest_retrieve), the shards agree on the winning suffix length and on how many
+// candidates each contributes (a few collectives, the caller's business), every GPU reads its
+// share of the candidate rows (rest_gather_rows), the rows travel, and the tree is built from
+// the runs of all shards (rest_draft_from_runs).
+// ---------------------------------------------------------------------------------------
+namespace {
+
+// One block per context: candidate j < take[b] of the matched range is slot lo + j when the
+// whole range is taken, else lo + floor(j * cnt / take[b]); its up to m tokens and its length.
+template <typename SaT>
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const int32_t* __restrict__ T, const SaT* __restrict__ sa, int64_t n_tokens, int64_t n_sa,
+                   int m, int sample_mode, const int32_t* __restrict__ match_n,
+                   const int64_t* __restrict__ match_range, const int32_t* __restrict__ take, int Kr,
+                   int32_t* __restrict__ rows, int32_t* __restrict__ row_len, int32_t* __restrict__ status) {
+  const int b = blockIdx.x;
+  const int n = match_n[b];
+  int64_t lo = match_range[2 * b], hi = match_range[2 * b + 1];
+  lo = lo < 0 ? 0 : (lo > n_sa ? n_sa : lo);
+  hi = hi < lo ? lo : (hi > n_sa ? n_sa : hi);
+  const int64_t cnt = hi - lo;
+  int k = take[b];
+  k = k < 0 ? 0 : (k > Kr ? Kr : k);
+  if ((int64_t)k > cnt) k = (int)cnt;
+  if (n <= 0) k = 0;
+  bool bad = false;
+  for (int j = threadIdx.x; j < Kr; j += blockDim.x) {
+    int32_t* out = rows + ((int64_t)b * Kr + j) * m;
+    int len = 0;
+    if (j < k) {
+      const int64_t slot = sample_slot(lo, cnt, k, sample_mode, j);
+      const int64_t p = (int64_t)__ldg(sa + slot);
+      if (p < 0 || p >= n_tokens) {
+        bad = true;
+      } else {
+        const int64_t rem = n_tokens - (p + n);
+        len = (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+        for (int d = 0; d < len; ++d) out[d] = __ldg(T + p + n + d);
+      }
+    }
+    for (int d = len; d < m; ++d) out[d] = 0;
+    row_len[(int64_t)b * Kr + j] = len;
+  }
+  if (bad) atomicOr(status + b, REST_CTX_BAD_DATASTORE);
+}
+
+}  // namespace
+
+extern "C" rest_status rest_retrieve(const rest_datastore* ds, const rest_draft_params* prm,
+                                     const int32_t* d_ctx, int64_t ctx_stride, const int32_t* d_ctx_len,
+                                     int32_t B, int32_t* d_match_n, int64_t* d_match_range,
+                                     int32_t* d_status, void* stream) {
+  if (!ds || !prm || B < 0) return REST_INVALID_ARG;
+  if (B == 0) return REST_OK;
+  if (!d_ctx || !d_ctx_len || !d_match_n || !d_match_range || !d_status || ctx_stride < 0) return REST_INVALID_ARG;
+  if (prm->n_min < 1 || prm->n_max < prm->n_min) return REST_INVALID_ARG;
+  if (prm->n_max > REST_MAX_SUFFIX || prm->n_max - prm->n_min + 1 > kWarps) return REST_UNSUPPORTED;
+  DraftArgs a = {};
+  a.T = ds->v.tokens; a.sa = ds->v.sa; a.n_tokens = ds->v.n_tokens; a.n_sa = ds->v.n_sa; a.vocab = ds->v.vocab;
+  a.idx = ds->v.idx;
+  a.n_max = prm->n_max; a.n_min = prm->n_min; a.K = 1; a.m = 1; a.N = 1; a.sample_mode = 0;
+  a.ctx = d_ctx; a.ctx_stride = ctx_stride; a.ctx_len = d_ctx_len;
+  a.match_n = d_match_n; a.match_range = d_match_range; a.status = d_status; a.B = B;
+  const bool narrow = ds->v.sa_bytes == 4;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (narrow) rest_draft_kernel<int32_t, false, kThreads, kRetrieve><<<B, kThreads, sizeof(Smem), st>>>(a);
+  else rest_draft_kernel<int64_t, false, kThreads, kRetrieve><<<B, kThreads, sizeof(Smem), st>>>(a);
+  rest::count_launch();
+  REST_CUDA_TRY(cudaGetLastError());
+  return REST_OK;
+}
+
+extern "C" rest_status rest_gather_rows(const rest_datastore* ds, const rest_draft_params* prm,
+                                        const int32_t* d_match_n, const int64_t* d_match_range,
+                                        const int32_t* d_take, int32_t B, int32_t Kr, int32_t* d_rows,
+                                        int32_t* d_row_len, int32_t* d_status, void* stream) {
+  if (!ds || !prm || B < 0 || Kr < 1) return REST_INVALID_ARG;
+  if (B == 0) return REST_OK;
+  if (!d_match_n || !d_match_range || !d_take || !d_rows || !d_row_len || !d_status) return REST_INVALID_ARG;
+  if (prm->m < 1) return REST_INVALID_ARG;
+  if (prm->m > REST_MAX_M || Kr > REST_MAX_K) return REST_UNSUPPORTED;
+  if (prm->sample_mode != REST_SAMPLE_STRIDED && prm->sample_mode != REST_SAMPLE_FIRST_K) return REST_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (ds->v.sa_bytes == 4)
+    gather_rows_kernel<int32_t><<<B, 256, 0, st>>>(ds->v.tokens, static_cast<const int32_t*>(ds->v.sa),
+                                                   ds->v.n_tokens, ds->v.n_sa, prm->m, prm->sample_mode, d_match_n,
+                                                   d_match_range, d_take, Kr, d_rows, d_row_len, d_status);
+  else
+    gather_rows_kernel<int64_t><<<B, 256, 0, st>>>(ds->v.tokens, static_cast<const int64_t*>(ds->v.sa),
+                                                   ds->v.n_tokens, ds->v.n_sa, prm->m, prm->sample_mode, d_match_n,
+                                                   d_match_range, d_take, Kr, d_rows, d_row_len, d_status);
+  rest::count_launch();
+  REST_CUDA_TRY(cudaGetLastError());
+  return REST_OK;
+}
+
+extern "C" size_t rest_draft_from_runs_workspace_bytes(int32_t B, int32_t R, int32_t Kr) {
+  if (B <= 0 || R <= 0 || Kr <= 0) return 0;
+  const size_t kcap = ((size_t)R * Kr + 31) / 32 * 32;
+  return (size_t)B * kcap * sizeof(uint32_t);
+}
+
+extern "C" rest_status rest_draft_from_runs(const rest_draft_params* prm, const int32_t* d_rows,
+                                            const int32_t* d_row_len, const int32_t* d_run_rows, int32_t R,
+                                            int32_t Kr, const int32_t* d_ctx_len, int32_t B,
+                                            int32_t* d_tokens, int32_t* d_parents, int32_t* d_depth,
+                                            int32_t* d_pos_ids, uint32_t* d_mask, int32_t* d_n_nodes,
+                                            int32_t* d_node_count, int32_t* d_status, void* d_ws,
+                                            size_t ws_bytes, void* stream) {
+  if (!prm || B < 0 || R < 1 || Kr < 1) return REST_INVALID_ARG;
+  if (B == 0) return REST_OK;
+  if (!d_rows || !d_row_len || !d_run_rows || !d_ctx_len || !d_tokens || !d_parents || !d_depth ||
+      !d_pos_ids || !d_mask || !d_n_nodes || !d_status)
+    return REST_INVALID_ARG;
+  if (prm->m < 1 || prm->N < 1) return REST_INVALID_ARG;
+  if (prm->m > REST_MAX_M || prm->N > REST_MAX_N || (int64_t)R * Kr > REST_MAX_K) return REST_UNSUPPORTED;
+  const size_t need = rest_draft_from_runs_workspace_bytes(B, R, Kr);
+  if (!d_ws) return REST_INVALID_ARG;
+  if (ws_bytes < need) return REST_WORKSPACE_TOO_SMALL;
+  DraftArgs a = {};
+  a.T = d_rows; a.row_len = d_row_len; a.run_rows = d_run_rows; a.R = R; a.Kr = Kr;
+  a.order = static_cast<uint32_t*>(d_ws);
+  a.n_tokens = (int64_t)B * R * Kr * prm->m; a.n_sa = a.n_tokens; a.vocab = 0x7FFFFFFFu;
+  a.n_max = 0; a.n_min = 0; a.K = R * Kr; a.m = prm->m; a.N = prm->N; a.sample_mode = 0;
+  a.ctx_len = d_ctx_len;
+  a.tokens = d_tokens; a.parents = d_parents; a.depth = d_depth; a.pos_ids = d_pos_ids; a.mask = d_mask;
+  a.n_nodes = d_n_nodes; a.node_count = d_node_count; a.status = d_status; a.B = B;
+  const bool big = (size_t)a.K * prm->m >= kBigRowsTimesM;
+  const int threads = big ? kBigThreads : kThreads;
+  const size_t smem = draft_smem_bytes(a.K, prm->m, threads, &a.kcap, &a.nwords, &a.pcache_rows);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (big) {
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(rest_draft_kernel<int32_t, false, kBigThreads, kFromRuns>),
+                                            rest::kSmemSlotDraft + 15, smem));
+    rest_draft_kernel<int32_t, false, kBigThreads, kFromRuns><<<B, kBigThreads, smem, st>>>(a);
+  } else {
+    REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(rest_draft_kernel<int32_t, false, kThreads, kFromRuns>),
+                                            rest::kSmemSlotDraft + 14, smem));
+    rest_draft_kernel<int32_t, false, kThreads, kFromRuns><<<B, kThreads, smem, st>>>(a);
+  }
+  rest::count_launch();
+  REST_CUDA_TRY(cudaGetLastError());
+  return REST_OK;
 }

@@ -11,6 +11,7 @@ import torch.distributed as dist
 import torch.multiprocessing as mp
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 from paper_2311_08252_b200.sharding import max_over_ranks, shard_bounds, whole_job_throughput
 
@@ -61,3 +62,112 @@ def test_two_ranks_gloo(tmp_path):
         port = s.getsockname()[1]
     mp.spawn(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True)
     assert open(tmp_path / "ok").read() == "1"
+
+
+# ---------------------------------------------------------------------------------------
+# A datastore spread over the ranks: the exchange logic of sharded_draft over gloo, with each
+# rank's compute steps done by plain scanning stand-ins (tests/sharded_util.py).
+# ---------------------------------------------------------------------------------------
+def _sharded_case():
+    rng = np.random.default_rng(5)
+    vocab, n_tok, B, Lc = 3, 2400, 24, 12
+    T = rng.integers(0, vocab, n_tok).astype(np.int32)
+    ctx = rng.integers(0, vocab, (B, Lc)).astype(np.int32)
+    for b in range(0, B, 2):
+        p = int(rng.integers(0, n_tok - Lc))
+        ctx[b] = T[p:p + Lc]
+    ctx[1] = T[1200 - 6:1200 + 6]            # a match that straddles the cut between the two shards
+    ctx_len = np.full(B, Lc, np.int32)
+    ctx_len[3] = 1                           # shorter than n_min: no tree
+    return vocab, T, ctx, ctx_len
+
+
+def _sharded_worker(rank, world, port, out_dir, K, n_max):
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import sharded_util as su
+    from paper_2311_08252_b200.sharding import SHARD_HALO, TorchComm, shard_tokens, sharded_draft
+    vocab, T, ctx, ctx_len = _sharded_case()
+    n_min, m, N = 2, 5, 24
+    ext, owned = shard_tokens(T, rank, world)
+    order = su.shard_order(ext, owned)
+    B = ctx.shape[0]
+
+    def retrieve_fn(c, cl):
+        mn, mr = np.zeros(B, np.int32), np.zeros((B, 2), np.int64)
+        for b in range(B):
+            mn[b], mr[b, 0], mr[b, 1] = su.shard_retrieve(ext, order, c[b, :cl[b]].numpy(), n_max, n_min)
+        return torch.from_numpy(mn), torch.from_numpy(mr), torch.zeros(B, dtype=torch.int32)
+
+    def gather_fn(mn, mr, take, Kr):
+        rows, lens = np.zeros((B, Kr, m), np.int32), np.zeros((B, Kr), np.int32)
+        for b in range(B):
+            got = su.shard_rows(ext, order, int(mn[b]), int(mr[b, 0]), int(mr[b, 1]), int(take[b]), m)
+            for j, r in enumerate(got):
+                rows[b, j, :len(r)] = r
+                lens[b, j] = len(r)
+        return torch.from_numpy(rows), torch.from_numpy(lens), torch.zeros(B, dtype=torch.int32)
+
+    def build_fn(rows, lens, runs, cl):
+        trees = []
+        for b in range(B):
+            flat = [rows[b, r, j, :lens[b, r, j]].tolist() for r in range(world) for j in range(int(runs[b, r]))]
+            trees.append(su.tree_from_rows(flat, N, int(cl[b])))
+        return trees
+
+    trees, info = sharded_draft(TorchComm(dist), retrieve_fn, gather_fn, build_fn,
+                                torch.from_numpy(ctx), torch.from_numpy(ctx_len), K)
+    if rank == 0:
+        import oracle
+        want, want_info = su.sharded_reference(T, world, SHARD_HALO, ctx, ctx_len, n_max, n_min, K, m, N)
+        ok = True
+        for b in range(B):
+            ok = ok and int(info["match_n"][b]) == want_info[b][0] and int(info["hits"][b]) == want_info[b][1]
+            ok = ok and info["taken"][:, b].tolist() == want_info[b][2]
+            for key in ("tokens", "parents", "depth", "pos_ids", "node_count", "mask", "n_nodes"):
+                ok = ok and np.array_equal(trees[b][key], want[b][key])
+        # where the cap does not bind the sharded draft is the draft over the whole datastore
+        full = oracle.draft(T, oracle.suffix_array(T), vocab, ctx, ctx_len, n_max=n_max, n_min=n_min, K=K, m=m, N=N)
+        free = [b for b in range(B) if want_info[b][1] <= K]
+        ok = ok and len(free) >= (B // 2 if K >= 2400 else 1)
+        binds = [b for b in range(B) if want_info[b][1] > K]
+        for b in free:
+            ok = ok and int(info["match_n"][b]) == int(full["match_n"][b])
+            ok = ok and int(info["hits"][b]) == int(full["match_range"][b, 1] - full["match_range"][b, 0])
+            for key in ("tokens", "parents", "depth", "pos_ids", "node_count", "mask"):
+                ok = ok and np.array_equal(trees[b][key], full[key][b])
+            ok = ok and trees[b]["n_nodes"] == int(full["n_nodes"][b])
+        ok = ok and (len(binds) >= B // 2) == (K < 2400)
+        open(os.path.join(out_dir, "ok"), "w").write("1" if ok else "0")
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("K,n_max", [(5000, 8), (40, 3)])
+def test_sharded_datastore_two_ranks_gloo(tmp_path, K, n_max):
+    """K = 5000 never binds on this datastore: the trees must be those of the oracle over the
+    whole stream.  K = 40 with suffixes of at most three tokens binds for most contexts (every
+    trigram occurs about ninety times): the trees must be those of the sharded definition
+    (rows per shard in proportion to its hits) computed directly."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_sharded_worker, args=(2, port, str(tmp_path), K, n_max), nprocs=2, join=True)
+    assert open(tmp_path / "ok").read() == "1"
+
+
+def test_allocate_rows_sums_to_the_cap_and_reduces_to_one_shard():
+    from paper_2311_08252_b200.sharding import allocate_rows
+    import sharded_util as su
+    rng = np.random.default_rng(2)
+    for _ in range(200):
+        world, K = int(rng.integers(1, 6)), int(rng.integers(1, 60))
+        cnt = rng.integers(0, 80, (world, 7))
+        cnt[:, 0] = 0
+        got = allocate_rows(torch.from_numpy(cnt), K).numpy()
+        for b in range(7):
+            assert got[:, b].tolist() == su.allocation(cnt[:, b].tolist(), K)
+            assert got[:, b].sum() == min(K, cnt[:, b].sum())
+            assert (got[:, b] <= cnt[:, b]).all()
+    assert allocate_rows(torch.tensor([[123456789012]]), 5000).item() == 5000
