@@ -341,14 +341,30 @@ rest_status rest_kv_commit(void* d_k, void* d_v, const int64_t* kv_strides, cons
  *   n_max + m <= 32 tokens of a suffix, so its results are those of the full order.
  *
  *   d_tokens  int32[n_tokens] device, values in [0, 2^31 - 1)
- *   sa_bytes  4 or 8: d_sa is int32[n_tokens] or int64[n_tokens] (device, written)
- *   d_ws      device scratch of rest_suffix_array_workspace_bytes(n_tokens) bytes (about
- *             32 bytes per token + 64 MiB), 256-byte aligned
- *   Limits: n_tokens <= 2^31 - 1 (REST_UNSUPPORTED beyond).  Asynchronous on `stream`.
+ *   sa_bytes  4 or 8: d_sa is int32[n_tokens] (n_tokens < 2^31) or int64[n_tokens] (device, written)
+ *   d_ws      device scratch, 256-byte aligned.  Two methods, picked by what fits:
+ *             - up to 2^31 - 1 tokens and at least rest_suffix_array_workspace_bytes(n_tokens)
+ *               (about 32 bytes per token + 64 MiB): prefix doubling, five sorts of the whole
+ *               stream, asynchronous on `stream`;
+ *             - otherwise (longer streams, or a smaller workspace): positions are put into
+ *               buckets by first token and groups of whole buckets are sorted one after the
+ *               other on their packed 32-token keys.  Scratch: 32 bytes per position of the
+ *               largest group + 0.2 GiB; rest_suffix_array_workspace_bytes answers for groups of
+ *               2^30 positions, rest_suffix_array_min_workspace_bytes for groups just large
+ *               enough for the most frequent first token.  This method reads the bucket
+ *               histogram back (it synchronises `stream`) and returns REST_UNSUPPORTED when one
+ *               first token starts more suffixes than the workspace can sort at once.
+ *   Limits: n_tokens <= 2^40.
  */
 size_t rest_suffix_array_workspace_bytes(uint64_t n_tokens);
+size_t rest_suffix_array_min_workspace_bytes(uint64_t n_tokens, uint64_t largest_bucket);
 rest_status rest_suffix_array_build(const int32_t* d_tokens, uint64_t n_tokens, int32_t sa_bytes,
                                     void* d_sa, void* d_ws, size_t ws_bytes, void* stream);
+/* The second method whatever the size: groups of at most max_group positions (0: as many as the
+ * workspace allows; at least the count of the most frequent first token). */
+rest_status rest_suffix_array_build_in_groups(const int32_t* d_tokens, uint64_t n_tokens,
+                                              int32_t sa_bytes, void* d_sa, uint64_t max_group,
+                                              void* d_ws, size_t ws_bytes, void* stream);
 
 /*
  * Device-side trouble that no per-call status can carry.  Every wait inside the kernels is

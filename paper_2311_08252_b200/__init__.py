@@ -35,7 +35,8 @@ EXPORTS = (
     "rest_tree_attention_workspace_bytes", "rest_tree_attention",
     "rest_tree_attention_static_scratch",
     "rest_device_error_flags", "rest_kv_commit", "rest_probe_dependent_reads",
-    "rest_suffix_array_workspace_bytes", "rest_suffix_array_build", "rest_tree_attention_plan",
+    "rest_suffix_array_workspace_bytes", "rest_suffix_array_min_workspace_bytes",
+    "rest_suffix_array_build", "rest_suffix_array_build_in_groups", "rest_tree_attention_plan",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -105,8 +106,12 @@ def lib():
     L.rest_kv_commit.argtypes = [vp, vp, ctypes.POINTER(i64), vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
     L.rest_suffix_array_workspace_bytes.restype = sz
     L.rest_suffix_array_workspace_bytes.argtypes = [u64]
+    L.rest_suffix_array_min_workspace_bytes.restype = sz
+    L.rest_suffix_array_min_workspace_bytes.argtypes = [u64, u64]
     L.rest_suffix_array_build.restype = i32
     L.rest_suffix_array_build.argtypes = [vp, u64, i32, vp, vp, sz, vp]
+    L.rest_suffix_array_build_in_groups.restype = i32
+    L.rest_suffix_array_build_in_groups.argtypes = [vp, u64, i32, vp, u64, vp, sz, vp]
     L.rest_tree_attention_plan.restype = i32
     L.rest_tree_attention_plan.argtypes = [i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
     L.rest_probe_dependent_reads.restype = i32
@@ -466,20 +471,30 @@ def dependent_read_latency_ns(table_bytes: int = 1 << 30, steps: int = 4096, dev
     return best
 
 
-def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None):
+def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None, max_group: int | None = None):
     """Suffix array of the int32 CUDA tensor `tokens`, built on the device and ordered on the
-    first 32 tokens of each suffix (ties by position).  Returns an int32 or int64 CUDA tensor."""
+    first 32 tokens of each suffix (ties by position).  Returns an int32 or int64 CUDA tensor.
+    max_group: sort the stream in groups of first-token buckets of at most that many positions
+    (the method for streams beyond 2^31 - 1 tokens), whatever its size."""
     import torch
     L = lib()
     _dev_i32(tokens, "tokens")
     n = tokens.numel()
     sa = torch.empty(n, dtype=torch.int32 if sa_bytes == 4 else torch.int64, device=tokens.device)
-    ws_bytes = L.rest_suffix_array_workspace_bytes(n)
+    if max_group is None:
+        ws_bytes = L.rest_suffix_array_workspace_bytes(n)
+    else:
+        ws_bytes = L.rest_suffix_array_min_workspace_bytes(n, int(max_group))
     if ws_bytes == 0:
-        raise RestError("rest_suffix_array_build: between 1 and 2^31 - 1 tokens are supported")
+        raise RestError("rest_suffix_array_build: between 1 and 2^40 tokens are supported")
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=tokens.device)
-    _check(L.rest_suffix_array_build(tokens.data_ptr(), n, sa_bytes, sa.data_ptr(), ws.data_ptr(),
-                                     ws_bytes, _stream(stream)), "rest_suffix_array_build")
+    if max_group is None:
+        rc = L.rest_suffix_array_build(tokens.data_ptr(), n, sa_bytes, sa.data_ptr(), ws.data_ptr(),
+                                       ws_bytes, _stream(stream))
+    else:
+        rc = L.rest_suffix_array_build_in_groups(tokens.data_ptr(), n, sa_bytes, sa.data_ptr(), int(max_group),
+                                                 ws.data_ptr(), ws_bytes, _stream(stream))
+    _check(rc, "rest_suffix_array_build")
     # set-up call: wait here, so that the scratch can be released whatever stream was used
     torch.cuda.synchronize(tokens.device)
     return sa

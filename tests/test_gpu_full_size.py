@@ -112,3 +112,43 @@ def test_draft_largest_datastores(name, n_tokens):
     ds.close()
     del d_T, d_sa, ds
     torch.cuda.empty_cache()
+
+
+def test_draft_large_workload_at_its_full_size():
+    """The large workload as stated: 4 B tokens, int64 suffix array (32 GB) built on the device
+    in groups of first-token buckets, positions beyond 2^31 in the matched ranges."""
+    w = datagen.WORKLOADS["large"]
+    n = w.n_tokens
+    need_dev = n * 12 + rest.lib().rest_suffix_array_workspace_bytes(n) + rest.lib().rest_datastore_aux_bytes(n, 8, w.vocab)
+    free, _ = torch.cuda.mem_get_info()
+    if free < need_dev + (4 << 30):
+        pytest.skip(f"needs {need_dev / 2**30:.0f} GiB of device memory, {free / 2**30:.0f} GiB free")
+    need_host = n * 12 * 2
+    if host_memory_available() < need_host + (8 << 30):
+        pytest.skip(f"needs {need_host / 2**30:.0f} GiB of host memory, "
+                    f"{host_memory_available() / 2**30:.0f} GiB available")
+    T = datagen.make_tokens(w)
+    d_T = to_dev(T)
+    d_sa = rest.rest_suffix_array_build(d_T, 8)
+    torch.cuda.empty_cache()
+    ds = rest.Datastore(d_T, d_sa, w.vocab, validate=True)
+    sa = d_sa.cpu().numpy()
+    B, Lc = w.B, 64
+    ctx = datagen.make_contexts(w, T, B=B, Lc=Lc)
+    ctx_len = np.full(B, Lc, np.int32)
+    kw = dict(K=w.K, m=w.m, N=w.N)
+    ref = oracle.draft(T, sa, w.vocab, ctx, ctx_len, **kw)
+    for search in (rest.REST_SEARCH_SINGLE, rest.REST_SEARCH_BATCHED):
+        out = rest.rest_draft(ds, to_dev(ctx), to_dev(ctx_len), search=search, **kw)
+        torch.cuda.synchronize()
+        got = {k: getattr(out, k).cpu().numpy() for k in DRAFT_KEYS}
+        got["mask"] = out.mask.cpu().numpy().view(np.uint32)
+        assert_draft_equal(got, ref, f"large, {n} tokens, search {search}")
+    assert (ref["n_nodes"] > 0).mean() > 0.5
+    # the matched ranges reach suffix-array slots and token positions that need 64 bits
+    assert ref["match_range"].max() > 2**31
+    high = [int(sa[int(lo):int(min(hi, lo + 5000))].max()) for lo, hi in ref["match_range"] if hi > lo]
+    assert max(high) > 2**31
+    ds.close()
+    del d_T, d_sa, ds
+    torch.cuda.empty_cache()

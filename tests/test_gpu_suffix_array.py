@@ -64,10 +64,48 @@ def test_workload_recipes_and_drafts_on_the_device_built_array(name):
     assert (ref["n_nodes"] > 0).mean() > 0.5
 
 
+def largest_first_token_bucket(T):
+    return int(np.unique(T, return_counts=True)[1].max())
+
+
+@pytest.mark.parametrize("case", ["single_stream", "large", "vocab50", "tokens_up_to_2^31", "constant", "binary"])
+def test_bucket_method_gives_the_same_array_as_prefix_doubling(case):
+    """The builder's second method (groups of first-token buckets sorted on their packed
+    32-token keys; what streams beyond 2^31 - 1 tokens get) must give the very same array."""
+    rng = np.random.default_rng(11)
+    sa_bytes = 4
+    if case in ("single_stream", "large"):
+        w = datagen.WORKLOADS[case].scaled(n_tokens=1_200_000)
+        T, sa_bytes = datagen.make_tokens(w), w.sa_bytes
+    elif case == "vocab50":
+        T = rng.integers(0, 50, 300_000).astype(np.int32)
+    elif case == "tokens_up_to_2^31":
+        T = rng.integers(0, 2**31 - 2, 40_000).astype(np.int32)      # 31-bit tokens: two per key word
+        T[::7] = T[3]                                                 # and some repetition
+    elif case == "constant":
+        T = np.full(5000, 3, np.int32)
+    else:
+        T = rng.integers(0, 2, 50_000).astype(np.int32)
+    d_T = to_dev(T)
+    want = rest.rest_suffix_array_build(d_T, sa_bytes)
+    biggest = largest_first_token_bucket(T)
+    got = rest.rest_suffix_array_build(d_T, sa_bytes, max_group=max(biggest, 1024))
+    assert got.dtype == want.dtype and torch.equal(got, want)
+    if case in ("single_stream", "vocab50"):
+        assert len(T) > 4 * max(biggest, 1024)        # several groups were sorted
+    if case == "vocab50":
+        # groups too small for the most frequent first token are refused
+        with pytest.raises(rest.RestError, match="unsupported"):
+            rest.rest_suffix_array_build(d_T, sa_bytes, max_group=1024)
+
+
 def test_argument_checks():
     L = rest.lib()
     assert L.rest_suffix_array_workspace_bytes(0) == 0
-    assert L.rest_suffix_array_workspace_bytes(1 << 31) == 0
+    assert L.rest_suffix_array_workspace_bytes((1 << 40) + 1) == 0
+    # beyond 2^31 - 1 tokens the recommended scratch is that of groups of 2^30 positions
+    assert 32 << 30 < L.rest_suffix_array_workspace_bytes(1 << 32) < 33 << 30
     assert L.rest_suffix_array_build(256, 10, 5, 256, 256, 1 << 30, None) == 1
     assert L.rest_suffix_array_build(256, 10, 4, 256, 256, 16, None) == 3
-    assert L.rest_suffix_array_build(256, 1 << 31, 4, 256, 256, 1 << 30, None) == 2
+    assert L.rest_suffix_array_build(256, 1 << 31, 4, 256, 256, 1 << 30, None) == 1     # needs 64-bit entries
+    assert L.rest_suffix_array_build(256, (1 << 40) + 1, 8, 256, 256, 1 << 30, None) == 2
