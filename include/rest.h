@@ -2,7 +2,8 @@
  * rest.h - C ABI of the GPU hot path of one REST decoding step
  * (Retrieval-Based Speculative Decoding, arXiv 2311.08252).
  *
- * Set-up:       rest_suffix_array_build, rest_datastore_create  (Sec. 3.2, datastore construction)
+ * Set-up:       rest_suffix_array_build (_full, _in_groups, _append), rest_datastore_create
+ *               (Sec. 3.2, datastore construction)
  * Draft side:   rest_draft                                 (Sec. 3.2, Algorithms 1 and 2)
  *               rest_retrieve, rest_gather_rows, rest_draft_from_runs: the same in pieces, for a
  *               datastore spread over several GPUs
@@ -360,6 +361,28 @@ size_t rest_suffix_array_workspace_bytes(uint64_t n_tokens);
 size_t rest_suffix_array_min_workspace_bytes(uint64_t n_tokens, uint64_t largest_bucket);
 rest_status rest_suffix_array_build(const int32_t* d_tokens, uint64_t n_tokens, int32_t sa_bytes,
                                     void* d_sa, void* d_ws, size_t ws_bytes, void* stream);
+/* The true suffix array (whole suffixes compared, no ties left): prefix doubling carried on
+ * past 32 tokens until every suffix is distinct, one flag read back per extra round (the call
+ * synchronises `stream`).  Streams of up to 2^31 - 1 tokens; workspace as for the first method.
+ * rest_draft gives the same results on either array; this one is for callers who want the
+ * array itself. */
+rest_status rest_suffix_array_build_full(const int32_t* d_tokens, uint64_t n_tokens, int32_t sa_bytes,
+                                         void* d_sa, void* d_ws, size_t ws_bytes, void* stream);
+/*
+ * rest_suffix_array_append - the suffix array after n_new tokens were appended to a stream of
+ * n_old tokens (Sec. 3.2 "Datastore construction": a datastore that grows).  Only the suffixes
+ * of the last 31 old positions and of the new tokens can change place under the 32-token
+ * order; they are sorted by themselves and merged into the old array in one pass.
+ *   d_tokens   int32[n_old + n_new]: the whole stream, old tokens first
+ *   d_sa_old   the array of the first n_old tokens as rest_suffix_array_build wrote it (NULL when n_old = 0)
+ *   d_sa_new   receives n_old + n_new entries of sa_bytes bytes; must not be d_sa_old
+ *   d_ws       rest_suffix_array_append_workspace_bytes(n_new) bytes (about 44 bytes per new
+ *              token + 64 MiB), 256-byte aligned.  Asynchronous on `stream`.
+ */
+size_t rest_suffix_array_append_workspace_bytes(uint64_t n_new);
+rest_status rest_suffix_array_append(const int32_t* d_tokens, uint64_t n_old, uint64_t n_new,
+                                     const void* d_sa_old, int32_t sa_bytes, void* d_sa_new,
+                                     void* d_ws, size_t ws_bytes, void* stream);
 /* The second method whatever the size: groups of at most max_group positions (0: as many as the
  * workspace allows; at least the count of the most frequent first token). */
 rest_status rest_suffix_array_build_in_groups(const int32_t* d_tokens, uint64_t n_tokens,

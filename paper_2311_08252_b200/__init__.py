@@ -36,7 +36,8 @@ EXPORTS = (
     "rest_tree_attention_static_scratch",
     "rest_device_error_flags", "rest_kv_commit", "rest_probe_dependent_reads",
     "rest_suffix_array_workspace_bytes", "rest_suffix_array_min_workspace_bytes",
-    "rest_suffix_array_build", "rest_suffix_array_build_in_groups", "rest_tree_attention_plan",
+    "rest_suffix_array_build", "rest_suffix_array_build_in_groups", "rest_suffix_array_build_full",
+    "rest_suffix_array_append_workspace_bytes", "rest_suffix_array_append", "rest_tree_attention_plan",
     "rest_accept", "rest_status_string", "rest_last_cuda_error", "rest_launch_count",
 )
 
@@ -110,6 +111,12 @@ def lib():
     L.rest_suffix_array_min_workspace_bytes.argtypes = [u64, u64]
     L.rest_suffix_array_build.restype = i32
     L.rest_suffix_array_build.argtypes = [vp, u64, i32, vp, vp, sz, vp]
+    L.rest_suffix_array_append_workspace_bytes.restype = sz
+    L.rest_suffix_array_append_workspace_bytes.argtypes = [u64]
+    L.rest_suffix_array_append.restype = i32
+    L.rest_suffix_array_append.argtypes = [vp, u64, u64, vp, i32, vp, vp, sz, vp]
+    L.rest_suffix_array_build_full.restype = i32
+    L.rest_suffix_array_build_full.argtypes = [vp, u64, i32, vp, vp, sz, vp]
     L.rest_suffix_array_build_in_groups.restype = i32
     L.rest_suffix_array_build_in_groups.argtypes = [vp, u64, i32, vp, u64, vp, sz, vp]
     L.rest_tree_attention_plan.restype = i32
@@ -471,11 +478,13 @@ def dependent_read_latency_ns(table_bytes: int = 1 << 30, steps: int = 4096, dev
     return best
 
 
-def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None, max_group: int | None = None):
+def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None, max_group: int | None = None,
+                            full: bool = False):
     """Suffix array of the int32 CUDA tensor `tokens`, built on the device and ordered on the
     first 32 tokens of each suffix (ties by position).  Returns an int32 or int64 CUDA tensor.
     max_group: sort the stream in groups of first-token buckets of at most that many positions
-    (the method for streams beyond 2^31 - 1 tokens), whatever its size."""
+    (the method for streams beyond 2^31 - 1 tokens), whatever its size.  full=True: the true
+    suffix array (whole suffixes compared) instead of the order on 32 tokens."""
     import torch
     L = lib()
     _dev_i32(tokens, "tokens")
@@ -488,7 +497,10 @@ def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None, max_group: i
     if ws_bytes == 0:
         raise RestError("rest_suffix_array_build: between 1 and 2^40 tokens are supported")
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=tokens.device)
-    if max_group is None:
+    if full:
+        rc = L.rest_suffix_array_build_full(tokens.data_ptr(), n, sa_bytes, sa.data_ptr(), ws.data_ptr(),
+                                            ws_bytes, _stream(stream))
+    elif max_group is None:
         rc = L.rest_suffix_array_build(tokens.data_ptr(), n, sa_bytes, sa.data_ptr(), ws.data_ptr(),
                                        ws_bytes, _stream(stream))
     else:
@@ -496,6 +508,25 @@ def rest_suffix_array_build(tokens, sa_bytes: int = 4, stream=None, max_group: i
                                                  ws.data_ptr(), ws_bytes, _stream(stream))
     _check(rc, "rest_suffix_array_build")
     # set-up call: wait here, so that the scratch can be released whatever stream was used
+    torch.cuda.synchronize(tokens.device)
+    return sa
+
+
+def rest_suffix_array_append(tokens, sa_old, stream=None):
+    """Suffix array of `tokens` (int32 CUDA tensor: the old stream followed by the appended
+    tokens) from the array `sa_old` of its first sa_old.numel() tokens."""
+    import torch
+    L = lib()
+    _dev_i32(tokens, "tokens")
+    n, n_old = tokens.numel(), sa_old.numel()
+    if not (sa_old.is_cuda and sa_old.dtype in (torch.int32, torch.int64) and sa_old.is_contiguous()) or n_old >= n:
+        raise RestError("sa_old must be a contiguous int32/int64 CUDA tensor shorter than tokens")
+    sa = torch.empty(n, dtype=sa_old.dtype, device=tokens.device)
+    ws_bytes = L.rest_suffix_array_append_workspace_bytes(n - n_old)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=tokens.device)
+    _check(L.rest_suffix_array_append(tokens.data_ptr(), n_old, n - n_old, _ptr(sa_old) if n_old else 0,
+                                      sa_old.element_size(), sa.data_ptr(), ws.data_ptr(), ws_bytes,
+                                      _stream(stream)), "rest_suffix_array_append")
     torch.cuda.synchronize(tokens.device)
     return sa
 

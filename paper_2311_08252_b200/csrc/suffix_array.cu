@@ -74,8 +74,15 @@ __global__ void sa_write(const uint32_t* __restrict__ vals, OutT* __restrict__ s
 
 }  // namespace
 
+__global__ void sa_any_tie(const uint64_t* __restrict__ keys, int64_t n, unsigned int* __restrict__ flag) {
+  const int64_t j = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+  if (j > 0 && j < n && keys[j] == keys[j - 1]) *flag = 1u;
+}
+
+// full = false: the order on the first 32 tokens (five rounds).  full = true: rounds go on, the
+// compared length doubling each time, until no two suffixes are tied: the true suffix array.
 static rest_status build_by_doubling(const int32_t* d_tokens, uint64_t n_tokens, int32_t sa_bytes, void* d_sa,
-                                     void* d_ws, size_t ws_bytes, void* stream) {
+                                     void* d_ws, size_t ws_bytes, void* stream, bool full = false) {
   const SaLayout l = sa_layout(n_tokens);
   if (ws_bytes < l.total) return REST_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -96,28 +103,40 @@ static rest_status build_by_doubling(const int32_t* d_tokens, uint64_t n_tokens,
     size_t need_sort = 0, need_scan = 0;
     REST_CUDA_TRY(cub::DeviceRadixSort::SortPairs(nullptr, need_sort, dk, dv, n, 0, 64, st));
     REST_CUDA_TRY(cub::DeviceScan::InclusiveScan(nullptr, need_scan, head, head, cub::Max(), n, st));
-    if (need_sort > temp_bytes || need_scan > temp_bytes) return REST_WORKSPACE_TOO_SMALL;
+    if (need_sort > temp_bytes - kAlign || need_scan > temp_bytes - kAlign) return REST_WORKSPACE_TOO_SMALL;
   }
 
   sa_init_rank<<<blocks, kBlock, 0, st>>>(d_tokens, rank, n);
   rest::count_launch();
   const uint32_t* result = nullptr;
-  for (int64_t h = 1; h <= 16; h *= 2) {
+  unsigned int* d_tie = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(temp) + temp_bytes - kAlign);
+  for (int64_t h = 1; h < ((int64_t)1 << 31); h *= 2) {
     sa_make_keys<<<blocks, kBlock, 0, st>>>(rank, keys[0], vals[0], n, h);
     cub::DoubleBuffer<uint64_t> dk(keys[0], keys[1]);
     cub::DoubleBuffer<uint32_t> dv(vals[0], vals[1]);
-    size_t tb = temp_bytes;
+    size_t tb = temp_bytes - kAlign;
     // ranks never exceed n <= 2^31 - 1 and tokens stay below 2^31: bit 63 and bit 31 are unused
     REST_CUDA_TRY(cub::DeviceRadixSort::SortPairs(temp, tb, dk, dv, n, 0, 64, st));
     result = dv.Current();
     rest::count_launch(2);
-    if (h < 16) {
-      sa_mark_heads<<<blocks, kBlock, 0, st>>>(dk.Current(), head, n);
-      tb = temp_bytes;
-      REST_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, tb, head, head, cub::Max(), n, st));
-      sa_scatter_rank<<<blocks, kBlock, 0, st>>>(dv.Current(), head, rank, n);
-      rest::count_launch(3);
+    bool last = !full && h == 16;
+    if (full && h >= 16) {
+      // the true suffix array is reached when no two suffixes compare equal any more (at the
+      // latest when the compared length exceeds the stream); one flag read back per round
+      unsigned int tie = 0;
+      REST_CUDA_TRY(cudaMemsetAsync(d_tie, 0, sizeof(unsigned int), st));
+      sa_any_tie<<<blocks, kBlock, 0, st>>>(dk.Current(), n, d_tie);
+      rest::count_launch();
+      REST_CUDA_TRY(cudaMemcpyAsync(&tie, d_tie, sizeof(tie), cudaMemcpyDeviceToHost, st));
+      REST_CUDA_TRY(cudaStreamSynchronize(st));
+      last = tie == 0 || 2 * h > n;
     }
+    if (last) break;
+    sa_mark_heads<<<blocks, kBlock, 0, st>>>(dk.Current(), head, n);
+    tb = temp_bytes - kAlign;
+    REST_CUDA_TRY(cub::DeviceScan::InclusiveScan(temp, tb, head, head, cub::Max(), n, st));
+    sa_scatter_rank<<<blocks, kBlock, 0, st>>>(dv.Current(), head, rank, n);
+    rest::count_launch(3);
   }
   if (sa_bytes == 4)
     sa_write<int32_t><<<blocks, kBlock, 0, st>>>(result, static_cast<int32_t*>(d_sa), n);
@@ -359,6 +378,16 @@ extern "C" rest_status rest_suffix_array_build(const int32_t* d_tokens, uint64_t
   return rest_suffix_array_build_in_groups(d_tokens, n_tokens, sa_bytes, d_sa, 0, d_ws, ws_bytes, stream);
 }
 
+extern "C" rest_status rest_suffix_array_build_full(const int32_t* d_tokens, uint64_t n_tokens,
+                                                    int32_t sa_bytes, void* d_sa, void* d_ws,
+                                                    size_t ws_bytes, void* stream) {
+  if (!d_tokens || !d_sa || !d_ws || n_tokens == 0) return REST_INVALID_ARG;
+  if (sa_bytes != 4 && sa_bytes != 8) return REST_INVALID_ARG;
+  if (n_tokens > 0x7FFFFFFFull) return REST_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(d_ws) & (kAlign - 1)) return REST_INVALID_ARG;
+  return build_by_doubling(d_tokens, n_tokens, sa_bytes, d_sa, d_ws, ws_bytes, stream, true);
+}
+
 extern "C" rest_status rest_suffix_array_build_in_groups(const int32_t* d_tokens, uint64_t n_tokens,
                                                          int32_t sa_bytes, void* d_sa, uint64_t max_group,
                                                          void* d_ws, size_t ws_bytes, void* stream) {
@@ -371,4 +400,159 @@ extern "C" rest_status rest_suffix_array_build_in_groups(const int32_t* d_tokens
   if (sa_bytes == 4)
     return build_by_buckets<int32_t>(d_tokens, n_tokens, static_cast<int32_t*>(d_sa), max_group, d_ws, ws_bytes, st);
   return build_by_buckets<int64_t>(d_tokens, n_tokens, static_cast<int64_t*>(d_sa), max_group, d_ws, ws_bytes, st);
+}
+
+// ---------------------------------------------------------------------------------------
+// Appending tokens to a datastore.  The order compares 32 tokens, so only the suffixes that
+// start in the last 31 old positions (their windows now reach into the new tokens) and the
+// suffixes of the new tokens can change place; all other old entries keep their relative
+// order.  The "dirty" positions are sorted by themselves (the tail of the stream is a stream
+// of its own), each is located among the old entries by bisection, and one pass writes the
+// merged array.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+// order of two suffixes on their first 32 tokens, ties by position: true when a sorts before b
+__device__ __forceinline__ bool suffix_before(const int32_t* __restrict__ T, int64_t n, int64_t a, int64_t b) {
+  for (int k = 0; k < kKeyTokens; ++k) {
+    const bool ea = a + k >= n, eb = b + k >= n;
+    if (ea || eb) {
+      if (ea != eb) return ea;
+      break;
+    }
+    const uint32_t x = (uint32_t)T[a + k], y = (uint32_t)T[b + k];
+    if (x != y) return x < y;
+  }
+  return a < b;
+}
+
+// slots of the old array that hold dirty positions (at most 31), in ascending slot order
+template <typename SaT>
+__global__ void sa_find_dirty_slots(const SaT* __restrict__ sa_old, int64_t n_old, int64_t t0,
+                                    long long* __restrict__ slots, unsigned int* __restrict__ count) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_old; i += stride)
+    if ((int64_t)sa_old[i] >= t0) {
+      const unsigned int at = atomicAdd(count, 1u);
+      if (at < 32) slots[at] = i;
+    }
+}
+__global__ void sa_sort_dirty_slots(long long* __restrict__ slots, const unsigned int* __restrict__ count) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const int c = (int)min(*count, 32u);
+  for (int i = 1; i < c; ++i) {              // insertion sort of at most 31 numbers
+    const long long v = slots[i];
+    int j = i - 1;
+    while (j >= 0 && slots[j] > v) { slots[j + 1] = slots[j]; --j; }
+    slots[j + 1] = v;
+  }
+  for (int i = c; i < 32; ++i) slots[i] = 0x7FFFFFFFFFFFFFFFll;
+}
+
+// where[k] = first old slot whose (clean) entry sorts after dirty suffix k; old slots that hold
+// dirty positions are stepped over
+template <typename SaT, typename SegT>
+__global__ void sa_locate_dirty(const int32_t* __restrict__ T, int64_t n, const SaT* __restrict__ sa_old,
+                                int64_t n_old, int64_t t0, const SegT* __restrict__ seg, int64_t d,
+                                long long* __restrict__ where) {
+  const int64_t k = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+  if (k >= d) return;
+  const int64_t q = t0 + (int64_t)seg[k];
+  int64_t lo = 0, hi = n_old;                // answer in [lo, hi]
+  while (lo < hi) {
+    int64_t mid = lo + ((hi - lo) >> 1), probe = mid;
+    while (probe < hi && (int64_t)sa_old[probe] >= t0) ++probe;     // skip dirty slots to the right
+    if (probe == hi) {                       // nothing clean in [mid, hi): the answer is at most mid
+      hi = mid;
+      continue;
+    }
+    if (suffix_before(T, n, (int64_t)sa_old[probe], q)) lo = probe + 1; else hi = mid;
+  }
+  where[k] = lo;
+}
+
+template <typename SaT, typename SegT>
+__global__ void sa_merge_append(const SaT* __restrict__ sa_old, int64_t n_old, int64_t t0,
+                                const SegT* __restrict__ seg, int64_t d, const long long* __restrict__ where,
+                                const long long* __restrict__ dirty_slots, SaT* __restrict__ sa_new) {
+  __shared__ long long ds[32];
+  if (threadIdx.x < 32) ds[threadIdx.x] = dirty_slots[threadIdx.x];
+  __syncthreads();
+  auto dirty_before = [&](int64_t slot) {    // old dirty slots below `slot`
+    int c = 0;
+    for (int i = 0; i < 32; ++i) c += ds[i] < slot;
+    return (int64_t)c;
+  };
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_old + d; i += stride) {
+    if (i < n_old) {
+      const int64_t p = (int64_t)sa_old[i];
+      if (p >= t0) continue;                 // its new place comes from the sorted tail
+      int64_t lo = 0, hi = d;                // dirty suffixes placed at or before slot i: where[k] <= i
+      while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (where[mid] <= i) lo = mid + 1; else hi = mid;
+      }
+      sa_new[i - dirty_before(i) + lo] = (SaT)p;
+    } else {
+      const int64_t k = i - n_old, w = where[k];
+      sa_new[w - dirty_before(w) + k] = (SaT)(t0 + (int64_t)seg[k]);
+    }
+  }
+}
+
+template <typename SaT>
+rest_status append_impl(const int32_t* d_tokens, int64_t n_old, int64_t n_new, const SaT* sa_old, SaT* sa_new,
+                        void* d_ws, size_t ws_bytes, cudaStream_t st) {
+  const int64_t n = n_old + n_new;
+  const int64_t t0 = n_old > (kKeyTokens - 1) ? n_old - (kKeyTokens - 1) : 0;
+  const int64_t d = n - t0;                  // dirty positions t0 ... n - 1
+  if (d > 0x7FFFFFFFll) return REST_UNSUPPORTED;
+  // workspace: [where: d x 8][dirty slots: 32 x 8 + counter][tail array: d x 4][tail build scratch]
+  unsigned char* ws = static_cast<unsigned char*>(d_ws);
+  size_t o = 0;
+  long long* where = reinterpret_cast<long long*>(ws + o); o += align_up((size_t)d * 8);
+  long long* slots = reinterpret_cast<long long*>(ws + o); o += align_up(32 * 8);
+  unsigned int* count = reinterpret_cast<unsigned int*>(ws + o); o += kAlign;
+  int32_t* seg = reinterpret_cast<int32_t*>(ws + o); o += align_up((size_t)d * 4);
+  const size_t seg_ws = sa_layout((uint64_t)d).total;
+  if (ws_bytes < o + seg_ws) return REST_WORKSPACE_TOO_SMALL;
+  rest_status rc = build_by_doubling(d_tokens + t0, (uint64_t)d, 4, seg, ws + o, seg_ws, st);
+  if (rc != REST_OK) return rc;
+  REST_CUDA_TRY(cudaMemsetAsync(count, 0, sizeof(unsigned int), st));
+  const int sms = rest::sm_count() > 0 ? rest::sm_count() : 148;
+  const unsigned wide = (unsigned)std::min<int64_t>((n + kBlock - 1) / kBlock, (int64_t)sms * 32);
+  if (n_old > 0) sa_find_dirty_slots<SaT><<<wide, kBlock, 0, st>>>(sa_old, n_old, t0, slots, count);
+  sa_sort_dirty_slots<<<1, 32, 0, st>>>(slots, count);
+  sa_locate_dirty<SaT, int32_t><<<(unsigned)((d + kBlock - 1) / kBlock), kBlock, 0, st>>>(
+      d_tokens, n, sa_old, n_old, t0, seg, d, where);
+  sa_merge_append<SaT, int32_t><<<wide, kBlock, 0, st>>>(sa_old, n_old, t0, seg, d, where, slots, sa_new);
+  rest::count_launch(4);
+  REST_CUDA_TRY(cudaGetLastError());
+  return REST_OK;
+}
+
+}  // namespace
+
+extern "C" size_t rest_suffix_array_append_workspace_bytes(uint64_t n_new) {
+  if (n_new == 0 || n_new > 0x7FFFFF00ull) return 0;
+  const uint64_t d = n_new + kKeyTokens - 1;
+  return align_up(d * 8) + align_up(32 * 8) + kAlign + align_up(d * 4) + sa_layout(d).total;
+}
+
+extern "C" rest_status rest_suffix_array_append(const int32_t* d_tokens, uint64_t n_old, uint64_t n_new,
+                                                const void* d_sa_old, int32_t sa_bytes, void* d_sa_new,
+                                                void* d_ws, size_t ws_bytes, void* stream) {
+  if (!d_tokens || !d_sa_new || !d_ws || n_new == 0 || (n_old > 0 && !d_sa_old)) return REST_INVALID_ARG;
+  if (sa_bytes != 4 && sa_bytes != 8) return REST_INVALID_ARG;
+  if (n_old + n_new > (1ull << 40) || n_new > 0x7FFFFF00ull) return REST_UNSUPPORTED;
+  if (sa_bytes == 4 && n_old + n_new > 0x7FFFFFFFull) return REST_INVALID_ARG;
+  if (d_sa_old == d_sa_new) return REST_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_ws) & (kAlign - 1)) return REST_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (sa_bytes == 4)
+    return append_impl<int32_t>(d_tokens, (int64_t)n_old, (int64_t)n_new, static_cast<const int32_t*>(d_sa_old),
+                                static_cast<int32_t*>(d_sa_new), d_ws, ws_bytes, st);
+  return append_impl<int64_t>(d_tokens, (int64_t)n_old, (int64_t)n_new, static_cast<const int64_t*>(d_sa_old),
+                              static_cast<int64_t*>(d_sa_new), d_ws, ws_bytes, st);
 }

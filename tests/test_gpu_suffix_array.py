@@ -99,6 +99,54 @@ def test_bucket_method_gives_the_same_array_as_prefix_doubling(case):
             rest.rest_suffix_array_build(d_T, sa_bytes, max_group=1024)
 
 
+@pytest.mark.parametrize("name", ["binary", "constant", "period3", "long_repeat", "recipe"])
+def test_full_order_equals_the_oracle_suffix_array(name):
+    """Streams whose suffixes share far more than 32 tokens: the full-order build must give the
+    true suffix array (the oracle's comparison sort of whole suffixes)."""
+    rng = np.random.default_rng(6)
+    if name == "recipe":
+        T = datagen.make_tokens(datagen.WORKLOADS["single_stream"].scaled(n_tokens=60_000))
+    else:
+        block = rng.integers(0, 9, 700)
+        T = {"binary": rng.integers(0, 2, 4000), "constant": np.full(900, 7),
+             "period3": np.tile([4, 1, 9], 500), "long_repeat": np.r_[block, block, [8], block]}[name]
+    T = T.astype(np.int32)
+    want = oracle.suffix_array(T)
+    for sa_bytes in (4, 8):
+        got = rest.rest_suffix_array_build(to_dev(T), sa_bytes, full=True).cpu().numpy()
+        assert np.array_equal(got, want)
+    if name in ("constant", "period3", "long_repeat"):
+        assert not np.array_equal(gpu_sa(T), want)      # the 32-token order differs on these streams
+
+
+@pytest.mark.parametrize("kind", ["recipe", "binary", "constant", "period3"])
+def test_append_equals_a_build_from_scratch(kind):
+    """Tokens appended to a stream: the merged array must be the one a build of the whole stream
+    gives, for tails shorter and longer than the 32-token window and for both entry widths."""
+    rng = np.random.default_rng(8)
+    if kind == "recipe":
+        T = datagen.make_tokens(datagen.WORKLOADS["single_stream"].scaled(n_tokens=400_000))
+    elif kind == "binary":
+        T = rng.integers(0, 2, 30_000)
+    elif kind == "constant":
+        T = np.full(3000, 5)
+    else:
+        T = np.tile([4, 1, 9], 1000)
+    d_T = to_dev(T.astype(np.int32))
+    n = len(T)
+    for sa_bytes in (4, 8):
+        want = rest.rest_suffix_array_build(d_T, sa_bytes)
+        for n_old in (1, 7, 31, 32, 33, n // 3, n - 40, n - 1):
+            old = rest.rest_suffix_array_build(d_T[:n_old].contiguous(), sa_bytes)
+            got = rest.rest_suffix_array_append(d_T, old)
+            assert got.dtype == want.dtype and torch.equal(got, want), (kind, sa_bytes, n_old)
+    # in steps: three appends in a row
+    sa = rest.rest_suffix_array_build(d_T[:1000].contiguous(), 4)
+    for upto in (1010, n // 2, n):
+        sa = rest.rest_suffix_array_append(d_T[:upto].contiguous(), sa)
+    assert torch.equal(sa, rest.rest_suffix_array_build(d_T, 4))
+
+
 def test_argument_checks():
     L = rest.lib()
     assert L.rest_suffix_array_workspace_bytes(0) == 0
