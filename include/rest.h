@@ -103,9 +103,11 @@ typedef struct {
  *              REST_BAD_DATASTORE on failure.
  *              REST_DS_INDEX: build a bucket index into d_aux (asynchronously on `stream`): for
  *              every token the suffix-array range of the suffixes that start with it, and a hash
- *              table with the ranges of the frequent token pairs (up to 256 MiB).  rest_draft
- *              then starts each search inside such a range instead of over the whole array:
- *              fewer dependent reads, identical results.  Needs vocab <= 2^22 (ignored beyond).
+ *              table with the ranges of the frequent sequences of two, three and four tokens
+ *              (up to 512 MiB).  rest_draft then starts each search inside such a range instead
+ *              of over the whole array, and a frequent suffix of up to four tokens needs no
+ *              search at all: fewer dependent reads, identical results.  Needs vocab <= 2^22
+ *              (ignored beyond).
  *   d_aux      device scratch of rest_datastore_aux_bytes() bytes, 256-byte aligned, needed with
  *              either flag (NULL otherwise).  With REST_DS_INDEX the handle keeps using it: it
  *              must stay allocated and untouched until rest_datastore_destroy.

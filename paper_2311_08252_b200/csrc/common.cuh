@@ -29,20 +29,27 @@ constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 16, kSmemSlotAttnWide = 17, kS
 
 // Bucket index over the suffix array (an accelerator built by rest_datastore_create; results
 // never depend on it).  `first[t]` is the first suffix-array slot whose suffix starts with token
-// t (first[vocab] = n_tokens), so suffixes starting with t occupy [first[t], first[t + 1]).
-// `table` is a hash table over the frequent token pairs (t0, t1): groups of four 32-byte
-// entries {key, lo, hi, unused}; an entry says that the suffixes starting with (t0, t1) occupy
-// slots [lo, hi).  Pairs that occur fewer times than a size-dependent minimum are not stored;
-// a search for them starts from the first-token range instead.
+// t (first[vocab] = n_sa), so suffixes starting with t occupy [first[t], first[t + 1]).
+// `table` is a hash table over the frequent token n-grams, n = 2 ... levels: groups of four
+// 32-byte entries {key, lo, hi, unused}; an entry says that the suffixes starting with that
+// n-gram occupy slots [lo, hi).  n-grams that occur fewer times than a size-dependent minimum
+// are not stored: a search for them starts from the range of a shorter prefix instead.
 struct BucketIndex {
   const long long* first;               // null: no index
   const unsigned long long* table;      // 4 words per entry
   uint32_t group_mask;                  // number of groups - 1 (a group = 4 entries = 128 bytes)
   const uint32_t* unusable;             // non-zero: the build met an entry or token out of range
+  int levels;                           // longest n-gram stored (2 ... 4)
+  int token_bits;                       // bits per token in a key
 };
 constexpr unsigned long long kIndexEmptyKey = ~0ull;
-__host__ __device__ inline unsigned long long index_pair_key(uint32_t t0, uint32_t t1) {
-  return ((unsigned long long)t0 << 32) | (unsigned long long)t1;
+constexpr int kIndexMaxLevel = 4;
+// key of an n-gram: n - 1 in the top two bits, the tokens below, first token lowest (n *
+// token_bits <= 60, so no key equals the empty marker)
+__host__ __device__ inline unsigned long long index_key(const int32_t* tok, int n, int token_bits) {
+  unsigned long long key = (unsigned long long)(n - 1) << 62;
+  for (int k = 0; k < n; ++k) key |= (unsigned long long)(uint32_t)tok[k] << (k * token_bits);
+  return key;
 }
 __host__ __device__ inline uint32_t index_group_of(unsigned long long key, uint32_t group_mask) {
   key ^= key >> 29;

@@ -94,23 +94,29 @@ __global__ void validate_kernel(const int32_t* __restrict__ T, const SaT* __rest
 
 // ---- bucket index ------------------------------------------------------------------------
 constexpr uint32_t kIndexMaxVocab = 1u << 22;       // the first-token table has vocab + 1 entries
-constexpr uint64_t kIndexMinEntries = 1ull << 12, kIndexMaxEntries = 1ull << 23;
+constexpr uint64_t kIndexMinEntries = 1ull << 12, kIndexMaxEntries = 1ull << 24;
 
 constexpr size_t kIndexHeaderBytes = 256;           // word 0: "the datastore has an entry or token out of range"
 struct IndexLayout {
   uint64_t entries;      // hash-table entries (a power of two; 0 = no index for this datastore)
-  int64_t min_run;       // token pairs with fewer occurrences are not stored
+  int64_t min_run;       // n-grams with fewer occurrences are not stored
+  int levels, token_bits;
   size_t first_bytes, table_bytes, total;
 };
 IndexLayout index_layout(uint64_t n, uint32_t vocab) {
   IndexLayout l = {};
   if (vocab > kIndexMaxVocab || n < 2) return l;
   uint64_t e = kIndexMinEntries;
-  while (e < n / 2 && e < kIndexMaxEntries) e <<= 1;
+  while (e < 2 * n && e < kIndexMaxEntries) e <<= 1;
   l.entries = e;
-  // at most n / min_run pairs are stored: the table stays at most one eighth full, so a group
-  // of four overflows practically never (and a pair that finds its group full is just left out)
-  l.min_run = (int64_t)((8 * n + e - 1) / e);
+  l.token_bits = 1;
+  while ((1ull << l.token_bits) < (uint64_t)vocab) ++l.token_bits;
+  l.levels = 60 / l.token_bits < rest::kIndexMaxLevel ? 60 / l.token_bits : rest::kIndexMaxLevel;
+  if (l.levels < 2) { l.entries = 0; return l; }
+  // at most n / min_run n-grams of each length are stored: the table stays at most one eighth
+  // full, so a group of four overflows practically never (and an n-gram that finds its group
+  // full is just left out)
+  l.min_run = (int64_t)((8 * (uint64_t)(l.levels - 1) * n + e - 1) / e);
   if (l.min_run < 1) l.min_run = 1;
   l.first_bytes = (((size_t)vocab + 1) * 8 + 255) / 256 * 256;
   l.table_bytes = (size_t)e * 32;
@@ -122,57 +128,75 @@ size_t validation_bytes(uint64_t n) {
   return ((n + 31) / 32) * 4 + 256;
 }
 
-// The token pair a suffix starts with; t1 = -1 for the one suffix that is a single token long.
-// false when the entry or a token is out of range (such a datastore gets no usable index).
+// The first tokens of the suffix in slot `slot`: tok[0 .. have), have <= kIndexMaxLevel (fewer
+// when the suffix is shorter).  false when the entry or a token is out of range (such a
+// datastore gets no usable index).
 template <typename SaT>
-__device__ __forceinline__ bool pair_at(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
-                                        int64_t n, uint32_t vocab, int64_t slot, int32_t& t0, int32_t& t1) {
+__device__ __forceinline__ bool head_at(const int32_t* __restrict__ T, const SaT* __restrict__ sa, int64_t n,
+                                        uint32_t vocab, int64_t slot, int32_t (&tok)[rest::kIndexMaxLevel], int& have) {
   const int64_t p = (int64_t)sa[slot];
+  have = 0;
   if (p < 0 || p >= n) return false;
-  t0 = T[p];
-  t1 = p + 1 < n ? T[p + 1] : -1;
-  return t0 >= 0 && (uint32_t)t0 < vocab && (t1 == -1 || (t1 >= 0 && (uint32_t)t1 < vocab));
+  for (int k = 0; k < rest::kIndexMaxLevel; ++k) {
+    tok[k] = -1;
+    if (p + k < n) {
+      tok[k] = T[p + k];
+      if (tok[k] < 0 || (uint32_t)tok[k] >= vocab) return false;
+      have = k + 1;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ bool same_head(const int32_t (&a)[rest::kIndexMaxLevel], int ha,
+                                          const int32_t (&b)[rest::kIndexMaxLevel], int hb, int len) {
+  if (ha < len || hb < len) return false;
+  for (int k = 0; k < len; ++k)
+    if (a[k] != b[k]) return false;
+  return true;
 }
 
-// One thread per suffix-array slot.  The slot where a first token begins writes first[t]; the
-// slots where a run of one token pair begins and ends write that pair's lo and hi, provided the
-// run has at least min_run members (seen by looking min_run - 1 slots ahead or back).
+// One thread per suffix-array slot.  The slot where a first token begins writes first[t]; for
+// every n-gram length 2 ... levels the slots where a run of one n-gram begins and ends write
+// that n-gram's lo and hi, provided the run has at least min_run members (seen by looking
+// min_run - 1 slots ahead or back).
 template <typename SaT>
 __global__ void index_build_kernel(const int32_t* __restrict__ T, const SaT* __restrict__ sa, int64_t n,
-                                   int64_t n_sa, uint32_t vocab, int64_t min_run, long long* __restrict__ first,
-                                   unsigned long long* __restrict__ table, uint32_t group_mask,
-                                   uint32_t* __restrict__ unusable) {
+                                   int64_t n_sa, uint32_t vocab, int64_t min_run, int levels, int token_bits,
+                                   long long* __restrict__ first, unsigned long long* __restrict__ table,
+                                   uint32_t group_mask, uint32_t* __restrict__ unusable) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_sa; i += stride) {
-    int32_t t0, t1, a0 = -2, a1 = -2, b0 = -2, b1 = -2;
+    int32_t me[rest::kIndexMaxLevel], up[rest::kIndexMaxLevel], dn[rest::kIndexMaxLevel], far[rest::kIndexMaxLevel];
+    int hme = 0, hup = 0, hdn = 0, hfar = 0;
     // a datastore with an entry or a token out of range gets no index: searches then run over
     // the whole array, where such an entry is reported when it is met
-    if (!pair_at(T, sa, n, vocab, i, t0, t1)) { *unusable = 1u; continue; }
-    if (i > 0 && !pair_at(T, sa, n, vocab, i - 1, a0, a1)) a0 = -2;
-    if (i + 1 < n_sa && !pair_at(T, sa, n, vocab, i + 1, b0, b1)) b0 = -2;
-    if (i == 0 || a0 != t0) first[t0] = i;
-    if (t1 < 0) continue;
-    const bool starts = i == 0 || a0 != t0 || a1 != t1;
-    const bool ends = i + 1 == n_sa || b0 != t0 || b1 != t1;
-    if (!starts && !ends) continue;
-    bool long_enough = true;
-    if (min_run > 1) {
-      long_enough = false;                       // a run of one is shorter than any minimum above one
-      if (!(starts && ends)) {
-        const int64_t far = starts ? i + min_run - 1 : i - min_run + 1;
-        int32_t f0, f1;
-        long_enough = far >= 0 && far < n_sa && pair_at(T, sa, n, vocab, far, f0, f1) && f0 == t0 && f1 == t1;
+    if (!head_at(T, sa, n, vocab, i, me, hme)) { *unusable = 1u; continue; }
+    if (i > 0 && !head_at(T, sa, n, vocab, i - 1, up, hup)) hup = 0;
+    if (i + 1 < n_sa && !head_at(T, sa, n, vocab, i + 1, dn, hdn)) hdn = 0;
+    if (i == 0 || hup < 1 || up[0] != me[0]) first[me[0]] = i;
+    for (int len = 2; len <= levels && len <= hme; ++len) {
+      const bool starts = i == 0 || !same_head(me, hme, up, hup, len);
+      const bool ends = i + 1 == n_sa || !same_head(me, hme, dn, hdn, len);
+      if (!starts && !ends) continue;
+      bool long_enough = true;
+      if (min_run > 1) {
+        long_enough = false;                     // a run of one is shorter than any minimum above one
+        if (!(starts && ends)) {
+          const int64_t f = starts ? i + min_run - 1 : i - min_run + 1;
+          long_enough = f >= 0 && f < n_sa && head_at(T, sa, n, vocab, f, far, hfar) &&
+                        same_head(me, hme, far, hfar, len);
+        }
       }
-    }
-    if (!long_enough) continue;
-    const unsigned long long key = rest::index_pair_key((uint32_t)t0, (uint32_t)t1);
-    unsigned long long* grp = table + (size_t)rest::index_group_of(key, group_mask) * 16;
-    for (int e = 0; e < 4; ++e) {
-      const unsigned long long cur = atomicCAS(grp + e * 4, rest::kIndexEmptyKey, key);
-      if (cur == rest::kIndexEmptyKey || cur == key) {
-        if (starts) grp[e * 4 + 1] = (unsigned long long)i;
-        if (ends) grp[e * 4 + 2] = (unsigned long long)(i + 1);
-        break;
+      if (!long_enough) continue;
+      const unsigned long long key = rest::index_key(me, len, token_bits);
+      unsigned long long* grp = table + (size_t)rest::index_group_of(key, group_mask) * 16;
+      for (int e = 0; e < 4; ++e) {
+        const unsigned long long cur = atomicCAS(grp + e * 4, rest::kIndexEmptyKey, key);
+        if (cur == rest::kIndexEmptyKey || cur == key) {
+          if (starts) grp[e * 4 + 1] = (unsigned long long)i;
+          if (ends) grp[e * 4 + 2] = (unsigned long long)(i + 1);
+          break;
+        }
       }
     }
   }
@@ -260,7 +284,7 @@ extern "C" rest_status rest_datastore_create_shard(const int32_t* d_tokens, uint
     REST_CUDA_TRY(cudaStreamSynchronize(st));
     if (h_flags != 0) return REST_BAD_DATASTORE;
   }
-  rest::BucketIndex idx = {nullptr, nullptr, 0, nullptr};
+  rest::BucketIndex idx = {nullptr, nullptr, 0, nullptr, 0, 0};
   if (il.entries > 0) {
     // built after a successful validation (when asked for), on the same stream, without a sync:
     // calls that use the handle on this stream see the finished index
@@ -275,14 +299,15 @@ extern "C" rest_status rest_datastore_create_shard(const int32_t* d_tokens, uint
     const int blocks = (int)((n_sa + 255) / 256 < wave ? (n_sa + 255) / 256 : wave);
     if (sa_bytes == 4)
       index_build_kernel<int32_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int32_t*>(d_sa),
-                                                          (int64_t)n_tokens, (int64_t)n_sa, vocab, il.min_run, first, table, group_mask, unusable);
+                                                          (int64_t)n_tokens, (int64_t)n_sa, vocab, il.min_run, il.levels, il.token_bits, first, table, group_mask, unusable);
     else
       index_build_kernel<int64_t><<<blocks, 256, 0, st>>>(d_tokens, static_cast<const int64_t*>(d_sa),
-                                                          (int64_t)n_tokens, (int64_t)n_sa, vocab, il.min_run, first, table, group_mask, unusable);
+                                                          (int64_t)n_tokens, (int64_t)n_sa, vocab, il.min_run, il.levels, il.token_bits, first, table, group_mask, unusable);
     index_fill_kernel<<<1, 1024, 0, st>>>(first, vocab, (int64_t)n_sa);
     rest::count_launch(2);
     REST_CUDA_TRY(cudaGetLastError());
     idx.first = first; idx.table = table; idx.group_mask = group_mask; idx.unusable = unusable;
+    idx.levels = il.levels; idx.token_bits = il.token_bits;
   }
   rest_datastore* ds = static_cast<rest_datastore*>(malloc(sizeof(rest_datastore)));
   if (!ds) return REST_INVALID_ARG;

@@ -39,7 +39,8 @@ constexpr int kHistHi = 2080;   // first-level bins: weights below 1024 one by o
 constexpr int kHistLo = 1024;
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kMaxTrunc = 32;                         // rows cut short by the end of the stream (at most m exist)
-constexpr int kMaxLoads = (33 * kMaxM + 31) / 32;     // load instructions for a warp's 33 rows
+constexpr int kRowLoads = 17;                         // load instructions for a warp's 33 rows, two rows each
+constexpr int kBigListCap = 4096;                     // nodes of weight >= 5 a block can list
 constexpr int kPositionCacheRows = 1024;              // rows whose suffix position stays in shared memory for phase 4
 // Batched path (calls with far more contexts than the GPU holds at once): threads per block,
 // lanes per probe round once the probes leave L2, the number of 32-wide rounds before that,
@@ -81,6 +82,7 @@ struct DraftArgs {
   int nwords;   // bitmap words per depth
   int kcap;     // rows the block's shared memory holds, a multiple of 32
   int pcache_rows;   // rows whose suffix position is kept in shared memory
+  int bigcap;        // nodes of weight >= 5 the block can list (an even number)
   // rows handed in by the caller as R sorted runs per context (rest_draft_from_runs): T then
   // points at the rows [B][R][Kr][m]
   const int32_t* row_len;     // [B][R][Kr]
@@ -203,14 +205,6 @@ __device__ __forceinline__ int next_set(const uint32_t* __restrict__ row,
   return bits ? (w << 5) + __ffs(bits) - 1 : (int)jump[w];
 }
 
-// Largest set bit at or before position j (bit 0 is always set).
-__device__ __forceinline__ int prev_set(const uint32_t* __restrict__ row, int j) {
-  int w = j >> 5;
-  uint32_t bits = row[w] & ((2u << (j & 31)) - 1u);
-  while (bits == 0 && w > 0) bits = row[--w];
-  return (w << 5) + 31 - __clz(bits | 1u);
-}
-
 // Executed by one warp.  hist[0..nbins) holds counts; total >= need >= 1.  Finds the largest
 // bin b with sum(hist[k], k > b) < need; returns b and that sum.
 __device__ void warp_threshold_desc(const uint32_t* hist, int nbins, uint32_t need, int lane,
@@ -261,26 +255,31 @@ struct Smem {
   uint32_t hist_lo[kHistLo];   // inside the threshold bin: by depth (and the weight's low bits)
 };
 
-// Suffix-array range of the suffixes that start with the token pair (t0, t1), from the bucket
-// index.  Warp-cooperative: four lanes read the four entries of the pair's group (one 128-byte
-// line).  false when the pair is not stored.
-__device__ __forceinline__ bool index_pair_range(const rest::BucketIndex& idx, uint32_t t0, uint32_t t1,
+// Suffix-array range of the suffixes that start with the longest indexed prefix of q (n tokens):
+// the bucket index is asked for q's first 2, 3, ... min(n, levels) tokens at once (four lanes
+// per length read the four entries of that n-gram's group, one 128-byte line each) and the
+// longest one stored wins.  Returns its length (0: none stored) and its range.
+__device__ __forceinline__ int index_ngram_range(const rest::BucketIndex& idx, const int (&q)[16], int n,
                                                  int lane, int64_t n_slots, int64_t& lo, int64_t& hi) {
-  const unsigned long long key = rest::index_pair_key(t0, t1);
-  const unsigned long long* grp = idx.table + (size_t)rest::index_group_of(key, idx.group_mask) * 16;
-  unsigned long long k = rest::kIndexEmptyKey;
+  const int level = 2 + (lane >> 2);
+  const bool asks = lane < 4 * (rest::kIndexMaxLevel - 1) && level <= n && level <= idx.levels;
+  unsigned long long key = (unsigned long long)(level - 1) << 62, k = rest::kIndexEmptyKey;
+#pragma unroll
+  for (int t = 0; t < rest::kIndexMaxLevel; ++t)
+    if (t < level) key |= (unsigned long long)(uint32_t)q[t] << (t * idx.token_bits);
   long long l = -1, h = -1;
-  if (lane < 4) {
-    k = __ldg(grp + lane * 4);
-    l = (long long)__ldg(grp + lane * 4 + 1);
-    h = (long long)__ldg(grp + lane * 4 + 2);
+  if (asks) {
+    const unsigned long long* e = idx.table + (size_t)rest::index_group_of(key, idx.group_mask) * 16 + (lane & 3) * 4;
+    k = __ldg(e);
+    l = (long long)__ldg(e + 1);
+    h = (long long)__ldg(e + 2);
   }
-  const unsigned hit = __ballot_sync(kFull, lane < 4 && k == key && l >= 0 && h > l && h <= n_slots);
-  if (hit == 0) return false;
-  const int src = __ffs(hit) - 1;
+  const unsigned hit = __ballot_sync(kFull, asks && k == key && l >= 0 && h > l && h <= n_slots);
+  if (hit == 0) return 0;
+  const int src = 31 - __clz(hit);           // the highest lane that hit asks for the longest n-gram
   lo = __shfl_sync(kFull, l, src);
   hi = __shfl_sync(kFull, h, src);
-  return true;
+  return 2 + (src >> 2);
 }
 
 // Rows in bitmap word w whose continuation is shorter than d tokens (they end a run like any
@@ -323,15 +322,19 @@ rest_draft_kernel(DraftArgs a) {
   static_assert(NT % 32 == 0 && NT >= 128, "whole warps; enough threads for the set-up loops");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& s = *reinterpret_cast<Smem*>(smem_raw);
-  // per warp: start position, length and comparable length of its 33 slots (the row before the
+  // per warp: token address and length of its 33 slots (the row before the
   // warp's first one, then its 32 rows); the suffix positions of the first rows (phase 4 reads
   // the kept nodes' tokens through them); then the block's bitmaps
   long long* slot_base = reinterpret_cast<long long*>(smem_raw + sizeof(Smem));            // [NW][34]
   long long* pcache = slot_base + NW * 34;                                                  // [pcache_rows]
-  int* slot_len = reinterpret_cast<int*>(pcache + a.pcache_rows);                           // [NW][66]
-  uint32_t* bm = reinterpret_cast<uint32_t*>(slot_len + NW * 66);                           // [m][nwords]
-  uint16_t* jump = reinterpret_cast<uint16_t*>(bm + a.m * a.nwords);                        // [m][nwords]
+  int* slot_len = reinterpret_cast<int*>(pcache + a.pcache_rows);                           // [NW][34]
+  uint32_t* bm = reinterpret_cast<uint32_t*>(slot_len + NW * 34);                           // [m][nwords]
+  // nodes of weight >= 5 met by the first pass over the bitmaps: (depth << 16 | row) and weight
+  // (the 32-bit arrays first, then the 16-bit ones: every array is aligned to its element size)
+  uint32_t* big_dj = bm + a.m * a.nwords;                                                   // [bigcap]
+  uint16_t* jump = reinterpret_cast<uint16_t*>(big_dj + a.bigcap);                          // [m][nwords]
   uint16_t* tiecnt = jump + a.m * a.nwords;                                                 // [nwords]
+  uint16_t* big_c = tiecnt + a.nwords;                                                      // [bigcap]
 
   if constexpr (PART == kBuild) {
     if ((int)blockIdx.x >= a.list_count[a.which]) return;
@@ -450,8 +453,8 @@ rest_draft_kernel(DraftArgs a) {
     int64_t next_gt = -1, lb;
     if (have_index) {
       // every suffix that starts with the query's first token lies in [f0, f1); when the index
-      // also stores the query's first token pair, every suffix that starts with that pair lies
-      // in [lo0, hi0).  Slot hi0 (or the end of the array) compares greater than the query.
+      // also stores the query's first two, three or four tokens, every suffix that starts with
+      // those lies in [lo0, hi0).  Slot hi0 (or the end of the array) compares greater than the query.
       int64_t lo0 = __ldg(a.idx.first + q[0]), hi0 = __ldg(a.idx.first + q[0] + 1);
       lo0 = lo0 < 0 ? 0 : (lo0 > n_sa ? n_sa : lo0);
       hi0 = hi0 < lo0 ? lo0 : (hi0 > n_sa ? n_sa : hi0);
@@ -459,11 +462,11 @@ rest_draft_kernel(DraftArgs a) {
         if (lane == 0) { s.lb[1] = lo0; s.ub[1] = hi0; s.bhi[1] = hi0; }
         return;
       }
-      int64_t plo, phi;
-      if (index_pair_range(a.idx, (uint32_t)q[0], (uint32_t)q[1], lane, n_sa, plo, phi) &&
-          plo >= lo0 && phi <= hi0) {
-        if (n == 2) {                     // the pair's range is the answer
-          if (lane == 0) { s.lb[2] = plo; s.ub[2] = phi; s.bhi[2] = phi; }
+      int64_t plo = 0, phi = 0;
+      const int found = index_ngram_range(a.idx, q, n, lane, n_sa, plo, phi);
+      if (found > 0 && plo >= lo0 && phi <= hi0) {
+        if (found == n) {                 // the n-gram's own range is the answer
+          if (lane == 0) { s.lb[n] = plo; s.ub[n] = phi; s.bhi[n] = phi; }
           return;
         }
         lo0 = plo; hi0 = phi;
@@ -505,11 +508,10 @@ rest_draft_kernel(DraftArgs a) {
   for (int n = nq; n >= a.n_min; --n)
     if (s.ub[n] != s.lb[n]) { n_win = n; break; }
   // 1b: only the winning length needs its upper bound, and only if the last round of its lower
-  // bound did not already show where the run ends.  The whole block searches: in the first
-  // round the first half of the threads probes the slots right behind the first match one by
-  // one and the second half probes at geometrically growing distances (so a short run is
-  // settled in one round whatever the size of the range); the rounds after that cut what is
-  // left into NT + 1 parts.
+  // bound did not already show where the run ends.  The block searches: in the first round
+  // half of the probing threads look at the slots right behind the first match one by one and
+  // the other half at geometrically growing distances (so a short run is settled in one round
+  // whatever the size of the range); the rounds after that cut what is left into NT + 1 parts.
   if (n_win != 0 && s.ub[n_win] < 0) {       // block-uniform
     const int n = n_win;
     int q[16];
@@ -518,7 +520,15 @@ rest_draft_kernel(DraftArgs a) {
     bool bad = false;
     const int64_t end = s.bhi[n];            // slots from here on are known to compare greater
     int64_t lo2 = s.lb[n] + 1, hi2 = end;    // the answer lies in [lo2, hi2]
-    constexpr int H = NT / 2, S = (H / 34) > 0 ? (H / 34) : 1;     // linear probes; geometric steps per octave
+    // A probe reads n tokens from a random place, so the first round uses fewer threads the
+    // longer the suffix (most runs are a handful of slots long and end inside its linear part);
+    // the geometric probes use as many steps per octave as cover the range that is left (the
+    // finer the steps, the smaller the bracket the second round has to settle).
+    const int P1 = min(NT, max(64, (2048 / n) & ~31));
+    const int H = P1 / 2;
+    int octaves = 1;
+    while (octaves < 44 && ((int64_t)H << octaves) < end - lo2) ++octaves;
+    const int S = max(1, (P1 - H) / octaves);
     auto first_round_pos = [&](int t) -> int64_t {
       if (t < H) return lo2 + t;
       const int e = t - H + 1, oct = e / S, frac = e - oct * S;
@@ -535,9 +545,13 @@ rest_draft_kernel(DraftArgs a) {
         if (exact) return lo2 + t;
         return lo2 + (int64_t)(((unsigned long long)(t + 1) * (unsigned long long)size) / (unsigned long long)(NT + 1));
       };
-      const int64_t pos = pos_of(tid);
-      bool t = true;                                      // slots from hi2 on compare greater
-      if (pos < hi2) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
+      const int width = first ? P1 : NT;                  // threads that probe in this round
+      bool t = false;
+      if (tid < width) {
+        const int64_t pos = pos_of(tid);
+        t = true;                                         // slots from hi2 on compare greater
+        if (pos < hi2) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
+      }
       const unsigned bal = __ballot_sync(kFull, t);
       if (lane == 0) s.warp_first[warp] = bal ? warp * 32 + __ffs(bal) - 1 : 0x7FFFFFFF;
       __syncthreads();
@@ -545,7 +559,7 @@ rest_draft_kernel(DraftArgs a) {
       for (int w = 0; w < NW; ++w) tf = min(tf, s.warp_first[w]);
       __syncthreads();
       if (tf == 0x7FFFFFFF) {
-        lo2 = pos_of(NT - 1) + 1;
+        lo2 = pos_of(width - 1) + 1;
         if (lo2 > hi2) lo2 = hi2;
       } else {
         const int64_t pf = pos_of(tf);
@@ -592,52 +606,81 @@ rest_draft_kernel(DraftArgs a) {
   const int nw = (Kp + 31) >> 5;            // bitmap words that hold rows
 
   // ---- phase 2: gather rows, common-prefix lengths, node-start bitmaps --------------------
-  // Slot 0 of a warp is the row before its first row, slot l + 1 the row of lane l.  The 33
-  // rows are read as one run of 33 m words, word f by lane f mod 32 in load f / 32: consecutive
-  // lanes read consecutive tokens of a row, so a load instruction touches three or four rows
-  // (a few cache lines) instead of 32.  Word f is compared with word f - m (the same column of
-  // the row before: lane - m of the same load, or of the load before) right where it sits; a
-  // ballot turns the "equal" and "smaller" outcomes of each load into bit strings, and lane l
-  // cuts the m bits of its row out of them: the number of leading equal columns is the common
-  // prefix.  The suffix-array entries of the next iteration are fetched one iteration ahead.
+  // Slot 0 of a warp is the row before its first row, slot l + 1 the row of lane l.  A load
+  // instruction fetches two slots, 16 columns each (lane = 16 * slot parity + column): the
+  // lanes of a row read consecutive tokens, so an instruction touches two rows (a few cache
+  // lines) instead of 32.  A token is compared with the token above it (the same column of the
+  // slot before: the other half-warp of the same load, or of the load before) right where it
+  // sits; a ballot turns the "equal" and "smaller" outcomes of each load into bit strings, and
+  // lane l cuts the 16 bits of its row out of them: the number of leading equal columns is the
+  // common prefix.  The suffix-array entries of the next iteration are fetched one iteration
+  // ahead.
   {
-    long long* sb = slot_base + warp * 34;
-    int* sl = slot_len + warp * 66;          // lengths, then comparable lengths min(len, len of the row before)
-    int* slim = sl + 33;
-    const uint32_t magic = (65536u + (uint32_t)m - 1u) / (uint32_t)m;    // f / m = (f * magic) >> 16 for f < 600
-    const int nload = (33 * m + 31) >> 5;
-    const int src_lane = (lane - m) & 31;
+    // per slot: address of the row's first token, and the row's length
+    const int32_t** sb = reinterpret_cast<const int32_t**>(slot_base + warp * 34);
+    int* sl = slot_len + warp * 34;
     // where row j comes from: the suffix-array entry of its sampled slot, or (rows handed in
-    // as runs) its place in the caller's row array, through the merged order
+    // as runs) its place in the caller's row array, through the merged order.  The sampled
+    // slot lo + floor(j cnt / K) advances by a fixed quotient and remainder from one iteration
+    // to the next (j grows by NT), which saves a 64-bit division per row.
     const uint32_t* ord = PART == kFromRuns ? a.order + (int64_t)b * a.kcap : nullptr;
-    auto row_entry = [&](int j) -> int64_t {
+    const bool strided = PART != kFromRuns && cnt > (int64_t)a.K && a.sample_mode == REST_SAMPLE_STRIDED;
+    const unsigned long long uK = (unsigned long long)a.K;
+    const unsigned long long step_q = strided ? ((unsigned long long)NT * (unsigned long long)cnt) / uK : (unsigned long long)NT;
+    const unsigned long long step_r = strided ? ((unsigned long long)NT * (unsigned long long)cnt) % uK : 0ull;
+    // this thread's rows j = tid, tid + NT, ...: slot offset and remainder of j cnt / K
+    unsigned long long off = strided ? ((unsigned long long)tid * (unsigned long long)cnt) / uK : (unsigned long long)tid;
+    unsigned long long rem = strided ? ((unsigned long long)tid * (unsigned long long)cnt) % uK : 0ull;
+    // the same for the row before the warp's rows of the NEXT iteration, j + NT - 1 (lane 0
+    // fetches it one iteration ahead)
+    unsigned long long poff = 0, prem = 0;
+    if (lane == 0) {
+      const unsigned long long jn = (unsigned long long)(tid + NT - 1);
+      poff = strided ? (jn * (unsigned long long)cnt) / uK : jn;
+      prem = strided ? (jn * (unsigned long long)cnt) % uK : 0ull;
+    }
+    auto advance = [&](unsigned long long& o, unsigned long long& r) {
+      o += step_q; r += step_r;
+      if (r >= uK) { r -= uK; ++o; }
+    };
+    auto entry_at = [&](int j, unsigned long long o) -> int64_t {
       if constexpr (PART == kFromRuns) return (int64_t)ord[j];
-      else return (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
+      else return (int64_t)__ldg(sa + lo + (int64_t)o);
     };
     // start of the row's tokens (relative to Trow) and its length; `bad` when the entry is out of range
     auto row_place = [&](int64_t& p, int64_t& base, int& len, bool& bad) {
       if constexpr (PART == kFromRuns) {
         if (p < 0 || p >= (int64_t)a.R * a.Kr) { bad = true; p = 0; }
+        len = bad ? 0 : min(max(a.row_len[(int64_t)b * a.R * a.Kr + p], 0), m);
         p *= m;
         base = p;
-        len = bad ? 0 : min(max(a.row_len[(int64_t)b * a.R * a.Kr + p / m], 0), m);
       } else {
         if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
         base = p + n_win;
-        const int64_t rem = n_tokens - base;
-        len = bad ? 0 : (int)(rem < 0 ? 0 : (rem > m ? m : rem));
+        const int64_t rem_t = n_tokens - base;
+        len = bad ? 0 : (int)(rem_t < 0 ? 0 : (rem_t > m ? m : rem_t));
       }
     };
     int64_t p_next = 0, pp_next = 0;
-    if (tid < Kp) p_next = row_entry(tid);
-    if (lane == 0 && tid > 0 && tid <= Kp) pp_next = row_entry(tid - 1);
+    if (tid < Kp) p_next = entry_at(tid, off);
+    if (lane == 0 && tid > 0 && tid <= Kp) {
+      const unsigned long long jp = (unsigned long long)(tid - 1);
+      pp_next = entry_at(tid - 1, strided ? (jp * (unsigned long long)cnt) / uK : jp);
+    }
+    const int half = lane >> 4, col = lane & 15;
+    if (lane == 0) { sl[33] = 0; sb[33] = Trow; }     // slot 33 does not exist
+    // columns past a row's end read as a value no token has (tokens are below 2^31), different
+    // for neighbouring slots: they never compare equal to anything above or below them
+    const uint32_t pad = 0x80000000u | (uint32_t)half;
     for (int it = 0; it < niter; ++it) {
       const int jbase = it * NT + warp * 32;
       const int j = jbase + lane;
       int64_t p = p_next;
       int64_t pp = pp_next;
-      if (j + NT < Kp) p_next = row_entry(j + NT);
-      if (lane == 0 && j + NT <= Kp) pp_next = row_entry(j + NT - 1);
+      advance(off, rem);
+      if (j + NT < Kp) p_next = entry_at(j + NT, off);
+      if (lane == 0 && j + NT <= Kp) pp_next = entry_at(j + NT - 1, poff);
+      advance(poff, prem);
       if (jbase >= Kp) continue;   // warp-uniform
       const bool valid = j < Kp;
       bool bad = false;
@@ -652,43 +695,32 @@ rest_draft_kernel(DraftArgs a) {
         plen = 0;
         int64_t pbase = 0;
         if (j > 0) row_place(pp, pbase, plen, bad);   // the row before belongs to another warp
-        sb[0] = pbase; sl[0] = plen; slim[0] = 0;
+        sb[0] = Trow + pbase; sl[0] = plen;
       }
       const int lim = min(len, plen);
-      sb[lane + 1] = base; sl[lane + 1] = len; slim[lane + 1] = lim;
+      sb[lane + 1] = Trow + base; sl[lane + 1] = len;
       __syncwarp();
-      uint32_t vals[kMaxLoads];
+      uint32_t vals[kRowLoads];
 #pragma unroll
-      for (int i = 0; i < kMaxLoads; ++i) {
-        vals[i] = 0;
-        if (i < nload) {
-          const uint32_t f = (uint32_t)(i * 32 + lane);
-          const uint32_t r = (f * magic) >> 16, c = f - r * (uint32_t)m;
-          if (r < 33u && (int)c < sl[r]) vals[i] = (uint32_t)__ldg(Trow + sb[r] + c);
-        }
+      for (int i = 0; i < kRowLoads; ++i) {
+        const int r = 2 * i + half;
+        vals[i] = col < sl[r] ? (uint32_t)__ldg(sb[r] + col) : pad;
       }
-      uint32_t my_eq = 0, my_lt = 0;         // lane i keeps the bit strings of load i
+      uint32_t my_eq = 0, my_lt = 0, other_prev = 0;     // lane i keeps the bit strings of load i
 #pragma unroll
-      for (int i = 0; i < kMaxLoads; ++i) {
-        if (i < nload) {                     // warp-uniform
-          const uint32_t f = (uint32_t)(i * 32 + lane);
-          const uint32_t r = (f * magic) >> 16, c = f - r * (uint32_t)m;
-          const uint32_t x = __shfl_sync(kFull, vals[i], src_lane);
-          const uint32_t y = i > 0 ? __shfl_sync(kFull, vals[i > 0 ? i - 1 : 0], src_lane) : 0u;
-          const uint32_t before = lane >= m ? x : y;
-          const bool comparable = r >= 1u && r < 33u && (int)c < slim[r];
-          const uint32_t eq = __ballot_sync(kFull, comparable && vals[i] == before);
-          const uint32_t lt = __ballot_sync(kFull, comparable && before < vals[i]);
-          if (lane == i) { my_eq = eq; my_lt = lt; }
-        }
+      for (int i = 0; i < kRowLoads; ++i) {
+        const uint32_t other = __shfl_xor_sync(kFull, vals[i], 16);   // same column, other slot of this load
+        const uint32_t above = half ? other : other_prev;             // the slot before this one
+        const uint32_t eq = __ballot_sync(kFull, vals[i] == above);
+        const uint32_t lt = __ballot_sync(kFull, above < vals[i]);
+        if (lane == i) { my_eq = eq; my_lt = lt; }
+        other_prev = other;
       }
-      // this lane's row is slot lane + 1: its m outcome bits start at bit (lane + 1) m
-      const int bitpos = (lane + 1) * m, wi = bitpos >> 5, sh = bitpos & 31;
-      const uint32_t e0 = __shfl_sync(kFull, my_eq, wi), e1 = __shfl_sync(kFull, my_eq, (wi + 1) & 31);
-      const uint32_t l0 = __shfl_sync(kFull, my_lt, wi), l1 = __shfl_sync(kFull, my_lt, (wi + 1) & 31);
-      const uint32_t eqf = (uint32_t)((((unsigned long long)e1 << 32) | e0) >> sh);
-      const uint32_t ltf = (uint32_t)((((unsigned long long)l1 << 32) | l0) >> sh);
-      int lcp = __ffs((int)(~eqf | (1u << m))) - 1;      // leading equal columns, at most m
+      // this lane's row is slot lane + 1: load (lane + 1) / 2, upper half of the word when odd
+      const int slot = lane + 1, sh = (slot & 1) << 4;
+      const uint32_t eqf = (__shfl_sync(kFull, my_eq, slot >> 1) >> sh) & 0xFFFFu;
+      const uint32_t ltf = (__shfl_sync(kFull, my_lt, slot >> 1) >> sh) & 0xFFFFu;
+      int lcp = __ffs((int)(~eqf | 0x10000u)) - 1;       // leading equal columns (padding never matches: at most lim)
       if (!valid || j == 0) lcp = 0;
       if (valid && j > 0) {
         // the first differing column decides the order; when one row is a prefix of the
@@ -704,10 +736,8 @@ rest_draft_kernel(DraftArgs a) {
       uint32_t myword = 0;
 #pragma unroll
       for (int d = 1; d <= kMaxM; ++d) {
-        if (d <= m) {
-          uint32_t w = __ballot_sync(kFull, !valid || lcp < d);
-          if (lane == d - 1) myword = w;
-        }
+        const uint32_t w = __ballot_sync(kFull, !valid || lcp < d);
+        if (lane == d - 1) myword = w;
       }
       if (lane < m) bm[lane * nwords + (jbase >> 5)] = myword;
       if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
@@ -779,7 +809,6 @@ rest_draft_kernel(DraftArgs a) {
 
   // ---- phase 3a: counts of the light nodes, histogram of the others ------------------------
   {
-    uint32_t nbig = 0;
     for (int item = tid; item < items; item += NT) {
       const int d = item / nw + 1, w = item - (d - 1) * nw;
       const WordNodes wn = word_nodes(d, w);
@@ -789,16 +818,20 @@ rest_draft_kernel(DraftArgs a) {
       const uint32_t* row = bm + (d - 1) * nwords;
       const uint16_t* jrow = jump + (d - 1) * nwords;
       uint32_t big = wn.big;
-      while (big) {
-        const int j = (w << 5) + __ffs(big) - 1;
-        big &= big - 1;
-        atomicAdd(&s.hist_hi[bin_of(next_set(row, jrow, j) - j)], 1u);
-        ++nbig;
+      if (big) {
+        // the word's heavy nodes also go into a list, which the later passes read instead of
+        // walking the bitmaps again (when it overflows they walk)
+        uint32_t at = atomicAdd(&s.big_total, (uint32_t)__popc(big));
+        while (big) {
+          const int j = (w << 5) + __ffs(big) - 1;
+          big &= big - 1;
+          const int c = next_set(row, jrow, j) - j;
+          atomicAdd(&s.hist_hi[bin_of(c)], 1u);
+          if (at < (uint32_t)a.bigcap) { big_dj[at] = ((uint32_t)d << 16) | (uint32_t)j; big_c[at] = (uint16_t)c; }
+          ++at;
+        }
       }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) nbig += __shfl_xor_sync(kFull, nbig, o);
-    if (lane == 0 && nbig) atomicAdd(&s.big_total, nbig);
   }
   __syncthreads();
 
@@ -807,10 +840,17 @@ rest_draft_kernel(DraftArgs a) {
   uint32_t r_tie = 0;  // plus the first r_tie nodes (by row) with key == tstar
   int c_tie = 0, d_tie = 0;
   const uint32_t big_total = s.big_total;
+  const bool listed = big_total <= (uint32_t)a.bigcap;     // the list holds every heavy node
   if (big_total >= (uint32_t)N) {
     if (warp == 0) warp_threshold_desc(s.hist_hi, kHistHi, (uint32_t)N, lane, &s.bin_hi, &s.above_hi);
     __syncthreads();
     const int bin_hi = s.bin_hi;
+    if (listed) {
+      for (uint32_t e = tid; e < big_total; e += NT) {
+        const int c = (int)big_c[e];
+        if (bin_of(c) == bin_hi) atomicAdd(&s.hist_lo[sub_of(c, (int)(big_dj[e] >> 16))], 1u);
+      }
+    } else
     for (int item = tid; item < items; item += NT) {
       const int d = item / nw + 1, w = item - (d - 1) * nw;
       uint32_t big = word_nodes(d, w).big;
@@ -865,6 +905,14 @@ rest_draft_kernel(DraftArgs a) {
     }
     return t;
   };
+  if (listed) {
+    for (uint32_t e = tid; e < big_total; e += NT) {
+      const int c = (int)big_c[e], d = (int)(big_dj[e] >> 16);
+      if (key_of(c, d) > tstar) keep(d, (int)(big_dj[e] & 0xFFFFu), c);
+    }
+  }
+  // the light nodes can only be wanted when the heavy ones do not fill the tree
+  if (!listed || tstar < key_of(5, kMaxM))
   for (int item = tid; item < items; item += NT) {
     const int d = item / nw + 1, w = item - (d - 1) * nw;
     const WordNodes wn = word_nodes(d, w);
@@ -880,7 +928,7 @@ rest_draft_kernel(DraftArgs a) {
     }
     const uint32_t* row = bm + (d - 1) * nwords;
     const uint16_t* jrow = jump + (d - 1) * nwords;
-    uint32_t big = wn.big;
+    uint32_t big = listed ? 0u : wn.big;
     while (big) {
       const int j = (w << 5) + __ffs(big) - 1;
       big &= big - 1;
@@ -936,17 +984,22 @@ rest_draft_kernel(DraftArgs a) {
     const int d = (int)(me >> 16), j = (int)(me & 0xFFFFu);
     int par = -1;
     if (d > 1) {
-      const int jp = prev_set(bm + (d - 2) * nwords, j);
-      const uint32_t pkey = ((uint32_t)(d - 1) << 16) | (uint32_t)jp;
-      int l = 0, r = nn - 1;
-      par = -2;
-      while (l <= r) {
-        int mid = (l + r) >> 1;
-        uint32_t v = s.sorted[mid];
-        if (v == pkey) { par = mid; break; }
-        if (v < pkey) l = mid + 1; else r = mid - 1;
+      // the parent is the node of depth d - 1 whose rows include row j: the kept set is closed
+      // under ancestors, so it is the last kept node (in breadth-first order) that starts at or
+      // before row j at depth d - 1
+      const uint32_t pmax = ((uint32_t)(d - 1) << 16) | (uint32_t)j;
+      int l = 0, r = nn;                   // first kept node whose key exceeds pmax
+      while (l < r) {
+        const int mid = (l + r) >> 1;
+        if (s.sorted[mid] <= pmax) l = mid + 1; else r = mid;
       }
-      if (par < 0) { atomicOr(&s.err, REST_CTX_INTERNAL); par = -1; }
+      par = l - 1;
+      bool ok = par >= 0 && (int)(s.sorted[par] >> 16) == d - 1;
+      if (ok) {                            // and no node of that depth may start between it and row j
+        const int jp = (int)(s.sorted[par] & 0xFFFFu);
+        ok = next_set(bm + (d - 2) * nwords, jump + (d - 2) * nwords, jp) > j;
+      }
+      if (!ok) { atomicOr(&s.err, REST_CTX_INTERNAL); par = -1; }
     }
     s.par[i] = par;
     int64_t p;
@@ -995,7 +1048,8 @@ rest_draft_kernel(DraftArgs a) {
 
 // Dynamic shared memory of a block of `threads` threads that builds trees from up to K rows of
 // m tokens (the search-only launch needs sizeof(Smem) alone).
-size_t draft_smem_bytes(int K, int m, int threads, int* kcap_out, int* nwords_out, int* pcache_out) {
+size_t draft_smem_bytes(int K, int m, int threads, int* kcap_out, int* nwords_out, int* pcache_out,
+                        int* bigcap_out) {
   const int kcap = (K + 31) / 32 * 32;
   const int nwords = kcap / 32 + 1;
   const int warps = threads / 32;
@@ -1003,13 +1057,17 @@ size_t draft_smem_bytes(int K, int m, int threads, int* kcap_out, int* nwords_ou
   if (kcap_out) *kcap_out = kcap;
   if (nwords_out) *nwords_out = nwords;
   if (pcache_out) *pcache_out = pcache_rows;
+  // every fifth row at most starts a node of weight >= 5 at a depth
+  const int bigcap = kcap < kBigListCap ? kcap : kBigListCap;
+  if (bigcap_out) *bigcap_out = bigcap;
   size_t bytes = sizeof(Smem);
   bytes += (size_t)warps * 34 * 8;                         // slots: start positions
   bytes += (size_t)pcache_rows * 8;                        // suffix positions of the first rows
-  bytes += (size_t)warps * 66 * 4;                         // slots: lengths and comparable lengths
+  bytes += (size_t)warps * 34 * 4;                         // slots: lengths
   bytes += (size_t)m * nwords * 4;                         // node-start bitmaps
   bytes += (size_t)m * nwords * 2;                         // jump tables
   bytes += (size_t)nwords * 2;                             // tie counts
+  bytes += (size_t)bigcap * 6;                             // list of the heavy nodes
   return (bytes + 15) / 16 * 16;
 }
 
@@ -1073,14 +1131,14 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   a.mask = d_mask; a.n_nodes = d_n_nodes; a.match_n = d_match_n; a.match_range = d_match_range;
   a.node_count = d_node_count; a.status = d_status;
   a.idx = ds->v.idx;
-  auto smem_for = [&](int K, int threads) { return draft_smem_bytes(K, prm->m, threads, &a.kcap, &a.nwords, &a.pcache_rows); };
+  auto smem_for = [&](int K, int threads) { return draft_smem_bytes(K, prm->m, threads, &a.kcap, &a.nwords, &a.pcache_rows, &a.bigcap); };
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool with_scratch = d_ws && ws_bytes >= split_workspace_bytes(B);
   bool batched = false;
   if (rest_status rc = wants_batched(search, B, with_scratch, &batched); rc != REST_OK) return rc;
   const bool narrow = ds->v.sa_bytes == 4;
   a.list = nullptr; a.list_count = nullptr; a.B = B; a.which = 0; a.light_rows = 0;
-  a.kcap = 0; a.nwords = 0; a.pcache_rows = 0;
+  a.kcap = 0; a.nwords = 0; a.pcache_rows = 0; a.bigcap = 0;
   auto launch = [&](auto kern, int slot, int threads, int blocks, size_t bytes) -> rest_status {
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
                                             rest::kSmemSlotDraft + slot + (narrow ? 0 : 1), bytes));
@@ -1272,7 +1330,7 @@ extern "C" rest_status rest_draft_from_runs(const rest_draft_params* prm, const 
   a.n_nodes = d_n_nodes; a.node_count = d_node_count; a.status = d_status; a.B = B;
   const bool big = (size_t)a.K * prm->m >= kBigRowsTimesM;
   const int threads = big ? kBigThreads : kThreads;
-  const size_t smem = draft_smem_bytes(a.K, prm->m, threads, &a.kcap, &a.nwords, &a.pcache_rows);
+  const size_t smem = draft_smem_bytes(a.K, prm->m, threads, &a.kcap, &a.nwords, &a.pcache_rows, &a.bigcap);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (big) {
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(rest_draft_kernel<int32_t, false, kBigThreads, kFromRuns>),
