@@ -61,6 +61,13 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-workloads", action="store_true",
                     help="skip the table of the other workloads and the sweeps")
+    ap.add_argument("--part", default="step", choices=["step", "draft", "attention"],
+                    help="time one call alone on a (possibly reduced) case and print its record: what "
+                         "the ncu captures under profiles/ run")
+    ap.add_argument("--batch", type=int, default=None, help="--part draft: contexts per call")
+    ap.add_argument("--max-gb", type=float, default=80.0,
+                    help="--part attention: cap on the K/V bytes (the batch is cut to fit)")
+    ap.add_argument("--iters", type=int, default=12, help="--part: timed calls")
     return ap.parse_args()
 
 
@@ -854,6 +861,29 @@ def other_workloads(rest, torch, dev, headline, headline_T, headline_ds, headlin
     return rows, sweeps
 
 
+def run_part(args):
+    """One call alone, on workload --workload (default stress), possibly reduced: the draft over a
+    datastore of --n-tokens tokens with --batch contexts, or the attention layer with its batch
+    cut to --max-gb of K/V.  Prints one JSON record."""
+    import torch
+    import paper_2311_08252_b200 as rest
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peak, peak_kind = measured_peaks()
+    w = datagen.WORKLOADS["stress" if args.workload == "auto" else args.workload]
+    if args.n_tokens is not None:
+        w = w.scaled(n_tokens=args.n_tokens)
+    if args.part == "draft":
+        T, d_T, d_sa, ds, setup = device_datastore(rest, torch, w, dev)
+        rec = time_draft(rest, torch, ds, w, T, args.batch or w.B, dev, iters=args.iters, peak=peak)
+        rec.update(setup)
+    else:
+        rec = time_attention(rest, torch, w, dev, iters=args.iters, peak=peak, budget_gb=args.max_gb)
+    rec.update({"part": args.part, "workload": w.name, "datastore_tokens": w.n_tokens, "peak_gbs": peak,
+                "peak_kind": peak_kind, "device_error_flags": rest.device_error_flags()})
+    print(json.dumps(rec))
+
+
 def spawn_ranks(args):
     """`bench.py --gpus N` started plainly (no launcher in the environment): start the N ranks
     through torch.distributed.run and pass their output through."""
@@ -872,6 +902,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.part != "step":
+        run_part(args)
         return
     run_ours(args, rank, world, local_rank)
 
