@@ -127,9 +127,10 @@ __device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* _
 // First slot in [lo, hi) whose comparison is >= 0 (STRICT = false) or > 0 (STRICT = true);
 // hi when there is none.  Warp-cooperative; all lanes return the same value.  `eq` reports
 // whether the returned slot compared equal (in: whether slot `hi` is known to compare equal).
-// `next_gt` (STRICT = false only): the first slot that compares greater, when the last round's
-// probes happen to show it (the run of equal slots ends inside the last 32 probed slots, or runs
-// up to a slot already known to be greater); -1 when it is not known.
+// `run` (STRICT = false only): what the probes of the search tell about the END of the run of
+// equal slots, for free: run[0] = the last probed slot that compared equal (-1: none), run[1] =
+// the first probed slot that compared greater (in: the slot the search may assume greater,
+// normally hi).  The first slot that compares greater lies in (run[0], run[1]].
 //
 // A = 32: every round all 32 lanes probe (fewest dependent rounds: the single-context path).
 // A < 32: only the first WIDE rounds are 32 wide (a search over the whole array: their probe
@@ -139,7 +140,7 @@ __device__ __forceinline__ int probe(const int32_t* __restrict__ T, const SaT* _
 template <typename SaT, bool STRICT, int A = 32, int WIDE = kWideRounds>
 __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __restrict__ sa,
                                    int64_t n_tokens, int64_t lo, int64_t hi, const int (&q)[16],
-                                   int n, int lane, bool& eq, bool& bad, int64_t* next_gt = nullptr) {
+                                   int n, int lane, bool& eq, bool& bad, int64_t* run = nullptr) {
   // floor(2^64 / (A + 1))
   constexpr unsigned long long kInv = A == 32 ? 0x07C1F07C1F07C1F0ull : ~0ull / (unsigned long long)(A + 1);
   int round = 0;
@@ -158,6 +159,13 @@ __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __r
     if (lane <= last) c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
     bool t = STRICT ? (c > 0) : (c >= 0);
     unsigned b = __ballot_sync(kFull, t && lane <= last);
+    if (!STRICT && run) {
+      // outcomes are monotone along the probes: smaller ... equal ... greater
+      const unsigned eqb = __ballot_sync(kFull, c == 0 && lane <= last);
+      const unsigned gtb = __ballot_sync(kFull, c > 0 && lane <= last);
+      if (eqb) run[0] = max(run[0], __shfl_sync(kFull, pos, 31 - __clz(eqb)));
+      if (gtb) run[1] = min(run[1], __shfl_sync(kFull, pos, __ffs(gtb) - 1));
+    }
     if (b == 0) {
       lo = __shfl_sync(kFull, pos, last) + 1;
     } else {
@@ -175,10 +183,11 @@ __device__ int64_t warp_first_true(const int32_t* __restrict__ T, const SaT* __r
   if (pos < hi) c = probe<SaT>(T, sa, n_tokens, pos, q, n, bad);
   bool t = (pos < hi) && (STRICT ? (c > 0) : (c >= 0));
   unsigned b = __ballot_sync(kFull, t);
-  if (!STRICT && next_gt) {
-    // slot hi compares greater unless `eq` says it is equal (hi = end of the array counts as greater)
-    const unsigned gt = __ballot_sync(kFull, (pos < hi) && c > 0);
-    *next_gt = gt ? lo + (__ffs(gt) - 1) : (eq ? (int64_t)-1 : hi);
+  if (!STRICT && run) {
+    const unsigned eqb = __ballot_sync(kFull, (pos < hi) && c == 0);
+    const unsigned gtb = __ballot_sync(kFull, (pos < hi) && c > 0);
+    if (eqb) run[0] = max(run[0], lo + (int64_t)(31 - __clz(eqb)));
+    if (gtb) run[1] = min(run[1], lo + (int64_t)(__ffs(gtb) - 1));
   }
   if (b != 0) {
     int f = __ffs(b) - 1;
@@ -234,7 +243,7 @@ __device__ void warp_threshold_desc(const uint32_t* hist, int nbins, uint32_t ne
 struct Smem {
   int q[16];
   long long lb[17], ub[17];
-  long long bhi[17];           // end of the range the lower bound of each length was searched in
+  long long ub_from[17];       // >= 0: ub[n] is only known to lie in (ub_from[n] - 1, ub[n]]
   uint32_t small[5][kMaxM + 1];   // [c][d]: nodes of weight c = 1 ... 4 at depth d
   uint32_t big_total;          // nodes of weight >= 5
   int err;
@@ -244,7 +253,6 @@ struct Smem {
   uint32_t above_lo;
   uint32_t nsel;
   int ntrunc;
-  int warp_first[32];          // block-wide searches: first probe of each warp that compared greater
   uint32_t trunc[kMaxTrunc];   // len << 16 | row: rows cut short by the end of the token stream
   uint32_t sel[kMaxN];         // depth << 16 | row
   uint32_t selcnt[kMaxN];
@@ -375,7 +383,7 @@ rest_draft_kernel(DraftArgs a) {
   if constexpr (PART == kWhole || PART == kSearch || PART == kFromRuns) write_defaults();
   const int nq = min(a.n_max, max(clen, 0));   // context tokens that can take part
   if (tid == 0) { s.err = 0; s.big_total = 0; s.nsel = 0; s.ntrunc = 0; }
-  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; s.bhi[tid] = n_sa; }
+  if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; s.ub_from[tid] = -1; }
   if (tid < 5 * (kMaxM + 1)) (&s.small[0][0])[tid] = 0;
   if constexpr (PART != kSearch && PART != kRetrieve) {
     for (int i = tid; i < kHistHi; i += NT) s.hist_hi[i] = 0;
@@ -441,8 +449,7 @@ rest_draft_kernel(DraftArgs a) {
   }
 
   // ---- phase 1: search --------------------------------------------------------------
-  // 1a: lower bound of every suffix length, one warp each.  ub = -1 marks "matches, end of the
-  // run not known yet".
+  // the range of every suffix length, one warp each (lb = ub: no match)
   constexpr int kArity = TP ? kTpArity : 32;
   const bool have_index = index_unusable == 0u;
   auto lower_bound_of = [&](int n) {     // executed by one whole warp
@@ -450,7 +457,21 @@ rest_draft_kernel(DraftArgs a) {
 #pragma unroll
     for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
     bool bad = false, eq = false;
-    int64_t next_gt = -1, lb;
+    int64_t lb;
+    // the end of the run of matches: first slot after lb that compares greater.  The probes of
+    // the lower bound bracket it for free (last probed slot seen equal, first seen greater).
+    // Only the longest matching length needs its end, so a bracket that is not settled yet is
+    // left as it is: the search inside it runs after the barrier, for the winner alone.
+    auto finish = [&](int64_t lb_, int64_t end, int64_t (&run)[2]) {
+      if (lane != 0) return;
+      s.lb[n] = lb_;
+      s.ub[n] = lb_;                       // no match: empty range
+      if (eq && lb_ < end) {
+        const int64_t from = (run[0] > lb_ ? run[0] : lb_) + 1;
+        s.ub[n] = run[1];                  // > lb_: a match
+        if (from < run[1]) s.ub_from[n] = from;
+      }
+    };
     if (have_index) {
       // every suffix that starts with the query's first token lies in [f0, f1); when the index
       // also stores the query's first two, three or four tokens, every suffix that starts with
@@ -459,24 +480,25 @@ rest_draft_kernel(DraftArgs a) {
       lo0 = lo0 < 0 ? 0 : (lo0 > n_sa ? n_sa : lo0);
       hi0 = hi0 < lo0 ? lo0 : (hi0 > n_sa ? n_sa : hi0);
       if (n == 1) {                       // the first-token range is the answer
-        if (lane == 0) { s.lb[1] = lo0; s.ub[1] = hi0; s.bhi[1] = hi0; }
+        if (lane == 0) { s.lb[1] = lo0; s.ub[1] = hi0; }
         return;
       }
       int64_t plo = 0, phi = 0;
       const int found = index_ngram_range(a.idx, q, n, lane, n_sa, plo, phi);
       if (found > 0 && plo >= lo0 && phi <= hi0) {
         if (found == n) {                 // the n-gram's own range is the answer
-          if (lane == 0) { s.lb[n] = plo; s.ub[n] = phi; s.bhi[n] = phi; }
+          if (lane == 0) { s.lb[n] = plo; s.ub[n] = phi; }
           return;
         }
         lo0 = plo; hi0 = phi;
       }
-      if (lane == 0) s.bhi[n] = hi0;
-      lb = warp_first_true<SaT, false, kArity, 0>(T, sa, n_tokens, lo0, hi0, q, n, lane, eq, bad, &next_gt);
-      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < hi0) ? next_gt : lb; }
+      int64_t run[2] = {-1, hi0};
+      lb = warp_first_true<SaT, false, kArity, 0>(T, sa, n_tokens, lo0, hi0, q, n, lane, eq, bad, run);
+      finish(lb, hi0, run);
     } else {
-      lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_sa, q, n, lane, eq, bad, &next_gt);
-      if (lane == 0) { s.lb[n] = lb; s.ub[n] = (eq && lb < n_sa) ? next_gt : lb; }
+      int64_t run[2] = {-1, n_sa};
+      lb = warp_first_true<SaT, false, kArity>(T, sa, n_tokens, 0, n_sa, q, n, lane, eq, bad, run);
+      finish(lb, n_sa, run);
     }
     if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
   };
@@ -507,70 +529,20 @@ rest_draft_kernel(DraftArgs a) {
   __syncthreads();
   for (int n = nq; n >= a.n_min; --n)
     if (s.ub[n] != s.lb[n]) { n_win = n; break; }
-  // 1b: only the winning length needs its upper bound, and only if the last round of its lower
-  // bound did not already show where the run ends.  The block searches: in the first round
-  // half of the probing threads look at the slots right behind the first match one by one and
-  // the other half at geometrically growing distances (so a short run is settled in one round
-  // whatever the size of the range); the rounds after that cut what is left into NT + 1 parts.
-  if (n_win != 0 && s.ub[n_win] < 0) {       // block-uniform
-    const int n = n_win;
-    int q[16];
+  if (n_win != 0 && s.ub_from[n_win] >= 0) {     // the same for the whole block
+    // the end of the winner's run: first slot in [ub_from, ub) that compares greater, else ub
+    // (the new ub is above lb like the old one, so warps still picking n_win read the same answer)
+    if (warp == 0) {
+      int q[16];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) q[k] = (k < n) ? s.q[nq - n + k] : 0;
-    bool bad = false;
-    const int64_t end = s.bhi[n];            // slots from here on are known to compare greater
-    int64_t lo2 = s.lb[n] + 1, hi2 = end;    // the answer lies in [lo2, hi2]
-    // A probe reads n tokens from a random place, so the first round uses fewer threads the
-    // longer the suffix (most runs are a handful of slots long and end inside its linear part);
-    // the geometric probes use as many steps per octave as cover the range that is left (the
-    // finer the steps, the smaller the bracket the second round has to settle).
-    const int P1 = min(NT, max(64, (2048 / n) & ~31));
-    const int H = P1 / 2;
-    int octaves = 1;
-    while (octaves < 44 && ((int64_t)H << octaves) < end - lo2) ++octaves;
-    const int S = max(1, (P1 - H) / octaves);
-    auto first_round_pos = [&](int t) -> int64_t {
-      if (t < H) return lo2 + t;
-      const int e = t - H + 1, oct = e / S, frac = e - oct * S;
-      if (oct > 44) return (int64_t)1 << 60;
-      const int64_t base = (int64_t)H << oct;
-      return lo2 + base + base * frac / S - 1;
-    };
-    bool first = true;
-    while (hi2 > lo2) {                      // block-uniform
-      const int64_t size = hi2 - lo2;
-      const bool exact = !first && size <= NT;            // one probe per remaining slot
-      auto pos_of = [&](int t) -> int64_t {
-        if (first) return first_round_pos(t);
-        if (exact) return lo2 + t;
-        return lo2 + (int64_t)(((unsigned long long)(t + 1) * (unsigned long long)size) / (unsigned long long)(NT + 1));
-      };
-      const int width = first ? P1 : NT;                  // threads that probe in this round
-      bool t = false;
-      if (tid < width) {
-        const int64_t pos = pos_of(tid);
-        t = true;                                         // slots from hi2 on compare greater
-        if (pos < hi2) t = probe<SaT>(T, sa, n_tokens, pos, q, n, bad) > 0;
-      }
-      const unsigned bal = __ballot_sync(kFull, t);
-      if (lane == 0) s.warp_first[warp] = bal ? warp * 32 + __ffs(bal) - 1 : 0x7FFFFFFF;
-      __syncthreads();
-      int tf = 0x7FFFFFFF;
-      for (int w = 0; w < NW; ++w) tf = min(tf, s.warp_first[w]);
-      __syncthreads();
-      if (tf == 0x7FFFFFFF) {
-        lo2 = pos_of(width - 1) + 1;
-        if (lo2 > hi2) lo2 = hi2;
-      } else {
-        const int64_t pf = pos_of(tf);
-        const int64_t nlo = tf > 0 ? pos_of(tf - 1) + 1 : lo2;
-        hi2 = pf < hi2 ? pf : hi2;
-        lo2 = nlo < hi2 ? nlo : hi2;
-      }
-      first = false;
+      for (int k = 0; k < 16; ++k) q[k] = (k < n_win) ? s.q[nq - n_win + k] : 0;
+      bool bad = false, eq = false;
+      const int64_t ub = warp_first_true<SaT, true, kArity, 0>(T, sa, n_tokens, s.ub_from[n_win], s.ub[n_win],
+                                                                q, n_win, lane, eq, bad);
+      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
+      __syncwarp();
+      if (lane == 0) s.ub[n_win] = ub;
     }
-    if (bad) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
-    if (tid == 0) s.ub[n] = hi2;
     __syncthreads();
   }
   if (s.err != 0 || n_win == 0) {
