@@ -18,8 +18,8 @@ cudaError_t ensure_dynamic_smem(const void* kernel, int kernel_slot, size_t byte
 // usable device.
 int sm_count();
 // One slot per kernel instance, library-wide: two kernels on one slot would skip each other's
-// attribute call.  The draft kernel's instances take kSmemSlotDraft + 0 ... 15.
-constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 16, kSmemSlotAttnWide = 17, kSmemSlots = 18;
+// attribute call.  The draft kernel's instances take kSmemSlotDraft + 0 ... 19.
+constexpr int kSmemSlotDraft = 0, kSmemSlotAttn = 20, kSmemSlotAttnWide = 21, kSmemSlots = 22;
 
 #define REST_CUDA_TRY(expr)                                              \
   do {                                                                   \

@@ -96,7 +96,60 @@ struct DraftArgs {
   int B;
   int which;              // list of this build launch
   int light_rows;         // candidate counts up to this go to list 0
+  // one-launch form with shared gathering (kWholeShare): see ShareDesc
+  int32_t* sh_hdr = nullptr;        // counters, zeroed before the launch like sh_ready and sh_desc
+  int32_t* sh_ready = nullptr;      // [B] 0: not offered, 1: chunks to claim, 2: all claimed
+  struct ShareDesc* sh_desc = nullptr;   // [B]
+  uint32_t* sh_trunc = nullptr;     // [B][kMaxTrunc]
+  uint32_t* sh_bm = nullptr;        // [B][m][nwords]
+  int share_rows = 0;         // a context with more candidates than this offers its gather to other blocks
 };
+
+// Shared gathering.  In a call with few contexts a call lasts as long as its slowest context, and
+// what makes a context slow is a long candidate list, whose rows one block reads alone while the
+// blocks of the other contexts have finished and other SMs never had a block.  So a context
+// with many candidates publishes its matched range, and every warp that has nothing else to do
+// - the owner's own warps, the warps of blocks whose own rows are read or whose context is
+// finished, the warps of blocks launched as helpers only - claims bitmap words (32 rows each)
+// from the context's counter, computes them into the scratch and counts them done.  The owner
+// waits only for words that some running warp has claimed (unclaimed ones it takes itself),
+// then reads the bitmaps back and goes on alone.  Nothing depends on a helper being there:
+// helpers that find nothing to do leave.
+struct ShareDesc {
+  long long lo, cnt;       // matched suffix-array range
+  int Kp, n_win, nw;       // rows taken, matched length, bitmap words that hold rows
+  int next;                // next word to claim (atomic)
+  int done;                // words finished (atomic)
+  int ntrunc;              // rows cut short by the end of the stream (atomic), listed in the context's trunc array
+  int err;                 // REST_CTX_* bits met by the gatherers (atomic)
+  int pad[5];
+};
+static_assert(sizeof(ShareDesc) == 64, "one descriptor per 64 bytes");
+constexpr int kShareRows = 512;         // candidate caps up to this never share (a block has a warp per word)
+// a single context does not share: the few microseconds that zeroing the counters and the look-outs
+// cost every call outweigh what the occasional long list gains
+constexpr int kShareMinContexts = 2;
+constexpr int kShareMaxContexts = 1024;  // calls with more contexts do not share (and take the batched path anyway)
+constexpr int kShareHdr = 16;           // int32 counters ahead of the per-context arrays: [0] blocks started, [1] contexts past their gather
+constexpr int kHelperPolls = 20000;     // idle polls (>= 200 ns each) after which a helper leaves
+constexpr int kOwnerPolls = 1 << 20;    // polls after which an owner gives up on claimed chunks (REST_CTX_INTERNAL)
+
+// Scratch of the shared gather for B contexts: counters, a state word and a descriptor per
+// context (this part is zeroed before every launch), then the lists of short rows and the bitmaps.
+struct ShareLayout {
+  size_t ready, desc, zeroed_bytes, trunc, bm, bytes;     // byte offsets
+};
+static ShareLayout share_layout(int B, int m, int nwords) {
+  ShareLayout l;
+  const size_t bpad = ((size_t)B + 31) / 32 * 32;
+  l.ready = kShareHdr * sizeof(int32_t);
+  l.desc = l.ready + bpad * sizeof(int32_t);
+  l.zeroed_bytes = l.desc + (size_t)B * sizeof(ShareDesc);
+  l.trunc = l.zeroed_bytes;
+  l.bm = l.trunc + (size_t)B * kMaxTrunc * sizeof(uint32_t);
+  l.bytes = l.bm + (size_t)B * m * nwords * sizeof(uint32_t);
+  return l;
+}
 
 // Three-way comparison of the first n tokens of the suffix stored in slot `slot` with q.
 // -1 / 0 / +1; a suffix that ends early is smaller.  An out-of-range suffix-array entry
@@ -253,6 +306,9 @@ struct Smem {
   uint32_t above_lo;
   uint32_t nsel;
   int ntrunc;
+  int counted;                 // shared gathering: this context is counted as past its gather
+  int help_b;                  // shared gathering: the context this block helps next
+  int help_base;               // shared gathering: first word of the block's current claim
   uint32_t trunc[kMaxTrunc];   // len << 16 | row: rows cut short by the end of the token stream
   uint32_t sel[kMaxN];         // depth << 16 | row
   uint32_t selcnt[kMaxN];
@@ -310,8 +366,9 @@ __device__ __forceinline__ uint32_t cut_short_mask(const Smem& s, int ntrunc, in
 // match_range, the defaults of every output slot, and the context's index into one of two
 // lists); kBuild = phases 2-4 for the contexts of one list; kRetrieve = phase 1 alone, nothing
 // but match_n, match_range and status written (rest_retrieve); kFromRuns = phases 2-4 over rows
-// that the caller hands in as sorted runs, merged first (rest_draft_from_runs).
-enum { kWhole = 0, kSearch = 1, kBuild = 2, kRetrieve = 3, kFromRuns = 4 };
+// that the caller hands in as sorted runs, merged first (rest_draft_from_runs); kWholeShare =
+// kWhole with shared gathering (see ShareDesc; the grid may hold more blocks than contexts).
+enum { kWhole = 0, kSearch = 1, kBuild = 2, kRetrieve = 3, kFromRuns = 4, kWholeShare = 5 };
 
 // Three-way comparison of two candidate rows (tokens as unsigned integers; a row that is a
 // proper prefix of the other sorts first).
@@ -323,12 +380,264 @@ __device__ __forceinline__ int compare_rows(const int32_t* __restrict__ y, int y
   }
   return ylen == xlen ? 0 : (ylen < xlen ? -1 : 1);
 }
+// ---- gather rows, common-prefix lengths, node-start bitmap words -----------------------------
+// Executed by one warp, for the context whose matched range is [lo, lo + cnt), of which Kp rows
+// are taken, behind a match of n_win tokens.  Bitmap word w covers candidate rows 32 w ... 32 w + 31;
+// the warp takes words first_word, first_word + stepw, ... below end_word.  The suffix-array
+// entries of the warp's next word travel while the rows of the current one do.
+// Slot 0 of the warp is the row before its first row, slot l + 1 the row of lane l.  A load
+// instruction fetches two slots, 16 columns each (lane = 16 * slot parity + column): the
+// lanes of a row read consecutive tokens, so an instruction touches two rows (a few cache
+// lines) instead of 32.  A token is compared with the token above it (the same column of the
+// slot before: the other half-warp of the same load, or of the load before) right where it
+// sits; a ballot turns the "equal" and "smaller" outcomes of each load into bit strings, and
+// lane l cuts the 16 bits of its row out of them: the number of leading equal columns is the
+// common prefix.
+// sb, sl: the warp's slot tables (34 entries each).  bm_out[d * a.nwords + w]: the words.  Rows
+// cut short by the end of the stream are appended to trunc_out (counter ntrunc_out), problems
+// OR-ed into err_out (all three in shared or global memory); pc[j], j < pc_rows, receives the
+// suffix position of row j.
+template <typename SaT, int PART>
+__device__ __forceinline__ void gather_words(const DraftArgs& a, int b, const int32_t** sb, int* sl, int lane,
+                                             int64_t lo, int64_t cnt, int Kp, int n_win, int first_word,
+                                             int stepw, int end_word, uint32_t* bm_out, int* ntrunc_out,
+                                             uint32_t* trunc_out, int* err_out, long long* pc, int pc_rows) {
+  const int m = a.m, nwords = a.nwords;
+  const int nw = end_word;
+  const int64_t n_tokens = a.n_tokens;
+  const SaT* __restrict__ sa = static_cast<const SaT*>(a.sa);
+  // where the rows' tokens live: the token stream, or the caller's rows of this context
+  const int32_t* __restrict__ Trow = PART == kFromRuns ? a.T + (int64_t)b * a.R * a.Kr * m : a.T;
+  // where row j comes from: the suffix-array entry of its sampled slot lo + floor(j cnt / K), or
+  // (rows handed in as runs) its place in the caller's row array, through the merged order.
+  // floor(j cnt / K) = j floor(cnt / K) + floor(j (cnt mod K) / K), and j (cnt mod K) < 2^30: one
+  // 64-bit division per context, a 32-bit one per row.
+  const uint32_t* ord = PART == kFromRuns ? a.order + (int64_t)b * a.kcap : nullptr;
+  const bool strided = PART != kFromRuns && cnt > (int64_t)a.K && a.sample_mode == REST_SAMPLE_STRIDED;
+  const uint32_t uK = (uint32_t)a.K;
+  const unsigned long long q1 = strided ? (unsigned long long)cnt / uK : 1ull;
+  const uint32_t r1 = strided ? (uint32_t)((unsigned long long)cnt % uK) : 0u;
+  auto entry_of = [&](int j) -> int64_t {
+    if constexpr (PART == kFromRuns) return (int64_t)ord[j];
+    else return (int64_t)__ldg(sa + lo + (int64_t)((unsigned long long)j * q1 + (unsigned long long)(((uint32_t)j * r1) / uK)));
+  };
+  // start of the row's tokens (relative to Trow) and its length; `bad` when the entry is out of range
+  auto row_place = [&](int64_t& p, int64_t& base, int& len, bool& bad) {
+    if constexpr (PART == kFromRuns) {
+      if (p < 0 || p >= (int64_t)a.R * a.Kr) { bad = true; p = 0; }
+      len = bad ? 0 : min(max(a.row_len[(int64_t)b * a.R * a.Kr + p], 0), m);
+      p *= m;
+      base = p;
+    } else {
+      if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
+      base = p + n_win;
+      const int64_t rem_t = n_tokens - base;
+      len = bad ? 0 : (int)(rem_t < 0 ? 0 : (rem_t > m ? m : rem_t));
+    }
+  };
+  // the entries of word w: this lane's row, and (lane 0) the row before the word
+  auto entries_of = [&](int w, int64_t& p, int64_t& pp) {
+    p = 0; pp = 0;
+    if (w >= nw) return;
+    const int j = w * 32 + lane;
+    if (j < Kp) p = entry_of(j);
+    if (lane == 0 && w > 0) pp = entry_of(w * 32 - 1);
+  };
+  int w = first_word;
+  int64_t p = 0, pp = 0;
+  entries_of(w, p, pp);
+  const int half = lane >> 4, col = lane & 15;
+  if (lane == 0) { sl[33] = 0; sb[33] = Trow; }     // slot 33 does not exist
+  // columns past a row's end read as a value no token has (tokens are below 2^31), different
+  // for neighbouring slots: they never compare equal to anything above or below them
+  const uint32_t pad = 0x80000000u | (uint32_t)half;
+  while (w < nw) {
+    const int jbase = w * 32;
+    const int j = jbase + lane;
+    const bool valid = j < Kp;
+    bool bad = false;
+    int len = 0;
+    int64_t base = 0;
+    if (valid) {
+      row_place(p, base, len, bad);
+      if (j < pc_rows) pc[j] = p;
+    }
+    int plen = __shfl_up_sync(kFull, len, 1);
+    if (lane == 0) {
+      plen = 0;
+      int64_t pbase = 0;
+      if (j > 0) row_place(pp, pbase, plen, bad);   // the row before belongs to another warp
+      sb[0] = Trow + pbase; sl[0] = plen;
+    }
+    const int lim = min(len, plen);
+    sb[lane + 1] = Trow + base; sl[lane + 1] = len;
+    __syncwarp();
+    uint32_t vals[kRowLoads];
+#pragma unroll
+    for (int i = 0; i < kRowLoads; ++i) {
+      const int r = 2 * i + half;
+      vals[i] = col < sl[r] ? (uint32_t)__ldg(sb[r] + col) : pad;
+    }
+    // the next word's suffix-array entries travel while this word's rows do
+    const int wn = w + stepw;
+    int64_t p_next, pp_next;
+    entries_of(wn, p_next, pp_next);
+    uint32_t my_eq = 0, my_lt = 0, other_prev = 0;     // lane i keeps the bit strings of load i
+#pragma unroll
+    for (int i = 0; i < kRowLoads; ++i) {
+      const uint32_t other = __shfl_xor_sync(kFull, vals[i], 16);   // same column, other slot of this load
+      const uint32_t above = half ? other : other_prev;             // the slot before this one
+      const uint32_t eq = __ballot_sync(kFull, vals[i] == above);
+      const uint32_t lt = __ballot_sync(kFull, above < vals[i]);
+      if (lane == i) { my_eq = eq; my_lt = lt; }
+      other_prev = other;
+    }
+    // this lane's row is slot lane + 1: load (lane + 1) / 2, upper half of the word when odd
+    const int slot = lane + 1, sh = (slot & 1) << 4;
+    const uint32_t eqf = (__shfl_sync(kFull, my_eq, slot >> 1) >> sh) & 0xFFFFu;
+    const uint32_t ltf = (__shfl_sync(kFull, my_lt, slot >> 1) >> sh) & 0xFFFFu;
+    int lcp = __ffs((int)(~eqf | 0x10000u)) - 1;       // leading equal columns (padding never matches: at most lim)
+    if (!valid || j == 0) lcp = 0;
+    if (valid && j > 0) {
+      // the first differing column decides the order; when one row is a prefix of the
+      // other the shorter one must come first
+      const bool ordered = lcp < lim ? ((ltf >> lcp) & 1u) != 0u : plen <= len;
+      if (!ordered) bad = true;
+    }
+    if (valid && len < m) {        // cut short by the end of the stream: at most m such rows exist
+      const int at = atomicAdd(ntrunc_out, 1);
+      if (at < kMaxTrunc) trunc_out[at] = ((uint32_t)len << 16) | (uint32_t)j;
+      else atomicOr(err_out, REST_CTX_INTERNAL);
+    }
+    uint32_t myword = 0;
+#pragma unroll
+    for (int d = 1; d <= kMaxM; ++d) {
+      const uint32_t wd = __ballot_sync(kFull, !valid || lcp < d);
+      if (lane == d - 1) myword = wd;
+    }
+    if (lane < m) bm_out[lane * nwords + w] = myword;
+    if (__any_sync(kFull, bad) && lane == 0) atomicOr(err_out, REST_CTX_BAD_DATASTORE);
+    __syncwarp();                  // the slot tables are rewritten by the next word
+    w = wn; p = p_next; pp = pp_next;
+  }
+}
+
+// Executed by a whole block: claims words of context hb's candidate rows, one per warp and
+// round, until none is left; computes them into the context's scratch and counts them done.
+// (One claim per block and round: thousands of warps claiming from one counter wait for one
+// another longer than the rows take.)
+template <typename SaT, int NT>
+__device__ __forceinline__ void share_work_on(const DraftArgs& a, Smem& s, int hb, const int32_t** sb, int* sl,
+                                              int64_t lo, int64_t cnt, int Kp, int n_win) {
+  constexpr int NW = NT / 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  ShareDesc* dsc = a.sh_desc + hb;
+  const int nw = (Kp + 31) >> 5;
+  int finished = 0;                      // words of the round before, not yet counted
+  for (;;) {
+    if (tid == 0) {
+      if (finished) atomicAdd(&dsc->done, finished);
+      s.help_base = atomicAdd(&dsc->next, NW);
+    }
+    __syncthreads();
+    const int base = s.help_base;
+    if (base >= nw) break;
+    const int end = min(nw, base + NW);
+    gather_words<SaT, kWholeShare>(a, hb, sb, sl, lane, lo, cnt, Kp, n_win, base + warp, NW, end,
+                                   a.sh_bm + (int64_t)hb * a.m * a.nwords, &dsc->ntrunc,
+                                   a.sh_trunc + (int64_t)hb * kMaxTrunc, &dsc->err, nullptr, 0);
+    __threadfence();                     // the words before the count
+    __syncthreads();
+    finished = end - base;
+  }
+  if (tid == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + hb) = 2;     // every word is claimed
+  __syncthreads();                       // help_base is read by all before anyone rewrites it
+}
+
+// Executed by a whole block: works on the words that other contexts offer until none is left to
+// claim (no waiting).  `start`: where the block begins its look-out.  only_if_all_started: do
+// nothing while contexts of the launch still wait for an SM (this block had better finish and
+// make room).  Warp 0 looks out and claims (a context whose words are all claimed costs it one
+// read, no barrier); the block meets only over a claim that succeeded.
+template <typename SaT, int NT>
+__device__ __forceinline__ void share_help_pass(const DraftArgs& a, Smem& s, const int32_t** sb, int* sl, int start,
+                                                bool only_if_all_started) {
+  constexpr int NW = NT / 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int B = a.B, bpad = (B + 31) & ~31;
+  int cur = -1;                        // the context the block worked on last (its fields are still at hand)
+  int64_t lo = 0, cnt = 0;
+  int Kp = 0, n_win = 0, nw = 0;
+  int finished = 0;                    // words of the round before, not yet counted
+  bool allowed = !only_if_all_started;
+  for (;;) {
+    if (warp == 0) {
+      if (finished && lane == 0) atomicAdd(&a.sh_desc[cur].done, finished);
+      int found = -1, base = 0;
+      if (!allowed) allowed = *reinterpret_cast<volatile int32_t*>(a.sh_hdr) >= B;
+      int prefer = cur;
+      for (int tries = 0; allowed && tries <= B && found < 0; ++tries) {
+        int cand = prefer;
+        prefer = -1;
+        if (cand < 0) {
+          for (int k = 0; k < bpad && cand < 0; k += 32) {
+            int bb = (start & ~31) + k + lane;
+            if (bb >= bpad) bb -= bpad;
+            const int st = bb < B ? *reinterpret_cast<volatile int32_t*>(a.sh_ready + bb) : 0;
+            const unsigned open = __ballot_sync(kFull, st == 1);
+            if (open) cand = __shfl_sync(kFull, bb, __ffs(open) - 1);
+          }
+          if (cand < 0) break;
+        }
+        ShareDesc* dsc = a.sh_desc + cand;
+        const int words = *reinterpret_cast<volatile int*>(&dsc->nw);
+        int at = *reinterpret_cast<volatile int*>(&dsc->next);
+        if (at < words) {
+          if (lane == 0) at = atomicAdd(&dsc->next, NW);
+          at = __shfl_sync(kFull, at, 0);
+        }
+        if (at < words) { found = cand; base = at; }
+        else if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + cand) = 2;     // every word is claimed
+      }
+      __threadfence();
+      if (lane == 0) { s.help_b = found; s.help_base = base; }
+    }
+    __syncthreads();
+    const int found = s.help_b, base = s.help_base;
+    __syncthreads();
+    finished = 0;
+    if (found < 0) break;
+    if (found != cur) {
+      const ShareDesc* dsc = a.sh_desc + found;
+      lo = __ldcg(&dsc->lo); cnt = __ldcg(&dsc->cnt);
+      Kp = __ldcg(&dsc->Kp); n_win = __ldcg(&dsc->n_win); nw = __ldcg(&dsc->nw);
+      cur = found;
+    }
+    // a descriptor that makes no sense is left to its owner (the words claimed from it stay
+    // uncounted: its owner reports the context as failed)
+    const bool sane = Kp > 0 && Kp <= a.kcap && cnt >= (int64_t)Kp && lo >= 0 && lo + cnt <= a.n_sa &&
+                      n_win >= 1 && nw == ((Kp + 31) >> 5) && base >= 0 && base < nw;
+    if (!sane) {
+      if (tid == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + found) = 2;
+      cur = -1;
+      continue;
+    }
+    const int end = min(nw, base + NW);
+    ShareDesc* dsc = a.sh_desc + found;
+    gather_words<SaT, kWholeShare>(a, found, sb, sl, lane, lo, cnt, Kp, n_win, base + warp, NW, end,
+                                   a.sh_bm + (int64_t)found * a.m * a.nwords, &dsc->ntrunc,
+                                   a.sh_trunc + (int64_t)found * kMaxTrunc, &dsc->err, nullptr, 0);
+    __threadfence();                   // the words before the count
+    __syncthreads();
+    finished = end - base;
+  }
+}
+
+// The work of one block on its context (blockIdx.x, or the blockIdx.x-th of a list).
 template <typename SaT, bool TP, int NT, int PART>
-__global__ void __launch_bounds__(NT, 1024 / NT)
-rest_draft_kernel(DraftArgs a) {
+__device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* smem_raw) {
   constexpr int NW = NT / 32;
   static_assert(NT % 32 == 0 && NT >= 128, "whole warps; enough threads for the set-up loops");
-  extern __shared__ __align__(16) unsigned char smem_raw[];
   Smem& s = *reinterpret_cast<Smem*>(smem_raw);
   // per warp: token address and length of its 33 slots (the row before the
   // warp's first one, then its 32 rows); the suffix positions of the first rows (phase 4 reads
@@ -380,9 +689,9 @@ rest_draft_kernel(DraftArgs a) {
     if (a.match_n) a.match_n[b] = 0;
     if (a.match_range) { a.match_range[2 * b] = 0; a.match_range[2 * b + 1] = 0; }
   };
-  if constexpr (PART == kWhole || PART == kSearch || PART == kFromRuns) write_defaults();
+  if constexpr (PART == kWhole || PART == kWholeShare || PART == kSearch || PART == kFromRuns) write_defaults();
   const int nq = min(a.n_max, max(clen, 0));   // context tokens that can take part
-  if (tid == 0) { s.err = 0; s.big_total = 0; s.nsel = 0; s.ntrunc = 0; }
+  if (tid == 0) { s.err = 0; s.big_total = 0; s.nsel = 0; s.ntrunc = 0; s.counted = 0; }
   if (tid < 17) { s.lb[tid] = 0; s.ub[tid] = 0; s.ub_from[tid] = -1; }
   if (tid < 5 * (kMaxM + 1)) (&s.small[0][0])[tid] = 0;
   if constexpr (PART != kSearch && PART != kRetrieve) {
@@ -574,148 +883,56 @@ rest_draft_kernel(DraftArgs a) {
   // where the rows' tokens live: the token stream, or the caller's rows of this context
   const int32_t* __restrict__ Trow = PART == kFromRuns ? T + (int64_t)b * a.R * a.Kr * m : T;
   const int nwords = a.nwords;
-  const int niter = (Kp + NT - 1) / NT;
   const int nw = (Kp + 31) >> 5;            // bitmap words that hold rows
 
   // ---- phase 2: gather rows, common-prefix lengths, node-start bitmaps --------------------
-  // Slot 0 of a warp is the row before its first row, slot l + 1 the row of lane l.  A load
-  // instruction fetches two slots, 16 columns each (lane = 16 * slot parity + column): the
-  // lanes of a row read consecutive tokens, so an instruction touches two rows (a few cache
-  // lines) instead of 32.  A token is compared with the token above it (the same column of the
-  // slot before: the other half-warp of the same load, or of the load before) right where it
-  // sits; a ballot turns the "equal" and "smaller" outcomes of each load into bit strings, and
-  // lane l cuts the 16 bits of its row out of them: the number of leading equal columns is the
-  // common prefix.  The suffix-array entries of the next iteration are fetched one iteration
-  // ahead.
-  {
-    // per slot: address of the row's first token, and the row's length
-    const int32_t** sb = reinterpret_cast<const int32_t**>(slot_base + warp * 34);
-    int* sl = slot_len + warp * 34;
-    // where row j comes from: the suffix-array entry of its sampled slot, or (rows handed in
-    // as runs) its place in the caller's row array, through the merged order.  The sampled
-    // slot lo + floor(j cnt / K) advances by a fixed quotient and remainder from one iteration
-    // to the next (j grows by NT), which saves a 64-bit division per row.
-    const uint32_t* ord = PART == kFromRuns ? a.order + (int64_t)b * a.kcap : nullptr;
-    const bool strided = PART != kFromRuns && cnt > (int64_t)a.K && a.sample_mode == REST_SAMPLE_STRIDED;
-    const unsigned long long uK = (unsigned long long)a.K;
-    const unsigned long long step_q = strided ? ((unsigned long long)NT * (unsigned long long)cnt) / uK : (unsigned long long)NT;
-    const unsigned long long step_r = strided ? ((unsigned long long)NT * (unsigned long long)cnt) % uK : 0ull;
-    // this thread's rows j = tid, tid + NT, ...: slot offset and remainder of j cnt / K
-    unsigned long long off = strided ? ((unsigned long long)tid * (unsigned long long)cnt) / uK : (unsigned long long)tid;
-    unsigned long long rem = strided ? ((unsigned long long)tid * (unsigned long long)cnt) % uK : 0ull;
-    // the same for the row before the warp's rows of the NEXT iteration, j + NT - 1 (lane 0
-    // fetches it one iteration ahead)
-    unsigned long long poff = 0, prem = 0;
-    if (lane == 0) {
-      const unsigned long long jn = (unsigned long long)(tid + NT - 1);
-      poff = strided ? (jn * (unsigned long long)cnt) / uK : jn;
-      prem = strided ? (jn * (unsigned long long)cnt) % uK : 0ull;
+  const int32_t** my_sb = reinterpret_cast<const int32_t**>(slot_base + warp * 34);
+  int* my_sl = slot_len + warp * 34;
+  bool shared_gather = false;
+  if constexpr (PART == kWholeShare) shared_gather = Kp > max(a.share_rows, NT);     // more words than warps
+  if (!shared_gather) {
+    // warp w takes words w, w + NW, ...
+    gather_words<SaT, PART>(a, b, my_sb, my_sl, lane, lo, cnt, Kp, n_win, warp, NW, nw, bm, &s.ntrunc,
+                            s.trunc, &s.err, pcache, a.pcache_rows);
+    if constexpr (PART == kWholeShare) {
+      if (tid == 0) { atomicAdd(a.sh_hdr + 1, 1); s.counted = 1; }     // this context offers nothing
+      // its own rows read, the block works on the rows that other contexts offer right now (the
+      // contexts that hold the call up) before it goes on with its own, smaller tree
+      share_help_pass<SaT, NT>(a, s, my_sb, my_sl, b, true);
     }
-    auto advance = [&](unsigned long long& o, unsigned long long& r) {
-      o += step_q; r += step_r;
-      if (r >= uK) { r -= uK; ++o; }
-    };
-    auto entry_at = [&](int j, unsigned long long o) -> int64_t {
-      if constexpr (PART == kFromRuns) return (int64_t)ord[j];
-      else return (int64_t)__ldg(sa + lo + (int64_t)o);
-    };
-    // start of the row's tokens (relative to Trow) and its length; `bad` when the entry is out of range
-    auto row_place = [&](int64_t& p, int64_t& base, int& len, bool& bad) {
-      if constexpr (PART == kFromRuns) {
-        if (p < 0 || p >= (int64_t)a.R * a.Kr) { bad = true; p = 0; }
-        len = bad ? 0 : min(max(a.row_len[(int64_t)b * a.R * a.Kr + p], 0), m);
-        p *= m;
-        base = p;
-      } else {
-        if (p < 0 || p >= n_tokens) { bad = true; p = 0; }
-        base = p + n_win;
-        const int64_t rem_t = n_tokens - base;
-        len = bad ? 0 : (int)(rem_t < 0 ? 0 : (rem_t > m ? m : rem_t));
-      }
-    };
-    int64_t p_next = 0, pp_next = 0;
-    if (tid < Kp) p_next = entry_at(tid, off);
-    if (lane == 0 && tid > 0 && tid <= Kp) {
-      const unsigned long long jp = (unsigned long long)(tid - 1);
-      pp_next = entry_at(tid - 1, strided ? (jp * (unsigned long long)cnt) / uK : jp);
+  } else {
+    // offer the rows to every idle warp of the launch, and take words like any of them
+    ShareDesc* dsc = a.sh_desc + b;
+    if (tid == 0) {
+      dsc->lo = lo; dsc->cnt = cnt; dsc->Kp = Kp; dsc->n_win = n_win; dsc->nw = nw;
+      __threadfence();
+      *reinterpret_cast<volatile int32_t*>(a.sh_ready + b) = 1;
     }
-    const int half = lane >> 4, col = lane & 15;
-    if (lane == 0) { sl[33] = 0; sb[33] = Trow; }     // slot 33 does not exist
-    // columns past a row's end read as a value no token has (tokens are below 2^31), different
-    // for neighbouring slots: they never compare equal to anything above or below them
-    const uint32_t pad = 0x80000000u | (uint32_t)half;
-    for (int it = 0; it < niter; ++it) {
-      const int jbase = it * NT + warp * 32;
-      const int j = jbase + lane;
-      int64_t p = p_next;
-      int64_t pp = pp_next;
-      advance(off, rem);
-      if (j + NT < Kp) p_next = entry_at(j + NT, off);
-      if (lane == 0 && j + NT <= Kp) pp_next = entry_at(j + NT - 1, poff);
-      advance(poff, prem);
-      if (jbase >= Kp) continue;   // warp-uniform
-      const bool valid = j < Kp;
-      bool bad = false;
-      int len = 0;
-      int64_t base = 0;
-      if (valid) {
-        row_place(p, base, len, bad);
-        if (j < a.pcache_rows) pcache[j] = p;
+    __syncthreads();
+    share_work_on<SaT, NT>(a, s, b, my_sb, my_sl, lo, cnt, Kp, n_win);
+    if (tid == 0) {
+      atomicAdd(a.sh_hdr + 1, 1); s.counted = 1;
+      // words still out are in the hands of running warps
+      int polls = 0;
+      while (*reinterpret_cast<volatile int*>(&dsc->done) < nw && polls < kOwnerPolls) { __nanosleep(100); ++polls; }
+      __threadfence();
+      int e = *reinterpret_cast<volatile int*>(&dsc->err);
+      if (*reinterpret_cast<volatile int*>(&dsc->done) < nw) e |= REST_CTX_INTERNAL;
+      if (e) atomicOr(&s.err, e);
+      s.ntrunc = *reinterpret_cast<volatile int*>(&dsc->ntrunc);
+    }
+    __syncthreads();
+    if (s.err == 0) {
+      const uint32_t* gbm = a.sh_bm + (int64_t)b * m * nwords;
+#pragma unroll 4
+      for (int i = tid; i < m * nw; i += NT) {
+        const int d = i / nw, w = i - d * nw;
+        bm[d * nwords + w] = __ldcg(gbm + d * nwords + w);
       }
-      int plen = __shfl_up_sync(kFull, len, 1);
-      if (lane == 0) {
-        plen = 0;
-        int64_t pbase = 0;
-        if (j > 0) row_place(pp, pbase, plen, bad);   // the row before belongs to another warp
-        sb[0] = Trow + pbase; sl[0] = plen;
-      }
-      const int lim = min(len, plen);
-      sb[lane + 1] = Trow + base; sl[lane + 1] = len;
-      __syncwarp();
-      uint32_t vals[kRowLoads];
-#pragma unroll
-      for (int i = 0; i < kRowLoads; ++i) {
-        const int r = 2 * i + half;
-        vals[i] = col < sl[r] ? (uint32_t)__ldg(sb[r] + col) : pad;
-      }
-      uint32_t my_eq = 0, my_lt = 0, other_prev = 0;     // lane i keeps the bit strings of load i
-#pragma unroll
-      for (int i = 0; i < kRowLoads; ++i) {
-        const uint32_t other = __shfl_xor_sync(kFull, vals[i], 16);   // same column, other slot of this load
-        const uint32_t above = half ? other : other_prev;             // the slot before this one
-        const uint32_t eq = __ballot_sync(kFull, vals[i] == above);
-        const uint32_t lt = __ballot_sync(kFull, above < vals[i]);
-        if (lane == i) { my_eq = eq; my_lt = lt; }
-        other_prev = other;
-      }
-      // this lane's row is slot lane + 1: load (lane + 1) / 2, upper half of the word when odd
-      const int slot = lane + 1, sh = (slot & 1) << 4;
-      const uint32_t eqf = (__shfl_sync(kFull, my_eq, slot >> 1) >> sh) & 0xFFFFu;
-      const uint32_t ltf = (__shfl_sync(kFull, my_lt, slot >> 1) >> sh) & 0xFFFFu;
-      int lcp = __ffs((int)(~eqf | 0x10000u)) - 1;       // leading equal columns (padding never matches: at most lim)
-      if (!valid || j == 0) lcp = 0;
-      if (valid && j > 0) {
-        // the first differing column decides the order; when one row is a prefix of the
-        // other the shorter one must come first
-        const bool ordered = lcp < lim ? ((ltf >> lcp) & 1u) != 0u : plen <= len;
-        if (!ordered) bad = true;
-      }
-      if (valid && len < m) {        // cut short by the end of the stream: at most m such rows exist
-        const int at = atomicAdd(&s.ntrunc, 1);
-        if (at < kMaxTrunc) s.trunc[at] = ((uint32_t)len << 16) | (uint32_t)j;
-        else atomicOr(&s.err, REST_CTX_INTERNAL);
-      }
-      uint32_t myword = 0;
-#pragma unroll
-      for (int d = 1; d <= kMaxM; ++d) {
-        const uint32_t w = __ballot_sync(kFull, !valid || lcp < d);
-        if (lane == d - 1) myword = w;
-      }
-      if (lane < m) bm[lane * nwords + (jbase >> 5)] = myword;
-      if (__any_sync(kFull, bad) && lane == 0) atomicOr(&s.err, REST_CTX_BAD_DATASTORE);
-      __syncwarp();                  // the slot tables are rewritten by the next iteration
+      if (tid < min(s.ntrunc, kMaxTrunc)) s.trunc[tid] = __ldcg(a.sh_trunc + (int64_t)b * kMaxTrunc + tid);
     }
   }
+  const int pcache_rows = shared_gather ? 0 : a.pcache_rows;   // rows whose position phase 4 finds in shared memory
   if (tid < m) bm[tid * nwords + ((Kp + 31) >> 5)] = kFull;   // sentinel past the last row
   __syncthreads();
   if (s.err != 0) {
@@ -975,7 +1192,7 @@ rest_draft_kernel(DraftArgs a) {
     }
     s.par[i] = par;
     int64_t p;
-    if (j < a.pcache_rows) p = (int64_t)pcache[j];
+    if (j < pcache_rows) p = (int64_t)pcache[j];
     else if constexpr (PART == kFromRuns) p = (int64_t)a.order[(int64_t)b * a.kcap + j] * m;
     else p = (int64_t)__ldg(sa + sample_slot(lo, cnt, a.K, a.sample_mode, j));
     int64_t o = (int64_t)b * N + i;
@@ -1015,6 +1232,62 @@ rest_draft_kernel(DraftArgs a) {
     a.n_nodes[b] = nn;
     if (a.match_n) a.match_n[b] = n_win;
     if (a.match_range) { a.match_range[2 * b] = lo; a.match_range[2 * b + 1] = hi; }
+  }
+}
+
+template <typename SaT, bool TP, int NT, int PART>
+__global__ void __launch_bounds__(NT, 1024 / NT)
+rest_draft_kernel(DraftArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  if constexpr (PART != kWholeShare) {
+    draft_block<SaT, TP, NT, PART>(a, smem_raw);
+  } else {
+    // blocks beyond the contexts only help
+    constexpr int NW = NT / 32;
+    Smem& s = *reinterpret_cast<Smem*>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool has_context = (int)blockIdx.x < a.B;
+    if (has_context) {
+      if (tid == 0) atomicAdd(a.sh_hdr, 1);
+      draft_block<SaT, TP, NT, PART>(a, smem_raw);
+    } else if (tid == 0) {
+      s.counted = 1;
+    }
+    __syncthreads();
+    if (tid == 0 && !s.counted) atomicAdd(a.sh_hdr + 1, 1);     // left before its gather: nothing to offer
+    // ---- help: while contexts may still offer rows, work on what is offered ---------------------
+    long long* slot_base = reinterpret_cast<long long*>(smem_raw + sizeof(Smem));
+    int* slot_len = reinterpret_cast<int*>(slot_base + NW * 34 + a.pcache_rows);
+    const int32_t** my_sb = reinterpret_cast<const int32_t**>(slot_base + warp * 34);
+    int* my_sl = slot_len + warp * 34;
+    const int B = a.B;
+    int polls = 0;
+    for (;;) {
+      if (warp == 0) {
+        // anything offered?  (all warps then look for themselves)
+        bool open = false;
+        for (int k = 0; k < B; k += 32) {
+          const int bb = k + lane;
+          const int st = bb < B ? *reinterpret_cast<volatile int32_t*>(a.sh_ready + bb) : 0;
+          open = open || __any_sync(kFull, st == 1);
+        }
+        int verdict = open ? 1 : 0;
+        if (!open) {
+          // Leave when nothing can come any more, or when contexts of this launch still wait
+          // for an SM (a block that only helps gives them time to start), or after a while
+          const int started = *reinterpret_cast<volatile int32_t*>(a.sh_hdr);
+          const int past = *reinterpret_cast<volatile int32_t*>(a.sh_hdr + 1);
+          if (past >= B || (started < B && has_context) || ++polls > kHelperPolls) verdict = -1;
+          else __nanosleep(500);
+        }
+        if (lane == 0) s.help_b = verdict;
+      }
+      __syncthreads();
+      const int verdict = s.help_b;
+      __syncthreads();
+      if (verdict < 0) break;
+      if (verdict > 0) share_help_pass<SaT, NT>(a, s, my_sb, my_sl, (int)blockIdx.x % B, false);
+    }
   }
 }
 
@@ -1065,8 +1338,13 @@ static size_t split_workspace_bytes(int B) { return (2 * (size_t)B + 16) * sizeo
 extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params* prm, int32_t B) {
   if (!prm || B <= 0) return 0;
   bool batched = false;
-  if (wants_batched(prm->search_path, B, true, &batched) != REST_OK || !batched) return 0;
-  return split_workspace_bytes(B);
+  if (wants_batched(prm->search_path, B, true, &batched) != REST_OK) return 0;
+  if (batched) return split_workspace_bytes(B);
+  // the one-launch form: scratch for shared gathering, where it can help
+  if (prm->K <= kShareRows || B < kShareMinContexts || B > kShareMaxContexts || prm->m < 1 || prm->m > REST_MAX_M || prm->K > REST_MAX_K) return 0;
+  int nwords = 0;
+  draft_smem_bytes(prm->K, prm->m, kThreads, nullptr, &nwords, nullptr, nullptr);
+  return share_layout(B, prm->m, nwords).bytes;
 }
 
 extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* prm,
@@ -1111,6 +1389,7 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
   const bool narrow = ds->v.sa_bytes == 4;
   a.list = nullptr; a.list_count = nullptr; a.B = B; a.which = 0; a.light_rows = 0;
   a.kcap = 0; a.nwords = 0; a.pcache_rows = 0; a.bigcap = 0;
+  a.sh_hdr = nullptr; a.sh_ready = nullptr; a.sh_desc = nullptr; a.sh_trunc = nullptr; a.sh_bm = nullptr; a.share_rows = 0;
   auto launch = [&](auto kern, int slot, int threads, int blocks, size_t bytes) -> rest_status {
     REST_CUDA_TRY(rest::ensure_dynamic_smem(reinterpret_cast<const void*>(kern),
                                             rest::kSmemSlotDraft + slot + (narrow ? 0 : 1), bytes));
@@ -1126,12 +1405,35 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     // context the whole SM (not the single context: its typical candidate list is short and
     // the larger block only adds barrier time)
     const int sms = rest::sm_count();
-    if (big || (B > 1 && B <= sms)) {
-      const size_t smem = smem_for(prm->K, kBigThreads);
+    const bool wide_block = big || (B > 1 && B <= sms);
+    const int threads = wide_block ? kBigThreads : kThreads;
+    const size_t smem = smem_for(prm->K, threads);
+    // With the caller's scratch, contexts with long candidate lists share their gather with
+    // the blocks that are idle: those of finished contexts and, when the call has fewer contexts
+    // than the GPU has SMs, blocks launched for nothing else (one per SM left over, so that
+    // every block of the launch is resident at once).
+    const ShareLayout lay = share_layout(B, prm->m, a.nwords);
+    const bool share = d_ws && ws_bytes >= lay.bytes && reinterpret_cast<uintptr_t>(d_ws) % 16 == 0 &&
+                       prm->K > kShareRows && B >= kShareMinContexts && B <= kShareMaxContexts;
+    if (share) {
+      unsigned char* ws = static_cast<unsigned char*>(d_ws);
+      a.sh_hdr = reinterpret_cast<int32_t*>(ws);
+      a.sh_ready = reinterpret_cast<int32_t*>(ws + lay.ready);
+      a.sh_desc = reinterpret_cast<ShareDesc*>(ws + lay.desc);
+      a.sh_trunc = reinterpret_cast<uint32_t*>(ws + lay.trunc);
+      a.sh_bm = reinterpret_cast<uint32_t*>(ws + lay.bm);
+      a.share_rows = kShareRows;
+      REST_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.zeroed_bytes, st));
+      const int blocks = B < sms ? sms : B;
+      if (wide_block)
+        return narrow ? launch(rest_draft_kernel<int32_t, false, kBigThreads, kWholeShare>, 18, kBigThreads, blocks, smem)
+                      : launch(rest_draft_kernel<int64_t, false, kBigThreads, kWholeShare>, 18, kBigThreads, blocks, smem);
+      return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWholeShare>, 16, kThreads, blocks, smem)
+                    : launch(rest_draft_kernel<int64_t, false, kThreads, kWholeShare>, 16, kThreads, blocks, smem);
+    }
+    if (wide_block)
       return narrow ? launch(rest_draft_kernel<int32_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem)
                     : launch(rest_draft_kernel<int64_t, false, kBigThreads, kWhole>, 10, kBigThreads, B, smem);
-    }
-    const size_t smem = smem_for(prm->K, kThreads);
     return narrow ? launch(rest_draft_kernel<int32_t, false, kThreads, kWhole>, 0, kThreads, B, smem)
                   : launch(rest_draft_kernel<int64_t, false, kThreads, kWhole>, 0, kThreads, B, smem);
   }

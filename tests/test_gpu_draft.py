@@ -99,7 +99,9 @@ def test_more_contexts_than_the_gpu_holds_at_once():
     for search in (rest.REST_SEARCH_AUTO, rest.REST_SEARCH_BATCHED):
         got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, workspace=False, **kw)
         assert_draft_equal(got, ref, f"one launch, search {search:#x}")
-    assert rest.draft_workspace_bytes(B, **kw) >= 8 * B and rest.draft_workspace_bytes(8, **kw) == 0
+    assert rest.draft_workspace_bytes(B, **kw) >= 8 * B
+    # few contexts: scratch only for sharing the gather of long candidate lists
+    assert rest.draft_workspace_bytes(8, **kw) > 0 and rest.draft_workspace_bytes(8, K=512, m=w.m, N=w.N) == 0
     assert len(set(ref["match_n"].tolist())) > 8          # matched lengths all over 2 ... 16
     with pytest.raises(rest.RestError):
         gpu_draft(T, sa, w.vocab, ctx[:2], ctx_len[:2], search=0x400, **kw)
