@@ -56,13 +56,14 @@ enum {
 
 enum { REST_SAMPLE_STRIDED = 0, REST_SAMPLE_FIRST_K = 1 };
 /* How rest_draft searches the suffix array (rest_draft_params.search_path); the results are the
- * same either way.  SINGLE: all suffix lengths at once, 32 probes per round, 512 threads per
- * context (fewest dependent reads, the fastest single context).  BATCHED: 256 threads per
- * context, six or seven searches instead of fifteen (the lengths that match are n_min ... n*
- * without a gap) and eight probes per round once the probes leave L2: more dependent rounds,
- * fewer random DRAM reads, more contexts in flight (most of all with the scratch that
- * rest_draft_workspace_bytes asks for, see d_ws).  AUTO picks BATCHED when the call has at
- * least 5 contexts per SM and that scratch, or at least 16 contexts per SM without it. */
+ * same either way.  SINGLE: every suffix length at once, a warp per length, 32 probes per round
+ * inside the range that the datastore's n-gram index gives for the query's first tokens (fewest
+ * dependent reads, the fastest single context); 512 or 1024 threads per context.  BATCHED: 256
+ * threads per context, six or seven searches instead of fifteen (the lengths that match are
+ * n_min ... n* without a gap) and eight probes per round once the probes leave L2: more
+ * dependent rounds, fewer random DRAM reads, more contexts in flight (most of all with the
+ * scratch that rest_draft_workspace_bytes asks for, see d_ws).  AUTO picks BATCHED when the call
+ * has at least 5 contexts per SM and that scratch, or at least 16 contexts per SM without it. */
 enum { REST_SEARCH_AUTO = 0, REST_SEARCH_SINGLE = 1, REST_SEARCH_BATCHED = 2 };
 enum { REST_DS_VALIDATE = 1u, REST_DS_INDEX = 2u };
 
@@ -161,12 +162,19 @@ rest_status rest_datastore_create_shard(const int32_t* d_tokens, uint64_t n_toke
  *   d_match_range int64[B,2] lo, hi of the matched suffix-array range
  *   d_node_count int32[B,N]  weight of each kept node (may be NULL)
  *   d_status     int32[B]    REST_CTX_* code
- *   d_ws         optional scratch of rest_draft_workspace_bytes() bytes (the query answers for
- *                the current device; 0 when the call takes the single-context path).  With it
- *                the batched path runs as three launches (search; build of the contexts with
- *                few candidates on small blocks; build of the others on large blocks) and the
- *                scratch holds the two context lists; with NULL or fewer bytes it runs as one
- *                launch.  The outputs are the same.
+ *   d_ws         optional scratch of rest_draft_workspace_bytes() bytes, 16-byte aligned (the
+ *                query answers for the current device and may be 0).  Never needed for the
+ *                results, only for speed; with NULL or fewer bytes every path runs as one launch
+ *                of one block per context.  What it buys:
+ *                - single-context path, 2 to 1024 contexts, K > 512: a context with a long
+ *                  candidate list lets idle blocks (those of finished or lighter contexts, and
+ *                  blocks started on SMs that have no context) read part of its rows; the scratch
+ *                  holds the contexts' counters and node-start bitmaps (about 6 m K / 32 bytes
+ *                  per context).  The call zeroes the counters itself.
+ *                - batched path: three launches (search; build of the contexts with few
+ *                  candidates on small blocks; build of the others on large blocks); the scratch
+ *                  holds the two context lists (8 bytes per context).
+ *                The scratch must not be shared by calls that may run at the same time.
  */
 size_t rest_draft_workspace_bytes(const rest_draft_params* params, int32_t B);
 rest_status rest_draft(const rest_datastore* ds, const rest_draft_params* params,

@@ -267,26 +267,43 @@ __device__ __forceinline__ int next_set(const uint32_t* __restrict__ row,
   return bits ? (w << 5) + __ffs(bits) - 1 : (int)jump[w];
 }
 
-// Executed by one warp.  hist[0..nbins) holds counts; total >= need >= 1.  Finds the largest
-// bin b with sum(hist[k], k > b) < need; returns b and that sum.
-__device__ void warp_threshold_desc(const uint32_t* hist, int nbins, uint32_t need, int lane,
-                                    int* out_bin, uint32_t* out_above) {
-  int per = (nbins + 31) / 32;
-  int top = nbins - 1 - lane * per;
-  int bot = max(0, top - per + 1);
-  uint32_t s = 0;
-  for (int b = top; b >= bot && b >= 0; --b) s += hist[b];
-  uint32_t incl = s;
+// Executed by a whole block of NT threads.  hist[0..nbins) holds counts; total >= need >= 1.
+// Finds the largest bin b with sum(hist[k], k > b) < need; writes b and that sum (visible after
+// the caller's next barrier).  scan: NT / 32 words of shared memory.
+template <int NT>
+__device__ __forceinline__ void block_threshold_desc(const uint32_t* hist, int nbins, uint32_t need, uint32_t* scan,
+                                                     int* out_bin, uint32_t* out_above) {
+  constexpr int NW = NT / 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = (nbins + NT - 1) / NT;        // bins per thread, from the top down
+  const int top = nbins - 1 - tid * per;
+  const int bot = max(0, top - per + 1);
+  uint32_t sum = 0;
+  for (int b = top; b >= bot; --b) sum += hist[b];
+  uint32_t incl = sum;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    uint32_t v = __shfl_up_sync(kFull, incl, o);
+    const uint32_t v = __shfl_up_sync(kFull, incl, o);
     if (lane >= o) incl += v;
   }
-  uint32_t excl = incl - s;
-  if (excl < need && need <= incl) {
+  if (lane == 31) scan[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {                              // exclusive prefix over the warps' totals
+    const uint32_t mine = lane < NW ? scan[lane] : 0u;
+    uint32_t t = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t v = __shfl_up_sync(kFull, t, o);
+      if (lane >= o) t += v;
+    }
+    if (lane < NW) scan[lane] = t - mine;
+  }
+  __syncthreads();
+  const uint32_t excl = scan[warp] + incl - sum;
+  if (excl < need && need <= excl + sum) {
     uint32_t acc = excl;
     for (int b = top; b >= bot; --b) {
-      uint32_t h = hist[b];
+      const uint32_t h = hist[b];
       if (acc + h >= need) { *out_bin = b; *out_above = acc; break; }
       acc += h;
     }
@@ -305,6 +322,7 @@ struct Smem {
   int bin_lo;
   uint32_t above_lo;
   uint32_t nsel;
+  uint32_t scan[32];           // warp totals of a block-wide prefix sum
   int ntrunc;
   int counted;                 // shared gathering: this context is counted as past its gather
   int help_b;                  // shared gathering: the context this block helps next
@@ -941,26 +959,61 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   }
   const int ntrunc = min(s.ntrunc, kMaxTrunc);
 
-  // jump table: for every depth (a warp each) a suffix scan over the bitmap words, last chunk
-  // of 32 words first: jump[w] = position of the first set bit in any word after w
-  for (int dd = warp; dd < m; dd += NW) {
-    const uint32_t* row = bm + dd * nwords;
-    uint16_t* jrow = jump + dd * nwords;
+  // jump table: jump[w] = position of the first set bit in any word after w (0xFFFF: none).  A
+  // warp takes a chunk of 32 words of a depth: a ballot of the non-empty words tells every lane
+  // which lane behind it holds the next set bit.  With several chunks per depth, the first set
+  // bit of every chunk is found first and, per depth, what the chunks behind a chunk hold.
+  {
     const int last = (Kp + 31) >> 5;              // the sentinel word
-    int carry = 0x7FFFFFFF;
-    for (int c = last >> 5; c >= 0; --c) {
-      const int wi = c * 32 + lane;
-      const uint32_t bits = wi <= last ? row[wi] : 0u;
-      int v = bits ? (wi << 5) + __ffs(bits) - 1 : 0x7FFFFFFF;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {          // inclusive suffix minimum over the lanes
-        const int u = __shfl_down_sync(kFull, v, o);
-        if (lane + o < 32) v = min(v, u);
+    const int nchunk = (last >> 5) + 1;
+    uint16_t* cmin = tiecnt;                      // [m][nchunk], free until phase 3c (16 nchunk <= nwords when nchunk > 1)
+    const int step_d = NW / nchunk, step_c = NW - step_d * nchunk;     // a warp's next pair: NW further
+    if (nchunk > 1) {                             // block-uniform
+      int dd = warp / nchunk, c = warp - dd * nchunk;
+#pragma unroll 2
+      for (int pair = warp; pair < m * nchunk; pair += NW) {
+        const int wi = c * 32 + lane;
+        const uint32_t bits = wi <= last ? bm[dd * nwords + wi] : 0u;
+        const unsigned nz = __ballot_sync(kFull, bits != 0u);
+        const int v = (wi << 5) + __ffs(bits) - 1;
+        const int first = __shfl_sync(kFull, v, nz ? __ffs(nz) - 1 : 0);
+        if (lane == 0) cmin[pair] = (uint16_t)(nz ? first : 0xFFFF);
+        dd += step_d; c += step_c;
+        if (c >= nchunk) { c -= nchunk; ++dd; }
       }
-      v = min(v, carry);
-      const int after = __shfl_down_sync(kFull, v, 1);
-      if (wi <= last) jrow[wi] = (uint16_t)min(lane < 31 ? after : carry, 0xFFFF);
-      carry = __shfl_sync(kFull, v, 0);
+      __syncthreads();
+      // per depth: exclusive suffix minimum over the (at most 33) chunks
+      for (int dd = warp; dd < m; dd += NW) {
+        uint16_t* cm = cmin + dd * nchunk;
+        int carry = 0xFFFF;
+        for (int g0 = ((nchunk - 1) >> 5) << 5; g0 >= 0; g0 -= 32) {
+          const int c = g0 + lane;
+          int v = c < nchunk ? (int)cm[c] : 0xFFFF;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_down_sync(kFull, v, o);
+            if (lane + o < 32) v = min(v, u);
+          }
+          v = min(v, carry);
+          const int after = __shfl_down_sync(kFull, v, 1);
+          if (c < nchunk) cm[c] = (uint16_t)(lane < 31 ? after : carry);
+          carry = __shfl_sync(kFull, v, 0);
+        }
+      }
+      __syncthreads();
+    }
+    int dd = warp / nchunk, c = warp - dd * nchunk;
+#pragma unroll 2
+    for (int pair = warp; pair < m * nchunk; pair += NW, dd += step_d, c += step_c) {
+      if (c >= nchunk) { c -= nchunk; ++dd; }
+      const int wi = c * 32 + lane;
+      const uint32_t bits = wi <= last ? bm[dd * nwords + wi] : 0u;
+      const unsigned nz = __ballot_sync(kFull, bits != 0u);
+      const int v = (wi << 5) + __ffs(bits) - 1;
+      const unsigned higher = nz & ~((2u << lane) - 1u);          // non-empty words behind this one in the chunk
+      const int nextv = __shfl_sync(kFull, v, higher ? __ffs(higher) - 1 : lane);
+      const int behind = nchunk > 1 ? (int)cmin[pair] : 0xFFFF;
+      if (wi <= last) jump[dd * nwords + wi] = (uint16_t)(higher ? nextv : behind);
     }
   }
   __syncthreads();
@@ -997,28 +1050,53 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   auto sub_of = [](int c, int d) -> int { return c < 1024 ? 16 - d : ((c & 31) << 5) | (16 - d); };
 
   // ---- phase 3a: counts of the light nodes, histogram of the others ------------------------
+  // First the words: light nodes are counted, heavy nodes only listed (depth, row).  Then the
+  // list, a thread per heavy node: its weight (distance to the next set bit) and its bin.  Short
+  // dependent chains in both passes; a thread that walked its words' heavy nodes one by one,
+  // weights included, held its warp up for a thousand cycles per word.
   {
+    int d = tid / nw + 1, w = tid - (d - 1) * nw;
+    const int step_d = NT / nw, step_w = NT - step_d * nw;          // a thread's next item: NT further
+#pragma unroll 2
     for (int item = tid; item < items; item += NT) {
-      const int d = item / nw + 1, w = item - (d - 1) * nw;
       const WordNodes wn = word_nodes(d, w);
 #pragma unroll
       for (int c = 1; c <= 4; ++c)
         if (wn.c[c]) atomicAdd(&s.small[c][d], (uint32_t)__popc(wn.c[c]));
-      const uint32_t* row = bm + (d - 1) * nwords;
-      const uint16_t* jrow = jump + (d - 1) * nwords;
       uint32_t big = wn.big;
       if (big) {
-        // the word's heavy nodes also go into a list, which the later passes read instead of
-        // walking the bitmaps again (when it overflows they walk)
         uint32_t at = atomicAdd(&s.big_total, (uint32_t)__popc(big));
         while (big) {
-          const int j = (w << 5) + __ffs(big) - 1;
+          if (at < (uint32_t)a.bigcap) big_dj[at] = ((uint32_t)d << 16) | (uint32_t)((w << 5) + __ffs(big) - 1);
           big &= big - 1;
-          const int c = next_set(row, jrow, j) - j;
-          atomicAdd(&s.hist_hi[bin_of(c)], 1u);
-          if (at < (uint32_t)a.bigcap) { big_dj[at] = ((uint32_t)d << 16) | (uint32_t)j; big_c[at] = (uint16_t)c; }
           ++at;
         }
+      }
+      d += step_d; w += step_w;
+      if (w >= nw) { w -= nw; ++d; }
+    }
+  }
+  __syncthreads();
+  const uint32_t big_total = s.big_total;
+  const bool listed = big_total <= (uint32_t)a.bigcap;     // the list holds every heavy node
+  if (listed) {
+    for (uint32_t e = tid; e < big_total; e += NT) {
+      const int d = (int)(big_dj[e] >> 16), j = (int)(big_dj[e] & 0xFFFFu);
+      const int c = next_set(bm + (d - 1) * nwords, jump + (d - 1) * nwords, j) - j;
+      big_c[e] = (uint16_t)c;
+      atomicAdd(&s.hist_hi[bin_of(c)], 1u);
+    }
+  } else {
+    // more heavy nodes than the list holds: this pass and the later ones walk the words again
+    for (int item = tid; item < items; item += NT) {
+      const int d = item / nw + 1, w = item - (d - 1) * nw;
+      uint32_t big = word_nodes(d, w).big;
+      const uint32_t* row = bm + (d - 1) * nwords;
+      const uint16_t* jrow = jump + (d - 1) * nwords;
+      while (big) {
+        const int j = (w << 5) + __ffs(big) - 1;
+        big &= big - 1;
+        atomicAdd(&s.hist_hi[bin_of(next_set(row, jrow, j) - j)], 1u);
       }
     }
   }
@@ -1028,10 +1106,8 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   uint32_t tstar = 0;  // nodes with key > tstar are kept
   uint32_t r_tie = 0;  // plus the first r_tie nodes (by row) with key == tstar
   int c_tie = 0, d_tie = 0;
-  const uint32_t big_total = s.big_total;
-  const bool listed = big_total <= (uint32_t)a.bigcap;     // the list holds every heavy node
   if (big_total >= (uint32_t)N) {
-    if (warp == 0) warp_threshold_desc(s.hist_hi, kHistHi, (uint32_t)N, lane, &s.bin_hi, &s.above_hi);
+    block_threshold_desc<NT>(s.hist_hi, kHistHi, (uint32_t)N, s.scan, &s.bin_hi, &s.above_hi);
     __syncthreads();
     const int bin_hi = s.bin_hi;
     if (listed) {
@@ -1053,8 +1129,7 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
       }
     }
     __syncthreads();
-    if (warp == 0)
-      warp_threshold_desc(s.hist_lo, kHistLo, (uint32_t)N - s.above_hi, lane, &s.bin_lo, &s.above_lo);
+    block_threshold_desc<NT>(s.hist_lo, kHistLo, (uint32_t)N - s.above_hi, s.scan, &s.bin_lo, &s.above_lo);
     __syncthreads();
     const int sub = s.bin_lo;
     d_tie = 16 - (sub & 31);
@@ -1062,14 +1137,29 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
     tstar = key_of(c_tie, d_tie);
     r_tie = (uint32_t)N - s.above_hi - s.above_lo;
   } else {
-    // every node of weight >= 5 is kept; the lighter ones fill up by weight, then depth, then row
-    uint32_t need = (uint32_t)N - big_total, cum = 0;
-    for (int c = 4; c >= 1 && tstar == 0; --c) {
-      for (int d = 1; d <= m; ++d) {
-        const uint32_t e = s.small[c][d];
-        if (cum + e >= need) { c_tie = c; d_tie = d; tstar = key_of(c, d); r_tie = need - cum; break; }
-        cum += e;
-      }
+    // every node of weight >= 5 is kept; the lighter ones fill up by weight, then depth, then
+    // row.  Every warp scans the 4 x 16 counts in that order for itself: lane l takes the
+    // classes 2 l and 2 l + 1 (class k = weight 4 - k / 16 at depth k % 16 + 1).
+    const uint32_t need = (uint32_t)N - big_total;
+    const int k0 = 2 * lane, k1 = 2 * lane + 1;
+    const int c0 = 4 - (k0 >> 4), d0 = (k0 & 15) + 1, c1 = 4 - (k1 >> 4), d1 = (k1 & 15) + 1;
+    const uint32_t e0 = d0 <= m ? s.small[c0][d0] : 0u, e1 = d1 <= m ? s.small[c1][d1] : 0u;
+    uint32_t incl = e0 + e1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t u = __shfl_up_sync(kFull, incl, o);
+      if (lane >= o) incl += u;
+    }
+    const uint32_t before = incl - e0 - e1;
+    const unsigned hit = __ballot_sync(kFull, incl >= need);      // need >= 1
+    if (hit) {
+      const int src = __ffs(hit) - 1;
+      const uint32_t bsrc = __shfl_sync(kFull, before, src), e0s = __shfl_sync(kFull, e0, src);
+      const bool first = bsrc + e0s >= need;
+      const int k = 2 * src + (first ? 0 : 1);
+      c_tie = 4 - (k >> 4); d_tie = (k & 15) + 1;
+      tstar = key_of(c_tie, d_tie);
+      r_tie = need - bsrc - (first ? 0u : e0s);
     }
   }
 
@@ -1079,6 +1169,14 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   auto keep = [&](int d, int j, int c) {
     const uint32_t slot = atomicAdd(&s.nsel, 1u);
     if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)j; s.selcnt[slot] = (uint32_t)c; }
+  };
+  // the first `take` nodes marked in `bits` (rows 32 w + bit) of depth d, weight c: one claim of slots
+  auto keep_bits = [&](int d, int w, int c, uint32_t bits, uint32_t take) {
+    uint32_t slot = atomicAdd(&s.nsel, take);
+    for (; take > 0; --take, ++slot) {
+      if (slot < (uint32_t)N) { s.sel[slot] = ((uint32_t)d << 16) | (uint32_t)((w << 5) + __ffs(bits) - 1); s.selcnt[slot] = (uint32_t)c; }
+      bits &= bits - 1;
+    }
   };
   auto tie_bits = [&](int w) -> uint32_t {         // tie candidates in word w of the tie depth
     const WordNodes wn = word_nodes(d_tie, w);
@@ -1107,13 +1205,7 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
     const WordNodes wn = word_nodes(d, w);
 #pragma unroll
     for (int c = 1; c <= 4; ++c) {
-      if (key_of(c, d) > tstar) {
-        uint32_t bits = wn.c[c];
-        while (bits) {
-          keep(d, (w << 5) + __ffs(bits) - 1, c);
-          bits &= bits - 1;
-        }
-      }
+      if (key_of(c, d) > tstar && wn.c[c]) keep_bits(d, w, c, wn.c[c], (uint32_t)__popc(wn.c[c]));
     }
     const uint32_t* row = bm + (d - 1) * nwords;
     const uint16_t* jrow = jump + (d - 1) * nwords;
@@ -1147,12 +1239,9 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
     for (int w = tid; w < nw; w += NT) {
       uint32_t rank = tiecnt[w];
       if (rank >= r_tie) continue;
-      uint32_t t = tie_bits(w);
-      while (t && rank < r_tie) {
-        keep(d_tie, (w << 5) + __ffs(t) - 1, c_tie);
-        t &= t - 1;
-        ++rank;
-      }
+      const uint32_t t = tie_bits(w);
+      const uint32_t take = min((uint32_t)__popc(t), r_tie - rank);
+      if (take) keep_bits(d_tie, w, c_tie, t, take);
     }
   }
   __syncthreads();
@@ -1160,12 +1249,21 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   if (s.nsel > (uint32_t)N && tid == 0) atomicOr(&s.err, REST_CTX_INTERNAL);
 
   // ---- phase 4: breadth-first order, parents, masks, tokens ---------------------------------
-  for (int i = tid; i < nn; i += NT) {
-    const uint32_t me = s.sel[i];
+  // rank of a kept node = kept nodes with a smaller (depth, row); four threads share a node
+  for (int idx0 = 0; idx0 < 4 * nn; idx0 += NT) {      // the same trip count for every thread
+    const int idx = idx0 + tid, i = idx >> 2, q = idx & 3;
+    uint32_t me = 0;
     int rank = 0;
-    for (int k = 0; k < nn; ++k) rank += (s.sel[k] < me);
-    s.sorted[rank] = me;
-    s.sortedcnt[rank] = s.selcnt[i];
+    if (i < nn) {
+      me = s.sel[i];
+      for (int k = q; k < nn; k += 4) rank += (s.sel[k] < me);     // the four read neighbouring words
+    }
+    rank += __shfl_xor_sync(kFull, rank, 1);
+    rank += __shfl_xor_sync(kFull, rank, 2);
+    if (i < nn && q == 0) {
+      s.sorted[rank] = me;
+      s.sortedcnt[rank] = s.selcnt[i];
+    }
   }
   __syncthreads();
   for (int i = tid; i < nn; i += NT) {
@@ -1203,21 +1301,16 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
     if (a.node_count) a.node_count[o] = (int32_t)s.sortedcnt[i];
   }
   __syncthreads();
-  for (int i = tid; i < nn; i += NT) {
-    uint32_t bits[(kMaxN + 31) / 32];
-#pragma unroll
-    for (int w = 0; w < (kMaxN + 31) / 32; ++w) bits[w] = 0;
+  // ancestor masks, a thread per (node, mask word): walk up the parents, keep the bits of its word
+  for (int idx = tid; idx < nn * Wm; idx += NT) {
+    const int i = idx / Wm, wq = idx - i * Wm;
+    uint32_t bits = 0;
     int k = i;
     for (int step = 0; step <= kMaxM && k >= 0; ++step) {
-#pragma unroll
-      for (int w = 0; w < (kMaxN + 31) / 32; ++w)
-        if (w == (k >> 5)) bits[w] |= 1u << (k & 31);
+      if ((k >> 5) == wq) bits |= 1u << (k & 31);
       k = s.par[k];
     }
-    int64_t o = ((int64_t)b * N + i) * Wm;
-#pragma unroll
-    for (int w = 0; w < (kMaxN + 31) / 32; ++w)
-      if (w < Wm) a.mask[o + w] = bits[w];
+    a.mask[((int64_t)b * N + i) * Wm + wq] = bits;
   }
   __syncthreads();
   if (s.err != 0) {
