@@ -43,10 +43,16 @@ L2_BYTES = 126e6
 # reads its own K/V once, so traffic grows in proportion).  Shapes without a capture report null.
 NCU_TRAFFIC_PER_UNIT = {
     # (kernel, N, L): bytes per (context, head)
-    ("tree_attention_wide_kernel", 128, 16384): 2448.4e6 / (9 * 32),
-    ("tree_attention_ws_kernel", 64, 4096): 970.3e6 / (14 * 32),
-    ("tree_attention_ws_kernel", 64, 2048): 35_185_920 / 32,
+    ("tree_attention_wide_kernel", 128, 16384): 2449.3e6 / (9 * 32),
+    ("tree_attention_ws_kernel", 64, 4096): 970.1e6 / (14 * 32),
+    ("tree_attention_ws_kernel", 64, 2048): 35_185_408 / 32,
 }
+
+
+# The same for the draft kernel of the single-context path: DRAM bytes of one launch per candidate
+# row gathered (stress recipe, 100 M tokens, B = 128, 2409 rows per context on average; the rows
+# and their suffix-array entries are nearly all of the traffic, so it grows with the rows).
+NCU_DRAFT_TRAFFIC_PER_ROW = {"stress": (73.87e6 + 2.48e6) / (128 * 2408.6)}
 
 
 def parse_args():
@@ -759,7 +765,10 @@ def run_ours(args, rank, world, local_rank):
                            "algorithmic_bytes_per_launch": d_bytes,
                            "sector_granular_bytes_per_launch": draft_sector_bytes(
                                w.n_tokens, w.sa_bytes, w.n_min, w.n_max, kp_mean, w.m, N) * B,
-                           "traffic": None,
+                           "traffic": None if w.name not in NCU_DRAFT_TRAFFIC_PER_ROW or args.n_tokens is not None
+                           else NCU_DRAFT_TRAFFIC_PER_ROW[w.name] * kp_mean * B,
+                           "traffic_source": "ncu capture of the same kernel on the same recipe at 100 M tokens "
+                                             "(profiles/), scaled by the candidate rows of this launch",
                            "dependent_read_ns": read_ns, "dependent_reads_on_critical_path": chain,
                            "latency_floor_us": chain * read_ns / 1e3,
                            "frac_of_latency_floor": chain * read_ns / 1e3 / (t_draft * 1e6)},
