@@ -109,20 +109,24 @@ struct DraftArgs {
 // what makes a context slow is a long candidate list, whose rows one block reads alone while the
 // blocks of the other contexts have finished and other SMs never had a block.  So a context
 // with many candidates publishes its matched range, and every warp that has nothing else to do
-// - the owner's own warps, the warps of blocks whose own rows are read or whose context is
-// finished, the warps of blocks launched as helpers only - claims bitmap words (32 rows each)
-// from the context's counter, computes them into the scratch and counts them done.  The owner
-// waits only for words that some running warp has claimed (unclaimed ones it takes itself),
-// then reads the bitmaps back and goes on alone.  Nothing depends on a helper being there:
-// helpers that find nothing to do leave.
+// - the warps of blocks whose own rows are read or whose context is finished, the warps of
+// blocks launched as helpers only - takes bitmap words (32 rows each) off the END of its list:
+// a block claims one word per warp with one atomic on the context's `back` counter, computes
+// them into the scratch and counts them done.  The owner meanwhile works up from word 0 at its
+// usual pace, looking at `back` before every word; when its warps have met the helpers it closes
+// the counter, waits for the words that running warps still hold, reads the helpers' part of
+// the bitmaps back and goes on alone.  A word may be computed twice where the two meet (the
+// owner sees `back` one word late): both write the same bits, to different places.  Nothing
+// depends on a helper being there: helpers that find nothing to do leave.
 struct ShareDesc {
   long long lo, cnt;       // matched suffix-array range
   int Kp, n_win, nw;       // rows taken, matched length, bitmap words that hold rows
-  int next;                // next word to claim (atomic)
-  int done;                // words finished (atomic)
+  int back;                // helpers hold the words from here to nw (atomic; the owner works up from word 0)
+  int floor;               // words below this one are the owner's, whatever happens
+  int done;                // words finished by helpers (atomic)
   int ntrunc;              // rows cut short by the end of the stream (atomic), listed in the context's trunc array
   int err;                 // REST_CTX_* bits met by the gatherers (atomic)
-  int pad[5];
+  int pad[4];
 };
 static_assert(sizeof(ShareDesc) == 64, "one descriptor per 64 bytes");
 constexpr int kShareRows = 512;         // candidate caps up to this never share (a block has a warp per word)
@@ -326,7 +330,7 @@ struct Smem {
   int ntrunc;
   int counted;                 // shared gathering: this context is counted as past its gather
   int help_b;                  // shared gathering: the context this block helps next
-  int help_base;               // shared gathering: first word of the block's current claim
+  int help_base, help_top;     // shared gathering: the words [base, top) of the block's current claim
   uint32_t trunc[kMaxTrunc];   // len << 16 | row: rows cut short by the end of the token stream
   uint32_t sel[kMaxN];         // depth << 16 | row
   uint32_t selcnt[kMaxN];
@@ -401,8 +405,9 @@ __device__ __forceinline__ int compare_rows(const int32_t* __restrict__ y, int y
 // ---- gather rows, common-prefix lengths, node-start bitmap words -----------------------------
 // Executed by one warp, for the context whose matched range is [lo, lo + cnt), of which Kp rows
 // are taken, behind a match of n_win tokens.  Bitmap word w covers candidate rows 32 w ... 32 w + 31;
-// the warp takes words first_word, first_word + stepw, ... below end_word.  The suffix-array
-// entries of the warp's next word travel while the rows of the current one do.
+// the warp takes words first_word, first_word + stepw, ... below end_word (and below *limit,
+// when given).  The suffix-array entries of the warp's next word travel while the rows of the
+// current one do.
 // Slot 0 of the warp is the row before its first row, slot l + 1 the row of lane l.  A load
 // instruction fetches two slots, 16 columns each (lane = 16 * slot parity + column): the
 // lanes of a row read consecutive tokens, so an instruction touches two rows (a few cache
@@ -419,7 +424,8 @@ template <typename SaT, int PART>
 __device__ __forceinline__ void gather_words(const DraftArgs& a, int b, const int32_t** sb, int* sl, int lane,
                                              int64_t lo, int64_t cnt, int Kp, int n_win, int first_word,
                                              int stepw, int end_word, uint32_t* bm_out, int* ntrunc_out,
-                                             uint32_t* trunc_out, int* err_out, long long* pc, int pc_rows) {
+                                             uint32_t* trunc_out, int* err_out, long long* pc, int pc_rows,
+                                             const int* limit = nullptr, int limit_floor = 0) {
   const int m = a.m, nwords = a.nwords;
   const int nw = end_word;
   const int64_t n_tokens = a.n_tokens;
@@ -469,7 +475,11 @@ __device__ __forceinline__ void gather_words(const DraftArgs& a, int b, const in
   // columns past a row's end read as a value no token has (tokens are below 2^31), different
   // for neighbouring slots: they never compare equal to anything above or below them
   const uint32_t pad = 0x80000000u | (uint32_t)half;
-  while (w < nw) {
+  // limit: words from max(*limit, limit_floor) on belong to somebody else (*limit only ever
+  // falls); read one word ahead
+  int stop = limit ? max(*reinterpret_cast<const volatile int*>(limit), limit_floor) : nw;
+  while (w < nw && w < stop) {
+    const int stop_next = limit ? max(*reinterpret_cast<const volatile int*>(limit), limit_floor) : nw;
     const int jbase = w * 32;
     const int j = jbase + lane;
     const bool valid = j < Kp;
@@ -537,39 +547,8 @@ __device__ __forceinline__ void gather_words(const DraftArgs& a, int b, const in
     if (__any_sync(kFull, bad) && lane == 0) atomicOr(err_out, REST_CTX_BAD_DATASTORE);
     __syncwarp();                  // the slot tables are rewritten by the next word
     w = wn; p = p_next; pp = pp_next;
+    stop = stop_next;
   }
-}
-
-// Executed by a whole block: claims words of context hb's candidate rows, one per warp and
-// round, until none is left; computes them into the context's scratch and counts them done.
-// (One claim per block and round: thousands of warps claiming from one counter wait for one
-// another longer than the rows take.)
-template <typename SaT, int NT>
-__device__ __forceinline__ void share_work_on(const DraftArgs& a, Smem& s, int hb, const int32_t** sb, int* sl,
-                                              int64_t lo, int64_t cnt, int Kp, int n_win) {
-  constexpr int NW = NT / 32;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  ShareDesc* dsc = a.sh_desc + hb;
-  const int nw = (Kp + 31) >> 5;
-  int finished = 0;                      // words of the round before, not yet counted
-  for (;;) {
-    if (tid == 0) {
-      if (finished) atomicAdd(&dsc->done, finished);
-      s.help_base = atomicAdd(&dsc->next, NW);
-    }
-    __syncthreads();
-    const int base = s.help_base;
-    if (base >= nw) break;
-    const int end = min(nw, base + NW);
-    gather_words<SaT, kWholeShare>(a, hb, sb, sl, lane, lo, cnt, Kp, n_win, base + warp, NW, end,
-                                   a.sh_bm + (int64_t)hb * a.m * a.nwords, &dsc->ntrunc,
-                                   a.sh_trunc + (int64_t)hb * kMaxTrunc, &dsc->err, nullptr, 0);
-    __threadfence();                     // the words before the count
-    __syncthreads();
-    finished = end - base;
-  }
-  if (tid == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + hb) = 2;     // every word is claimed
-  __syncthreads();                       // help_base is read by all before anyone rewrites it
 }
 
 // Executed by a whole block: works on the words that other contexts offer until none is left to
@@ -591,7 +570,7 @@ __device__ __forceinline__ void share_help_pass(const DraftArgs& a, Smem& s, con
   for (;;) {
     if (warp == 0) {
       if (finished && lane == 0) atomicAdd(&a.sh_desc[cur].done, finished);
-      int found = -1, base = 0;
+      int found = -1, base = 0, top = 0;
       if (!allowed) allowed = *reinterpret_cast<volatile int32_t*>(a.sh_hdr) >= B;
       int prefer = cur;
       for (int tries = 0; allowed && tries <= B && found < 0; ++tries) {
@@ -608,20 +587,20 @@ __device__ __forceinline__ void share_help_pass(const DraftArgs& a, Smem& s, con
           if (cand < 0) break;
         }
         ShareDesc* dsc = a.sh_desc + cand;
-        const int words = *reinterpret_cast<volatile int*>(&dsc->nw);
-        int at = *reinterpret_cast<volatile int*>(&dsc->next);
-        if (at < words) {
-          if (lane == 0) at = atomicAdd(&dsc->next, NW);
-          at = __shfl_sync(kFull, at, 0);
+        const int floor = *reinterpret_cast<volatile int*>(&dsc->floor);
+        int hi = *reinterpret_cast<volatile int*>(&dsc->back);
+        if (hi > floor) {
+          if (lane == 0) hi = atomicSub(&dsc->back, NW);
+          hi = __shfl_sync(kFull, hi, 0);
         }
-        if (at < words) { found = cand; base = at; }
-        else if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + cand) = 2;     // every word is claimed
+        if (hi > floor) { found = cand; base = max(floor, hi - NW); top = hi; }
+        else if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + cand) = 2;     // every word is taken
       }
       __threadfence();
-      if (lane == 0) { s.help_b = found; s.help_base = base; }
+      if (lane == 0) { s.help_b = found; s.help_base = base; s.help_top = top; }
     }
     __syncthreads();
-    const int found = s.help_b, base = s.help_base;
+    const int found = s.help_b, base = s.help_base, end = s.help_top;
     __syncthreads();
     finished = 0;
     if (found < 0) break;
@@ -634,13 +613,12 @@ __device__ __forceinline__ void share_help_pass(const DraftArgs& a, Smem& s, con
     // a descriptor that makes no sense is left to its owner (the words claimed from it stay
     // uncounted: its owner reports the context as failed)
     const bool sane = Kp > 0 && Kp <= a.kcap && cnt >= (int64_t)Kp && lo >= 0 && lo + cnt <= a.n_sa &&
-                      n_win >= 1 && nw == ((Kp + 31) >> 5) && base >= 0 && base < nw;
+                      n_win >= 1 && nw == ((Kp + 31) >> 5) && base >= 0 && base < end && end <= nw;
     if (!sane) {
       if (tid == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + found) = 2;
       cur = -1;
       continue;
     }
-    const int end = min(nw, base + NW);
     ShareDesc* dsc = a.sh_desc + found;
     gather_words<SaT, kWholeShare>(a, found, sb, sl, lane, lo, cnt, Kp, n_win, base + warp, NW, end,
                                    a.sh_bm + (int64_t)found * a.m * a.nwords, &dsc->ntrunc,
@@ -907,7 +885,8 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   const int32_t** my_sb = reinterpret_cast<const int32_t**>(slot_base + warp * 34);
   int* my_sl = slot_len + warp * 34;
   bool shared_gather = false;
-  if constexpr (PART == kWholeShare) shared_gather = Kp > max(a.share_rows, NT);     // more words than warps
+  // worth it with more words than warps, and with words beyond the rows whose positions stay here
+  if constexpr (PART == kWholeShare) shared_gather = Kp > max(a.share_rows, NT) && nw > ((a.pcache_rows + 31) >> 5);
   if (!shared_gather) {
     // warp w takes words w, w + NW, ...
     gather_words<SaT, PART>(a, b, my_sb, my_sl, lane, lo, cnt, Kp, n_win, warp, NW, nw, bm, &s.ntrunc,
@@ -919,38 +898,52 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
       share_help_pass<SaT, NT>(a, s, my_sb, my_sl, b, true);
     }
   } else {
-    // offer the rows to every idle warp of the launch, and take words like any of them
+    // offer the end of the list to every idle block of the launch and work up from its start
     ShareDesc* dsc = a.sh_desc + b;
+    const int floor = (a.pcache_rows + 31) >> 5;     // the rows whose positions phase 4 wants cached stay here
     if (tid == 0) {
       dsc->lo = lo; dsc->cnt = cnt; dsc->Kp = Kp; dsc->n_win = n_win; dsc->nw = nw;
+      dsc->floor = floor; dsc->back = nw;
       __threadfence();
       *reinterpret_cast<volatile int32_t*>(a.sh_ready + b) = 1;
     }
+    __syncthreads();                                 // `back` is set before any warp looks at it
+    gather_words<SaT, PART>(a, b, my_sb, my_sl, lane, lo, cnt, Kp, n_win, warp, NW, nw, bm, &s.ntrunc,
+                            s.trunc, &s.err, pcache, a.pcache_rows, &dsc->back, floor);
     __syncthreads();
-    share_work_on<SaT, NT>(a, s, b, my_sb, my_sl, lo, cnt, Kp, n_win);
     if (tid == 0) {
+      // close: what the helpers hold now is all they will ever hold
+      int from = atomicExch(&dsc->back, 0);
+      from = max(floor, min(from, nw));
+      *reinterpret_cast<volatile int32_t*>(a.sh_ready + b) = 2;
       atomicAdd(a.sh_hdr + 1, 1); s.counted = 1;
-      // words still out are in the hands of running warps
       int polls = 0;
-      while (*reinterpret_cast<volatile int*>(&dsc->done) < nw && polls < kOwnerPolls) { __nanosleep(100); ++polls; }
+      while (*reinterpret_cast<volatile int*>(&dsc->done) < nw - from && polls < kOwnerPolls) { __nanosleep(100); ++polls; }
       __threadfence();
       int e = *reinterpret_cast<volatile int*>(&dsc->err);
-      if (*reinterpret_cast<volatile int*>(&dsc->done) < nw) e |= REST_CTX_INTERNAL;
+      if (*reinterpret_cast<volatile int*>(&dsc->done) < nw - from) e |= REST_CTX_INTERNAL;
       if (e) atomicOr(&s.err, e);
-      s.ntrunc = *reinterpret_cast<volatile int*>(&dsc->ntrunc);
+      s.help_base = from;
+      s.help_top = min(max(*reinterpret_cast<volatile int*>(&dsc->ntrunc), 0), kMaxTrunc);
     }
     __syncthreads();
     if (s.err == 0) {
+      // the helpers' part of the bitmaps, and the short rows they met
+      const int from = s.help_base, nhelped = nw - from, ntr = s.help_top;
       const uint32_t* gbm = a.sh_bm + (int64_t)b * m * nwords;
 #pragma unroll 4
-      for (int i = tid; i < m * nw; i += NT) {
-        const int d = i / nw, w = i - d * nw;
+      for (int i = tid; i < m * nhelped; i += NT) {
+        const int d = i / nhelped, w = from + i - d * nhelped;
         bm[d * nwords + w] = __ldcg(gbm + d * nwords + w);
       }
-      if (tid < min(s.ntrunc, kMaxTrunc)) s.trunc[tid] = __ldcg(a.sh_trunc + (int64_t)b * kMaxTrunc + tid);
+      if (tid < ntr) {
+        const int at = atomicAdd(&s.ntrunc, 1);
+        if (at < kMaxTrunc) s.trunc[at] = __ldcg(a.sh_trunc + (int64_t)b * kMaxTrunc + tid);
+        else atomicOr(&s.err, REST_CTX_INTERNAL);
+      }
     }
   }
-  const int pcache_rows = shared_gather ? 0 : a.pcache_rows;   // rows whose position phase 4 finds in shared memory
+  const int pcache_rows = a.pcache_rows;   // rows whose position phase 4 finds in shared memory
   if (tid < m) bm[tid * nwords + ((Kp + 31) >> 5)] = kFull;   // sentinel past the last row
   __syncthreads();
   if (s.err != 0) {
