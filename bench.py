@@ -16,6 +16,7 @@ deliberately plain program) on a bounded sample of the same workload.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import math
 import os
@@ -64,6 +65,10 @@ def parse_args():
     ap.add_argument("--workload", default="auto", choices=["auto"] + list(datagen.WORKLOADS))
     ap.add_argument("--n-tokens", type=int, default=None,
                     help="override the datastore size (debugging only; changes the workload name)")
+    ap.add_argument("--e2e-chunks", default=None,
+                    help="end-to-end leg: sizes of the context chunks whose copies overlap the compute of "
+                         "their neighbours, e.g. 32,32,32,32 (default: B/8, 3B/8, 3B/8, B/8 for a single-layer "
+                         "step of 64 contexts or more, else one chunk)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-workloads", action="store_true",
                     help="skip the table of the other workloads and the sweeps")
@@ -661,8 +666,19 @@ def run_ours(args, rank, world, local_rank):
     # A single layer over a large batch has no second layer to hide its copies behind: the batch
     # is then cut into chunks of contexts (one attention call each), so that the queries of
     # chunk i + 1 arrive and the outputs of chunk i - 1 leave while chunk i is computed.
-    n_chunks = 4 if (layers == 1 and B >= 64) else 1
-    bounds = [(c * B // n_chunks, (c + 1) * B // n_chunks) for c in range(n_chunks)]
+    # The first chunk's queries and the last chunk's outputs cannot hide behind anything: those two
+    # chunks are small (an eighth of the batch each), the two in between large.
+    if layers == 1 and B >= 64:
+        edges = [0, B // 8, B // 2, B - B // 8, B]
+        bounds = list(zip(edges[:-1], edges[1:]))
+    else:
+        bounds = [(0, B)]
+    if args.e2e_chunks:                      # explicit chunk sizes (contexts), e.g. 16,48,48,16
+        sizes = [int(x) for x in args.e2e_chunks.split(",")]
+        if sum(sizes) != B or min(sizes) < 1:
+            raise SystemExit("--e2e-chunks must be positive sizes that add up to the contexts per step")
+        edges = np.cumsum([0] + sizes).tolist()
+        bounds = list(zip(edges[:-1], edges[1:]))
 
     def e2e_calls(_):
         main = torch.cuda.current_stream()
@@ -850,6 +866,11 @@ def other_workloads(rest, torch, dev, headline, headline_T, headline_ds, headlin
             row["note"] = "not enough free device memory for this datastore"
         row["attention"] = time_attention(rest, torch, w0, dev, peak=peak)
         rows.append(row)
+
+    # the largest tree the library takes (N = 256: two 128-row blocks per head) on the stress shape
+    w256 = dataclasses.replace(datagen.WORKLOADS["stress"], N=256)
+    rows.append({"workload": "stress shape with N = 256 draft rows (attention only)",
+                 "attention": time_attention(rest, torch, w256, dev, peak=peak)})
 
     # datastore-size sweep on the batched recipe: shorter streams are prefixes of the longest one
     wb = datagen.WORKLOADS["batched"]

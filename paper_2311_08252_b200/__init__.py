@@ -247,7 +247,7 @@ def alloc_draft_output(B: int, N: int, device) -> DraftOutput:
 def draft_workspace_bytes(B: int, n_max=16, n_min=2, K=5000, m=10, N=64,
                           sample_mode=REST_SAMPLE_STRIDED, search=REST_SEARCH_AUTO) -> int:
     """Scratch bytes rest_draft can use for a call of B contexts on the current device (0 when
-    the call takes the single-context path)."""
+    a scratch would not make the call faster)."""
     prm = _Params(n_max, n_min, K, m, N, sample_mode, search)
     return int(lib().rest_draft_workspace_bytes(ctypes.byref(prm), B))
 

@@ -210,3 +210,36 @@ def test_random_parameters_against_the_oracle():
         got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=search, index=index, **kw)
         assert_draft_equal(got, ref, f"case {case}: vocab {vocab}, {n_tok} tokens, {kw}, search {search:#x}, "
                                      f"index {index}")
+
+
+@pytest.mark.parametrize("B", [2, 40, 200])
+def test_long_candidate_lists_shared_between_blocks(B):
+    """Contexts whose candidate lists run into the thousands hand part of their rows to idle
+    blocks through the caller's scratch (fewer contexts than SMs: blocks that only help; more:
+    blocks that help once their own context is done).  Same trees as the oracle, with the scratch
+    the library asks for, with a scratch full of ones from an earlier use, and without one."""
+    import torch
+    from gpu_util import to_dev
+    rng = np.random.default_rng(100 + B)
+    vocab, n_tok, Lc = 2, 60000, 24
+    T = rng.integers(0, vocab, n_tok).astype(np.int32)
+    sa = datagen.build_suffix_array(T, vocab, W=32, sa_bytes=4)
+    ctx = rng.integers(0, vocab, (B, Lc)).astype(np.int32)
+    # short contexts: their longest matching suffix is the whole context, with thousands of matches
+    ctx_len = np.resize(np.array([3, 4, 2, 9, Lc, 5, 12, 3, 7, Lc], np.int32), B)
+    ctx[1, :4] = T[n_tok - 6:n_tok - 2]                     # one of its rows is cut short by the end of the stream
+    for K, m, N, mode in ((20000, 16, 128, 0), (5000, 10, 64, 1), (3000, 5, 256, 0)):
+        kw = dict(K=K, m=m, N=N, sample_mode=mode)
+        ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
+        hits = ref["match_range"][:, 1] - ref["match_range"][:, 0]
+        assert (hits > 2048).sum() >= min(B, 2) and (hits < 512).sum() >= (1 if B > 3 else 0)
+        need = rest.draft_workspace_bytes(B, **{k: v for k, v in kw.items() if k != "sample_mode"})
+        assert need > 0
+        dirty = torch.full((need,), 0xFF, dtype=torch.uint8, device="cuda:0")
+        for workspace in (None, dirty, False):
+            got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, search=rest.REST_SEARCH_SINGLE,
+                               workspace=workspace, **kw)
+            assert_draft_equal(got, ref, f"B {B}, K {K}, workspace {type(workspace).__name__}")
+        # the same scratch again, straight after a call that used it
+        got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, search=rest.REST_SEARCH_SINGLE, workspace=dirty, **kw)
+        assert_draft_equal(got, ref, f"B {B}, K {K}, scratch reused")
