@@ -122,7 +122,7 @@ struct ShareDesc {
   long long lo, cnt;       // matched suffix-array range
   int Kp, n_win, nw;       // rows taken, matched length, bitmap words that hold rows
   int back;                // helpers hold the words from here to nw (atomic; the owner works up from word 0)
-  int floor;               // words below this one are the owner's, whatever happens
+  int floor;               // words below this one are the owner's, whatever happens (set once, before the context opens)
   int done;                // words finished by helpers (atomic)
   int ntrunc;              // rows cut short by the end of the stream (atomic), listed in the context's trunc array
   int err;                 // REST_CTX_* bits met by the gatherers (atomic)
@@ -406,7 +406,7 @@ __device__ __forceinline__ int compare_rows(const int32_t* __restrict__ y, int y
 // Executed by one warp, for the context whose matched range is [lo, lo + cnt), of which Kp rows
 // are taken, behind a match of n_win tokens.  Bitmap word w covers candidate rows 32 w ... 32 w + 31;
 // the warp takes words first_word, first_word + stepw, ... below end_word (and below *limit,
-// when given).  The suffix-array entries of the warp's next word travel while the rows of the
+// when given; see the shared gather).  The suffix-array entries of the warp's next word travel while the rows of the
 // current one do.
 // Slot 0 of the warp is the row before its first row, slot l + 1 the row of lane l.  A load
 // instruction fetches two slots, 16 columns each (lane = 16 * slot parity + column): the
@@ -587,6 +587,8 @@ __device__ __forceinline__ void share_help_pass(const DraftArgs& a, Smem& s, con
           if (cand < 0) break;
         }
         ShareDesc* dsc = a.sh_desc + cand;
+        // take the NW words below `back` (fewer when that reaches under the floor, the words
+        // that must be the owner's own)
         const int floor = *reinterpret_cast<volatile int*>(&dsc->floor);
         int hi = *reinterpret_cast<volatile int*>(&dsc->back);
         if (hi > floor) {
@@ -885,6 +887,7 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
   const int32_t** my_sb = reinterpret_cast<const int32_t**>(slot_base + warp * 34);
   int* my_sl = slot_len + warp * 34;
   bool shared_gather = false;
+  int own_words = nw;                  // bitmap words whose rows this block read itself
   // worth it with more words than warps, and with words beyond the rows whose positions stay here
   if constexpr (PART == kWholeShare) shared_gather = Kp > max(a.share_rows, NT) && nw > ((a.pcache_rows + 31) >> 5);
   if (!shared_gather) {
@@ -927,9 +930,10 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
       s.help_top = min(max(*reinterpret_cast<volatile int*>(&dsc->ntrunc), 0), kMaxTrunc);
     }
     __syncthreads();
+    own_words = s.help_base;
     if (s.err == 0) {
       // the helpers' part of the bitmaps, and the short rows they met
-      const int from = s.help_base, nhelped = nw - from, ntr = s.help_top;
+      const int from = own_words, nhelped = nw - from, ntr = s.help_top;
       const uint32_t* gbm = a.sh_bm + (int64_t)b * m * nwords;
 #pragma unroll 4
       for (int i = tid; i < m * nhelped; i += NT) {
@@ -943,7 +947,8 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
       }
     }
   }
-  const int pcache_rows = a.pcache_rows;   // rows whose position phase 4 finds in shared memory
+  // rows whose position phase 4 finds in shared memory (only rows this block read itself)
+  const int pcache_rows = min(a.pcache_rows, own_words * 32);
   if (tid < m) bm[tid * nwords + ((Kp + 31) >> 5)] = kFull;   // sentinel past the last row
   __syncthreads();
   if (s.err != 0) {
