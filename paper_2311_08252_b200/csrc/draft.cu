@@ -123,12 +123,14 @@ struct ShareDesc {
   int Kp, n_win, nw;       // rows taken, matched length, bitmap words that hold rows
   int back;                // helpers hold the words from here to nw (atomic; the owner works up from word 0)
   int floor;               // words below this one are the owner's, whatever happens (set once, before the context opens)
+  int front;               // how far the owner will get before a helper could finish a claim made now (it rises)
   int done;                // words finished by helpers (atomic)
   int ntrunc;              // rows cut short by the end of the stream (atomic), listed in the context's trunc array
   int err;                 // REST_CTX_* bits met by the gatherers (atomic)
-  int pad[4];
+  int pad[3];
 };
 static_assert(sizeof(ShareDesc) == 64, "one descriptor per 64 bytes");
+constexpr int kShareMargin = 2;         // rounds (a word per warp) an owner gets through while a helper finishes one claim
 constexpr int kShareRows = 512;         // candidate caps up to this never share (a block has a warp per word)
 // a single context does not share: the few microseconds that zeroing the counters and the look-outs
 // cost every call outweigh what the occasional long list gains
@@ -425,7 +427,8 @@ __device__ __forceinline__ void gather_words(const DraftArgs& a, int b, const in
                                              int64_t lo, int64_t cnt, int Kp, int n_win, int first_word,
                                              int stepw, int end_word, uint32_t* bm_out, int* ntrunc_out,
                                              uint32_t* trunc_out, int* err_out, long long* pc, int pc_rows,
-                                             const int* limit = nullptr, int limit_floor = 0) {
+                                             const int* limit = nullptr, int limit_floor = 0,
+                                             int* front_out = nullptr) {
   const int m = a.m, nwords = a.nwords;
   const int nw = end_word;
   const int64_t n_tokens = a.n_tokens;
@@ -476,10 +479,12 @@ __device__ __forceinline__ void gather_words(const DraftArgs& a, int b, const in
   // for neighbouring slots: they never compare equal to anything above or below them
   const uint32_t pad = 0x80000000u | (uint32_t)half;
   // limit: words from max(*limit, limit_floor) on belong to somebody else (*limit only ever
-  // falls); read one word ahead
+  // falls); read one word ahead.  front_out: where this warp tells helpers how far it will be
+  // by the time a claim made now could be finished (a hint: claims below it are not worth making)
   int stop = limit ? max(*reinterpret_cast<const volatile int*>(limit), limit_floor) : nw;
   while (w < nw && w < stop) {
     const int stop_next = limit ? max(*reinterpret_cast<const volatile int*>(limit), limit_floor) : nw;
+    if (front_out && lane == 0) *reinterpret_cast<volatile int*>(front_out) = w + kShareMargin * stepw;
     const int jbase = w * 32;
     const int j = jbase + lane;
     const bool valid = j < Kp;
@@ -589,11 +594,16 @@ __device__ __forceinline__ void share_help_pass(const DraftArgs& a, Smem& s, con
         ShareDesc* dsc = a.sh_desc + cand;
         // take the NW words below `back` (fewer when that reaches under the floor, the words
         // that must be the owner's own)
+        // ... and none at all when the owner will be there before this block could finish them: it
+        // would only have to wait for them
         const int floor = *reinterpret_cast<volatile int*>(&dsc->floor);
+        const int front = *reinterpret_cast<volatile int*>(&dsc->front);
         int hi = *reinterpret_cast<volatile int*>(&dsc->back);
-        if (hi > floor) {
+        if (hi > floor && hi - NW >= front) {
           if (lane == 0) hi = atomicSub(&dsc->back, NW);
           hi = __shfl_sync(kFull, hi, 0);
+        } else {
+          hi = 0;
         }
         if (hi > floor) { found = cand; base = max(floor, hi - NW); top = hi; }
         else if (lane == 0) *reinterpret_cast<volatile int32_t*>(a.sh_ready + cand) = 2;     // every word is taken
@@ -912,7 +922,7 @@ __device__ __forceinline__ void draft_block(const DraftArgs& a, unsigned char* s
     }
     __syncthreads();                                 // `back` is set before any warp looks at it
     gather_words<SaT, PART>(a, b, my_sb, my_sl, lane, lo, cnt, Kp, n_win, warp, NW, nw, bm, &s.ntrunc,
-                            s.trunc, &s.err, pcache, a.pcache_rows, &dsc->back, floor);
+                            s.trunc, &s.err, pcache, a.pcache_rows, &dsc->back, floor, warp == 0 ? &dsc->front : nullptr);
     __syncthreads();
     if (tid == 0) {
       // close: what the helpers hold now is all they will ever hold
