@@ -1,28 +1,30 @@
 // rest_draft: Algorithm 1 (longest-suffix retrieval over a suffix array), Algorithm 2
 // (Trie weights and the c heaviest nodes) and the breadth-first pseudo sequence with its
-// ancestor mask (Sec. 3.2), one thread block per context, everything in one launch.
+// ancestor mask (Sec. 3.2), one thread block per context, everything in one launch (three
+// for calls with thousands of contexts).
 //
 // Phases inside the block:
-//   1 search   a warp per suffix length: the bucket index (when the datastore has one) gives the
-//              suffix-array range of the query's first token pair, a 32-ary lower bound inside
-//              it (every lane probes one slot per round, a ballot narrows the interval) finds
-//              the first match, and for the longest length that matched a galloping + 32-ary
-//              upper bound finds the end of the run.
+//   1 search   a warp per suffix length.  The datastore's n-gram index (when it has one) gives
+//              the suffix-array range of the query's first two to four tokens in one read - the
+//              answer itself for a short frequent suffix - and a 32-ary lower bound inside it
+//              (every lane probes one slot per round, a ballot narrows the interval) finds the
+//              first match.  Its probes also bracket the end of the run; only the longest
+//              length that matched searches inside its bracket for the end.
 //   2 gather   candidate rows in suffix-array order, which is also the lexicographic order of
-//              the continuations.  A warp fetches its 32 rows (and the row before them) with
-//              coalesced loads: lane l reads word l, 32 + l, ... of the rows laid end to end,
-//              so a load touches three or four rows instead of 32, and the rows pass through
-//              a shared-memory staging area.  Only the common-prefix length with the previous
+//              the continuations.  A warp takes 32 rows (one bitmap word) at a time; a load
+//              instruction fetches two rows, 16 columns each, and every token is compared with
+//              the one above it where it sits.  Only the common-prefix length with the previous
 //              row survives: for every depth d the bitmap "row j starts a new Trie node at
-//              depth d" (lcp_j < d).
+//              depth d" (lcp_j < d).  A context with thousands of rows shares them with blocks
+//              that have nothing else to do (see ShareDesc).
 //   3 select   weight of node (d, j) = distance to the next set bit of bitmap d.  All passes
-//              run over (depth, bitmap word) pairs, not over rows: two adjacent set bits are a
-//              node of weight 1 (counted with one popcount per word), a set bit followed by a
-//              clear one is a heavier node (visited one by one).  The N largest by (weight
-//              desc, depth asc, row asc) come from a two-level radix histogram over (weight,
-//              depth) and a prefix sum over the words of the tie depth.
-//   4 emit     rank the kept nodes by (depth, row), look up parents through the bitmap of the
-//              depth above, build ancestor masks, fetch the node tokens.
+//              run over (depth, bitmap word) pairs, not over rows: nodes of weight 1 to 4 are
+//              read off the bit pattern of a word and counted with a popcount each, heavier
+//              nodes are listed and weighed by a thread each.  The N largest by (weight desc,
+//              depth asc, row asc) come from a two-level radix histogram over (weight, depth)
+//              and a prefix sum over the words of the tie depth.
+//   4 emit     rank the kept nodes by (depth, row), find parents by a predecessor search among
+//              them, build ancestor masks, fetch the node tokens.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
