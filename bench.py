@@ -53,7 +53,7 @@ NCU_TRAFFIC_PER_UNIT = {
 # The same for the draft kernel of the single-context path: DRAM bytes of one launch per candidate
 # row gathered (stress recipe, 100 M tokens, B = 128, 2409 rows per context on average; the rows
 # and their suffix-array entries are nearly all of the traffic, so it grows with the rows).
-NCU_DRAFT_TRAFFIC_PER_ROW = {"stress": (73.87e6 + 2.48e6) / (128 * 2408.6)}
+NCU_DRAFT_TRAFFIC_PER_ROW = {"stress": (73.84e6 + 2.52e6) / (128 * 2408.6)}
 
 
 def parse_args():
