@@ -84,6 +84,14 @@ def parse_args():
     return ap.parse_args()
 
 
+def measured_tensor_peak():
+    """Sustained dense bf16 TFLOP/s of the measured-peaks file (fallback: 1400)."""
+    try:
+        return float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1400.0, "fallback"
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -358,6 +366,11 @@ def time_attention(rest, torch, w, dev, B=None, iters=12, peak=6650.0, budget_gb
            "target_50pct_met": bool(alg / us / 1e3 / peak >= 0.5),
            "traffic": None if per_unit is None else per_unit * B * H,
            "plan": rest.tree_attention_plan(B, H, N, D, L + N)}
+    # the same launch against the tensor roofline (S = Q K^T and O = P V: 4 N D (L + N) flops per
+    # (context, head)): wide trees are bound by both
+    tpeak, tkind = measured_tensor_peak()
+    tflops = 4.0 * N * D * (L + N) * H * B / us / 1e6
+    res.update({"tensor_tflops": tflops, "frac_of_tensor_sustained": tflops / tpeak, "tensor_peak_kind": tkind})
     del bufs, q, out, ws, graph
     torch.cuda.empty_cache()
     return res
