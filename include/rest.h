@@ -166,11 +166,12 @@ rest_status rest_datastore_create_shard(const int32_t* d_tokens, uint64_t n_toke
  *                query answers for the current device and may be 0).  Never needed for the
  *                results, only for speed; with NULL or fewer bytes every path runs as one launch
  *                of one block per context.  What it buys:
- *                - single-context path, 2 to 1024 contexts, K > 512: a context with a long
- *                  candidate list lets idle blocks (those of finished or lighter contexts, and
- *                  blocks started on SMs that have no context) read part of its rows; the scratch
- *                  holds the contexts' counters and node-start bitmaps (about 6 m K / 32 bytes
- *                  per context).  The call zeroes the counters itself.
+ *                - single-context path, 2 to 1024 contexts (48 to 1024 when K < 8192; never when
+ *                  K <= 512): a context with a long candidate list lets idle blocks (those of
+ *                  finished or lighter contexts, and blocks started on SMs that have no context)
+ *                  read part of its rows; the scratch holds the contexts' counters and
+ *                  node-start bitmaps (about 6 m K / 32 bytes per context).  The call zeroes the
+ *                  counters itself.
  *                - batched path: three launches (search; build of the contexts with few
  *                  candidates on small blocks; build of the others on large blocks); the scratch
  *                  holds the two context lists (8 bytes per context).

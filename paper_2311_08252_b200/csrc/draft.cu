@@ -134,10 +134,19 @@ struct ShareDesc {
 static_assert(sizeof(ShareDesc) == 64, "one descriptor per 64 bytes");
 constexpr int kShareMargin = 2;         // rounds (a word per warp) an owner gets through while a helper finishes one claim
 constexpr int kShareRows = 512;         // candidate caps up to this never share (a block has a warp per word)
-// a single context does not share: the few microseconds that zeroing the counters and the look-outs
-// cost every call outweigh what the occasional long list gains
+// Sharing costs every call a few microseconds (zeroing the counters, a grid of at least one block
+// per SM, the look-outs), which the occasional long list must win back.  Measured on 100 M-token
+// datastores: with a candidate cap of 20000 it pays from two contexts on (2: 38 -> 31 us,
+// 16: 94 -> 50 us), with a cap of 5000 only from about 64 contexts on (2: 20 -> 26 us, 32: 31 ->
+// 34 us, 64: equal, 128: 48 -> 43 us); a single context never shares.
 constexpr int kShareMinContexts = 2;
-constexpr int kShareMaxContexts = 1024;  // calls with more contexts do not share (and take the batched path anyway)
+constexpr int kShareMaxContexts = 1024;
+constexpr int kShareLongCap = 8192;     // candidate caps from here on share whatever the batch
+constexpr int kShareFromContexts = 48;  // shorter caps share from this many contexts on
+static bool wants_share(int K, int B) {
+  return K > kShareRows && B >= kShareMinContexts && B <= kShareMaxContexts &&
+         (K >= kShareLongCap || B >= kShareFromContexts);
+}  // calls with more contexts do not share (and take the batched path anyway)
 constexpr int kShareHdr = 16;           // int32 counters ahead of the per-context arrays: [0] blocks started, [1] contexts past their gather
 constexpr int kHelperPolls = 20000;     // idle polls (>= 200 ns each) after which a helper leaves
 constexpr int kOwnerPolls = 1 << 20;    // polls after which an owner gives up on claimed chunks (REST_CTX_INTERNAL)
@@ -1444,7 +1453,7 @@ extern "C" size_t rest_draft_workspace_bytes(const rest_draft_params* prm, int32
   if (wants_batched(prm->search_path, B, true, &batched) != REST_OK) return 0;
   if (batched) return split_workspace_bytes(B);
   // the one-launch form: scratch for shared gathering, where it can help
-  if (prm->K <= kShareRows || B < kShareMinContexts || B > kShareMaxContexts || prm->m < 1 || prm->m > REST_MAX_M || prm->K > REST_MAX_K) return 0;
+  if (!wants_share(prm->K, B) || prm->m < 1 || prm->m > REST_MAX_M || prm->K > REST_MAX_K) return 0;
   int nwords = 0;
   draft_smem_bytes(prm->K, prm->m, kThreads, nullptr, &nwords, nullptr, nullptr);
   return share_layout(B, prm->m, nwords).bytes;
@@ -1517,7 +1526,7 @@ extern "C" rest_status rest_draft(const rest_datastore* ds, const rest_draft_par
     // every block of the launch is resident at once).
     const ShareLayout lay = share_layout(B, prm->m, a.nwords);
     const bool share = d_ws && ws_bytes >= lay.bytes && reinterpret_cast<uintptr_t>(d_ws) % 16 == 0 &&
-                       prm->K > kShareRows && B >= kShareMinContexts && B <= kShareMaxContexts;
+                       wants_share(prm->K, B);
     if (share) {
       unsigned char* ws = static_cast<unsigned char*>(d_ws);
       a.sh_hdr = reinterpret_cast<int32_t*>(ws);

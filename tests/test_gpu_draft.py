@@ -100,8 +100,10 @@ def test_more_contexts_than_the_gpu_holds_at_once():
         got, _ = gpu_draft(T, sa, w.vocab, ctx, ctx_len, search=search, workspace=False, **kw)
         assert_draft_equal(got, ref, f"one launch, search {search:#x}")
     assert rest.draft_workspace_bytes(B, **kw) >= 8 * B
-    # few contexts: scratch only for sharing the gather of long candidate lists
-    assert rest.draft_workspace_bytes(8, **kw) > 0 and rest.draft_workspace_bytes(8, K=512, m=w.m, N=w.N) == 0
+    # fewer contexts: scratch only where sharing the gather of long candidate lists pays
+    assert rest.draft_workspace_bytes(64, **kw) > 0 and rest.draft_workspace_bytes(8, **kw) == 0
+    assert rest.draft_workspace_bytes(8, K=20000, m=w.m, N=w.N) > 0
+    assert rest.draft_workspace_bytes(64, K=512, m=w.m, N=w.N) == 0 and rest.draft_workspace_bytes(1, K=20000) == 0
     assert len(set(ref["match_n"].tolist())) > 8          # matched lengths all over 2 ... 16
     with pytest.raises(rest.RestError):
         gpu_draft(T, sa, w.vocab, ctx[:2], ctx_len[:2], search=0x400, **kw)
@@ -228,14 +230,14 @@ def test_long_candidate_lists_shared_between_blocks(B):
     # short contexts: their longest matching suffix is the whole context, with thousands of matches
     ctx_len = np.resize(np.array([3, 4, 2, 9, Lc, 5, 12, 3, 7, Lc], np.int32), B)
     ctx[1, :4] = T[n_tok - 6:n_tok - 2]                     # one of its rows is cut short by the end of the stream
-    for K, m, N, mode in ((20000, 16, 128, 0), (5000, 10, 64, 1), (3000, 5, 256, 0)):
+    for K, m, N, mode in ((20000, 16, 128, 0), (8192, 10, 64, 1), (3000, 5, 256, 0)):
         kw = dict(K=K, m=m, N=N, sample_mode=mode)
         ref = oracle.draft(T, sa, vocab, ctx, ctx_len, **kw)
         hits = ref["match_range"][:, 1] - ref["match_range"][:, 0]
         assert (hits > 2048).sum() >= min(B, 2) and (hits < 512).sum() >= (1 if B > 3 else 0)
         need = rest.draft_workspace_bytes(B, **{k: v for k, v in kw.items() if k != "sample_mode"})
-        assert need > 0
-        dirty = torch.full((need,), 0xFF, dtype=torch.uint8, device="cuda:0")
+        assert (need > 0) == (K >= 8192 or B >= 48)      # where the library expects sharing to pay
+        dirty = torch.full((max(need, 16),), 0xFF, dtype=torch.uint8, device="cuda:0")
         for workspace in (None, dirty, False):
             got, _ = gpu_draft(T, sa, vocab, ctx, ctx_len, validate=True, search=rest.REST_SEARCH_SINGLE,
                                workspace=workspace, **kw)
